@@ -1,0 +1,173 @@
+/*
+ * fedattn.h -- C ABI of the FedAttn attention hot path for NVIDIA B200 (sm_100a).
+ *
+ * FedAttn (federated attention): N participants each hold a contiguous segment of a global
+ * token sequence.  In most Transformer blocks every participant runs causal self-attention
+ * over its own segment only (fedattn_local).  Every H-th block the participants' K/V are
+ * aggregated -- concatenated in participant order, or sparsified (fedattn_aggregate_kv) --
+ * and each participant's queries attend over the aggregated KV under the global-position
+ * causal mask (fedattn_sync).  Cached K/V are reused for one-token decoding (fedattn_decode).
+ *
+ * Conventions for every call
+ *   - "dev" pointers are device memory on the context's device; "host" pointers are ordinary
+ *     host memory that is read before the call returns.  The caller owns every buffer,
+ *     including the workspace.  Unless a function says otherwise it allocates nothing and
+ *     frees nothing.
+ *   - Work is enqueued on the given stream (a cudaStream_t passed as void*; NULL = default
+ *     stream) and the call returns without synchronising.
+ *   - Errors are return codes.  Arguments are validated on the host before anything is
+ *     launched; a rejected call launches nothing.  A device-side anomaly (a bounded wait that
+ *     ran out, an out-of-range index in INDEXED mode) sets a status word in the workspace that
+ *     fedattn_poll reads; the kernel still terminates and the context stays usable.
+ *   - Layouts are row-major with head_dim contiguous.  Packed queries Q[L, Hq, d]; packed keys
+ *     and values K,V[L, Hkv, d]; L = sum of segment lengths; query head h reads KV head
+ *     h / (Hq / Hkv).  dtype is FEDATTN_F32 or FEDATTN_BF16 for all of Q, K, V, O of a call;
+ *     lse is always float.  Softmax and accumulation are fp32.
+ *   - One context serves one stream at a time: calls that share a context and may overlap on
+ *     the GPU race on its workspace.
+ */
+#ifndef FEDATTN_H_
+#define FEDATTN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define FEDATTN_MAX_PARTICIPANTS 64
+#define FEDATTN_MAX_HEAD_DIM 128
+
+typedef struct fedattn_ctx fedattn_ctx; /* opaque */
+typedef void *fedattn_stream;           /* a cudaStream_t */
+
+typedef enum {
+    FEDATTN_OK = 0,
+    FEDATTN_ERR_INVALID_ARG = 1, /* null pointer, bad shape, non-monotone cu_seqlens, k_sel > L_n ... */
+    FEDATTN_ERR_UNSUPPORTED = 2, /* valid request this build has no kernel for */
+    FEDATTN_ERR_WORKSPACE = 3,   /* workspace missing, misaligned or too small */
+    FEDATTN_ERR_CUDA = 4,        /* a CUDA runtime/driver call failed */
+    FEDATTN_ERR_TIMEOUT = 5,     /* device status: a bounded wait inside a kernel ran out */
+    FEDATTN_ERR_INDEX = 6        /* device status: INDEXED selection index out of range */
+} fedattn_status;
+
+typedef enum { FEDATTN_F32 = 0, FEDATTN_BF16 = 1 } fedattn_dtype;
+
+typedef struct {
+    int32_t n_participants; /* N, 1..FEDATTN_MAX_PARTICIPANTS */
+    int32_t n_q_heads;      /* Hq */
+    int32_t n_kv_heads;     /* Hkv, divides Hq */
+    int32_t head_dim;       /* d, multiple of 8, <= FEDATTN_MAX_HEAD_DIM */
+    int32_t dtype;          /* fedattn_dtype */
+    int32_t causal;         /* 1 = decoder (masked) attention, 0 = bidirectional */
+    float scale;            /* softmax scale; 0 selects 1/sqrt(head_dim) */
+} fedattn_shape;
+
+/* ---- context ------------------------------------------------------------------------------ */
+
+/* Bytes of workspace the calls below need for this shape when no call handles more than
+ * max_total_tokens query rows or max_total_kv aggregated KV rows.  Returns 0 for a bad shape. */
+size_t fedattn_workspace_bytes(const fedattn_shape *shape, int64_t max_total_tokens,
+                               int64_t max_total_kv);
+
+/* Creates a context on `device` around a caller-owned dev workspace (256-byte aligned).  The
+ * workspace's first bytes hold the device status word, which this call clears (the only
+ * synchronous device operation besides fedattn_poll).  Host memory for the context itself is
+ * allocated here and released by fedattn_destroy; the workspace is never freed. */
+fedattn_status fedattn_create(fedattn_ctx **ctx, int device, void *workspace, size_t workspace_bytes);
+void fedattn_destroy(fedattn_ctx *ctx);
+const char *fedattn_status_string(fedattn_status s);
+
+/* Synchronises `stream`, returns the device status word (FEDATTN_OK when no kernel reported
+ * an anomaly) and clears it. */
+fedattn_status fedattn_poll(fedattn_ctx *ctx, fedattn_stream stream);
+
+/* Number of kernels this context has launched so far (for launch accounting). */
+int64_t fedattn_launch_count(const fedattn_ctx *ctx);
+
+/* ---- local attention: Phase I, o_n = Attention(q_n, k_n, v_n) ----------------------------------
+ * Paper: Sec. IV-B "Phase I: Local Self-Attention", eq. (update_local_o), Algorithm 1 inner loop;
+ * causal mask of Sec. III-B read as "key j allowed for query i iff j <= i" (self included).
+ * Row i of segment n (cu_seqlens[n] <= i < cu_seqlens[n+1]) attends keys cu_seqlens[n] .. i
+ * (the whole segment when shape->causal == 0).
+ *   q dev [L,Hq,d]; k, v dev [L,Hkv,d]; cu_seqlens_host host int32 [N+1], cu[0] = 0, non-decreasing,
+ *   cu[N] = L (zero-length segments allowed); o dev [L,Hq,d] written; lse dev float [L,Hq] or NULL
+ *   (natural-log-sum-exp of the scaled logits). */
+fedattn_status fedattn_local(fedattn_ctx *ctx, const fedattn_shape *shape,
+                             const void *q, const void *k, const void *v,
+                             const int32_t *cu_seqlens_host,
+                             void *o, float *lse, fedattn_stream stream);
+
+/* ---- KV aggregation: [K V] = sum_n Pi_n [k_n v_n] ---------------------------------------------
+ * Paper: Sec. IV-B Phase II eq. (update_global_kv_H), Algorithm 1 exchange step (dense); Sec. V
+ * Observation "Aggregation method": sparse KV exchange / adaptive KV aggregation pi_n(t) with
+ * L'_n(t) subset of L_n (TOPK_KNORM, INDEXED; k_sel[n] = 0 excludes participant n).
+ *
+ *   FEDATTN_AGG_CONCAT      k_agg, v_agg dev [L,Hkv,d]: participant n's rows copied to rows
+ *                           off_n .. off_n+L_n-1.  kv_pos dev int32 [L] = 0..L-1.  cu_kv = off.
+ *   FEDATTN_AGG_TOPK_KNORM  per participant and per KV head keep the k_sel[n] rows with the
+ *                           largest score s = sum_c k[j,h,c]^2 (fp64, c increasing); equal scores:
+ *                           lower index first.  Kept rows are emitted in ascending index order.
+ *   FEDATTN_AGG_INDEXED     as TOPK but the kept local indices are given in sel_idx_in
+ *                           (dev int32 [Hkv, T], T = sum k_sel, block n at cu_kv[n], ascending).
+ *   Sparse outputs are head-major: k_agg, v_agg dev [Hkv, T, d]; kv_pos dev int32 [Hkv, T] =
+ *   off_n + local index; sel_idx_out dev int32 [Hkv, T] local indices (TOPK; nullable);
+ *   cu_kv dev int32 [N+1] = prefix sum of k_sel.  Dropped rows are removed, not zeroed.
+ *
+ *   k_parts, v_parts: host arrays of N dev pointers, participant n's [L_n,Hkv,d] (may be slices
+ *   of one packed buffer).  seqlens_host host int32 [N].  k_sel_host host int32 [N], 0 <= k_sel[n]
+ *   <= L_n (ignored for CONCAT).  TOPK needs L_n <= 4096 per participant (else UNSUPPORTED).
+ *   kv_pos and cu_kv may be NULL when not wanted. */
+typedef enum {
+    FEDATTN_AGG_CONCAT = 0,
+    FEDATTN_AGG_TOPK_KNORM = 1,
+    FEDATTN_AGG_INDEXED = 2
+} fedattn_agg_mode;
+
+fedattn_status fedattn_aggregate_kv(fedattn_ctx *ctx, const fedattn_shape *shape, int32_t mode,
+                                    const void *const *k_parts, const void *const *v_parts,
+                                    const int32_t *seqlens_host, const int32_t *k_sel_host,
+                                    const int32_t *sel_idx_in,
+                                    void *k_agg, void *v_agg, int32_t *kv_pos, int32_t *cu_kv,
+                                    int32_t *sel_idx_out, fedattn_stream stream);
+
+/* ---- global (sync) attention: Phase II, o_n = Attention(q_n, K, V) ----------------------------
+ * Paper: Sec. IV-B "Phase II: Global Self-Attention", eq. (update_local_o_H), Algorithm 1 second
+ * parallel loop.  The mask is causal on the global token index (so that syncing at every block
+ * equals centralised attention): query row i with position p_i = q_pos ? q_pos[i] : i attends
+ * aggregated row j of KV head h iff kv_pos[h][j] <= p_i (every row when causal == 0).  A row whose
+ * allowed set is empty gets o = 0 and lse = -inf.
+ *   q dev [L,Hq,d] (all participants' rows, packed; L = n_q_rows).
+ *   k_agg, v_agg dev: kv_head_major == 0: [T,Hkv,d], kv_pos dev int32 [T] or NULL (= 0..T-1);
+ *                     kv_head_major == 1: [Hkv,T,d], kv_pos dev int32 [Hkv,T] or NULL.
+ *   kv_pos must be non-decreasing along T (aggregate_kv always produces that).
+ *   q_pos dev int32 [L] or NULL.  o dev [L,Hq,d]; lse dev float [L,Hq] or NULL. */
+fedattn_status fedattn_sync(fedattn_ctx *ctx, const fedattn_shape *shape,
+                            const void *q, int64_t n_q_rows, const int32_t *q_pos,
+                            const void *k_agg, const void *v_agg, const int32_t *kv_pos,
+                            int64_t total_kv, int32_t kv_head_major,
+                            void *o, float *lse, fedattn_stream stream);
+
+/* ---- decode: one new query token per participant over cached KV -------------------------------
+ * Paper: Sec. IV-C "Output Generation" (blocks that ran local attention cache local KV, blocks
+ * that ran global attention cache the global KV), Sec. III-C (O(L) per step, memory-bound).
+ * The new token is later than every cached row, so no mask applies.
+ *   FEDATTN_DECODE_LOCAL  participant n reads rows 0..kv_len[n]-1 of its own cache at
+ *                         k_cache + n * cache_stride_participant elements, layout [cap,Hkv,d];
+ *                         kv_len dev int32 [N].
+ *   FEDATTN_DECODE_SYNC   every participant reads rows 0..kv_len[0]-1 of one shared cache
+ *                         [T,Hkv,d]; kv_len dev int32 [1]; cache_stride_participant ignored.
+ *   q, o dev [N,Hq,d]; lse dev float [N,Hq] or NULL; max_kv_len >= every kv_len (host; sizes the
+ *   split-KV grid).  kv_len = 0 gives o = 0, lse = -inf.  Uses the workspace for split-KV partials. */
+typedef enum { FEDATTN_DECODE_LOCAL = 0, FEDATTN_DECODE_SYNC = 1 } fedattn_decode_mode;
+
+fedattn_status fedattn_decode(fedattn_ctx *ctx, const fedattn_shape *shape, int32_t mode,
+                              const void *q, const void *k_cache, const void *v_cache,
+                              int64_t cache_stride_participant, const int32_t *kv_len,
+                              int32_t max_kv_len, void *o, float *lse, fedattn_stream stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FEDATTN_H_ */

@@ -1,0 +1,186 @@
+"""ctypes binding of include/fedattn.h.  Function names match the C entry points; torch tensors
+supply device memory and the current CUDA stream."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Sequence
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_PKG, "lib", "libfedattn.so")
+
+F32, BF16 = 0, 1
+AGG_CONCAT, AGG_TOPK_KNORM, AGG_INDEXED = 0, 1, 2
+DECODE_LOCAL, DECODE_SYNC = 0, 1
+
+_SYMBOLS = ["fedattn_workspace_bytes", "fedattn_create", "fedattn_destroy", "fedattn_status_string",
+            "fedattn_poll", "fedattn_launch_count", "fedattn_local", "fedattn_aggregate_kv",
+            "fedattn_sync", "fedattn_decode"]
+
+
+class FedAttnError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__("%s failed: %s (status %d)" % (where, status_string(code), code))
+
+
+class Shape(C.Structure):
+    """Mirror of fedattn_shape."""
+    _fields_ = [("n_participants", C.c_int32), ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32),
+                ("head_dim", C.c_int32), ("dtype", C.c_int32), ("causal", C.c_int32), ("scale", C.c_float)]
+
+    def __init__(self, n_participants, n_q_heads, n_kv_heads, head_dim, dtype, causal=1, scale=0.0):
+        super().__init__(int(n_participants), int(n_q_heads), int(n_kv_heads), int(head_dim), int(dtype),
+                         int(causal), float(scale))
+
+    @property
+    def torch_dtype(self):
+        return torch.bfloat16 if self.dtype == BF16 else torch.float32
+
+
+def library_path() -> str:
+    return _LIB_PATH
+
+
+def _load():
+    if not os.path.exists(_LIB_PATH):
+        raise ImportError("FedAttn CUDA library missing: %s (run `python -m paper_2511_02647_b200.build` "
+                          "or __graft_entry__.build()); there is no fallback path" % _LIB_PATH)
+    lib = C.CDLL(_LIB_PATH)
+    vp, i32, i64 = C.c_void_p, C.c_int32, C.c_int64
+    lib.fedattn_workspace_bytes.restype = C.c_size_t
+    lib.fedattn_workspace_bytes.argtypes = [C.POINTER(Shape), i64, i64]
+    lib.fedattn_create.restype = C.c_int
+    lib.fedattn_create.argtypes = [C.POINTER(vp), C.c_int, vp, C.c_size_t]
+    lib.fedattn_destroy.restype = None
+    lib.fedattn_destroy.argtypes = [vp]
+    lib.fedattn_status_string.restype = C.c_char_p
+    lib.fedattn_status_string.argtypes = [C.c_int]
+    lib.fedattn_poll.restype = C.c_int
+    lib.fedattn_poll.argtypes = [vp, vp]
+    lib.fedattn_launch_count.restype = i64
+    lib.fedattn_launch_count.argtypes = [vp]
+    lib.fedattn_local.restype = C.c_int
+    lib.fedattn_local.argtypes = [vp, C.POINTER(Shape), vp, vp, vp, C.POINTER(i32), vp, vp, vp]
+    lib.fedattn_aggregate_kv.restype = C.c_int
+    lib.fedattn_aggregate_kv.argtypes = [vp, C.POINTER(Shape), i32, C.POINTER(vp), C.POINTER(vp),
+                                         C.POINTER(i32), C.POINTER(i32), vp, vp, vp, vp, vp, vp, vp]
+    lib.fedattn_sync.restype = C.c_int
+    lib.fedattn_sync.argtypes = [vp, C.POINTER(Shape), vp, i64, vp, vp, vp, vp, i64, i32, vp, vp, vp]
+    lib.fedattn_decode.restype = C.c_int
+    lib.fedattn_decode.argtypes = [vp, C.POINTER(Shape), i32, vp, vp, vp, i64, vp, i32, vp, vp, vp]
+    return lib
+
+
+_lib = _load()
+
+
+def exported_symbols():
+    """Names declared in include/fedattn.h that the loaded library exports."""
+    return [s for s in _SYMBOLS if hasattr(_lib, s)]
+
+
+def status_string(code: int) -> str:
+    return _lib.fedattn_status_string(int(code)).decode()
+
+
+def _check(code: int, where: str):
+    if code != 0:
+        raise FedAttnError(code, where)
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    if t is None:
+        return None
+    if not t.is_contiguous():
+        raise ValueError("tensor must be contiguous")
+    return t.data_ptr()
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def _i32_array(xs: Sequence[int]):
+    return (C.c_int32 * len(xs))(*[int(x) for x in xs])
+
+
+def fedattn_workspace_bytes(shape: Shape, max_total_tokens: int, max_total_kv: int) -> int:
+    return int(_lib.fedattn_workspace_bytes(C.byref(shape), int(max_total_tokens), int(max_total_kv)))
+
+
+class Context:
+    """Owns a device workspace tensor and the library context built around it."""
+
+    def __init__(self, shape: Shape, max_total_tokens: int, max_total_kv: int, device: int = 0):
+        nbytes = fedattn_workspace_bytes(shape, max_total_tokens, max_total_kv)
+        if nbytes == 0:
+            raise FedAttnError(1, "fedattn_workspace_bytes")
+        self.device = int(device)
+        self.workspace = torch.empty(nbytes, dtype=torch.uint8, device="cuda:%d" % self.device)
+        self._h = C.c_void_p()
+        _check(_lib.fedattn_create(C.byref(self._h), self.device, self.workspace.data_ptr(), nbytes),
+               "fedattn_create")
+
+    @property
+    def handle(self):
+        return self._h
+
+    def poll(self, stream=None) -> int:
+        """Synchronise the stream and return (and clear) the device status word."""
+        return int(_lib.fedattn_poll(self._h, _stream(stream)))
+
+    def launch_count(self) -> int:
+        return int(_lib.fedattn_launch_count(self._h))
+
+    def close(self):
+        if self._h:
+            _lib.fedattn_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def fedattn_local(ctx: Context, shape: Shape, q, k, v, cu_seqlens_host: Sequence[int], o, lse=None,
+                  stream=None):
+    cu = _i32_array(cu_seqlens_host)
+    if len(cu) != shape.n_participants + 1:
+        raise ValueError("cu_seqlens must have N+1 entries")
+    _check(_lib.fedattn_local(ctx.handle, C.byref(shape), _ptr(q), _ptr(k), _ptr(v), cu, _ptr(o), _ptr(lse),
+                              _stream(stream)), "fedattn_local")
+
+
+def fedattn_aggregate_kv(ctx: Context, shape: Shape, mode: int, k_parts, v_parts, seqlens_host,
+                         k_sel_host=None, sel_idx_in=None, k_agg=None, v_agg=None, kv_pos=None, cu_kv=None,
+                         sel_idx_out=None, stream=None):
+    n = shape.n_participants
+    if len(k_parts) != n or len(v_parts) != n or len(seqlens_host) != n:
+        raise ValueError("need one K part, V part and length per participant")
+    kp = (C.c_void_p * n)(*[_ptr(t) for t in k_parts])
+    vp = (C.c_void_p * n)(*[_ptr(t) for t in v_parts])
+    ks = None if k_sel_host is None else _i32_array(k_sel_host)
+    _check(_lib.fedattn_aggregate_kv(ctx.handle, C.byref(shape), int(mode), kp, vp, _i32_array(seqlens_host), ks,
+                                     _ptr(sel_idx_in), _ptr(k_agg), _ptr(v_agg), _ptr(kv_pos), _ptr(cu_kv),
+                                     _ptr(sel_idx_out), _stream(stream)), "fedattn_aggregate_kv")
+
+
+def fedattn_sync(ctx: Context, shape: Shape, q, q_pos, k_agg, v_agg, kv_pos, total_kv: int,
+                 kv_head_major: bool, o, lse=None, stream=None):
+    _check(_lib.fedattn_sync(ctx.handle, C.byref(shape), _ptr(q), int(q.shape[0]), _ptr(q_pos), _ptr(k_agg),
+                             _ptr(v_agg), _ptr(kv_pos), int(total_kv), int(bool(kv_head_major)), _ptr(o),
+                             _ptr(lse), _stream(stream)), "fedattn_sync")
+
+
+def fedattn_decode(ctx: Context, shape: Shape, mode: int, q, k_cache, v_cache, cache_stride_participant: int,
+                   kv_len, max_kv_len: int, o, lse=None, stream=None):
+    _check(_lib.fedattn_decode(ctx.handle, C.byref(shape), int(mode), _ptr(q), _ptr(k_cache), _ptr(v_cache),
+                               int(cache_stride_participant), _ptr(kv_len), int(max_kv_len), _ptr(o), _ptr(lse),
+                               _stream(stream)), "fedattn_decode")

@@ -1,0 +1,113 @@
+// Shared declarations of the FedAttn CUDA library (host dispatch <-> kernel launchers).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "fedattn.h"
+
+namespace fedattn {
+
+// Workspace layout: [0, kStatusBytes) status words, then the scratch region.
+constexpr size_t kStatusBytes = 256;
+constexpr int kMaxP = FEDATTN_MAX_PARTICIPANTS;
+// Upper bound on spin iterations of any in-kernel wait before it gives up.
+constexpr uint32_t kSpinLimit = 1u << 22;
+
+struct Context {
+    int device;
+    int sm_count;
+    char *workspace;       // dev
+    size_t workspace_bytes;
+    int32_t *status;       // dev, == workspace
+    char *scratch;         // dev, workspace + kStatusBytes
+    size_t scratch_bytes;
+    int64_t launches;
+    void *encode_tiled;    // cuTensorMapEncodeTiled entry point (driver), or nullptr
+};
+
+// ---- generic SIMT attention (fp32 or bf16 storage, any head_dim <= 128) --------------------
+enum GenericMode { kLocal = 0, kSync = 1, kDecodeLocal = 2, kDecodeSync = 3 };
+
+struct GenericParams {
+    const void *q, *k, *v;
+    void *o;
+    float *lse;
+    int64_t n_rows;               // query rows (tokens, or participants for decode)
+    int32_t hq, hkv, d;
+    float scale;
+    int32_t causal;
+    int32_t mode;                 // GenericMode
+    int64_t kv_tok_stride;        // elements between consecutive KV rows of one head
+    int64_t kv_head_stride;       // elements between KV heads
+    int64_t kv_pos_head_stride;   // ints between heads in kv_pos (0 = shared)
+    int64_t total_kv;             // sync: rows of the aggregated KV
+    const int32_t *q_pos;         // nullable
+    const int32_t *kv_pos;        // nullable
+    const int32_t *kv_len;        // decode: dev lengths
+    int64_t cache_stride;         // decode local: elements between participants' caches
+    int32_t n_seg;
+    int32_t cu[kMaxP + 1];        // local: segment offsets
+};
+
+cudaError_t launch_attn_generic(const GenericParams &p, int dtype, cudaStream_t s, int64_t *launches);
+
+// ---- aggregation -----------------------------------------------------------------------------
+struct PartsParams {
+    const void *k[kMaxP];
+    const void *v[kMaxP];
+    int32_t n;
+    int32_t off[kMaxP + 1];       // prefix sum of L_n  (rows)
+    int32_t cu_kv[kMaxP + 1];     // prefix sum of k_sel (rows), sparse modes
+};
+
+cudaError_t launch_concat(const PartsParams &pp, int hkv, int d, int elt_bytes, void *k_agg, void *v_agg,
+                          int32_t *kv_pos, int32_t *cu_kv, cudaStream_t s, int sm_count, int64_t *launches);
+
+// scores: dev double [sum_n Hkv*L_n] laid out participant-major, then head, then token.
+cudaError_t launch_knorm_scores(const PartsParams &pp, int hkv, int d, int dtype, double *scores,
+                                cudaStream_t s, int64_t *launches);
+cudaError_t launch_topk_select(const PartsParams &pp, int hkv, const double *scores, int32_t *sel_idx,
+                               cudaStream_t s, int64_t *launches);
+cudaError_t launch_gather(const PartsParams &pp, int hkv, int d, int elt_bytes, const int32_t *sel_idx,
+                          void *k_agg, void *v_agg, int32_t *kv_pos, int32_t *cu_kv, int32_t *sel_idx_out,
+                          int32_t *status, cudaStream_t s, int64_t *launches);
+
+// ---- bf16 prefill on tensor cores (tcgen05 + TMEM + TMA), head_dim 128 ------------------------
+struct PrefillParams {
+    const void *q, *k, *v;
+    void *o;
+    float *lse;
+    int64_t n_q_rows;
+    int64_t total_kv;             // rows of K/V (== n_q_rows for local)
+    int32_t hq, hkv;
+    float scale;
+    int32_t causal;
+    int32_t sync;                 // 0 local, 1 sync
+    int32_t kv_head_major;
+    const int32_t *kv_pos;        // nullable
+    int32_t n_seg;
+    int32_t cu[kMaxP + 1];        // query segments (local: also the KV segments)
+};
+bool prefill_sm100_supported(const Context *ctx);
+cudaError_t launch_prefill_sm100(const Context *ctx, const PrefillParams &p, cudaStream_t s, int64_t *launches);
+
+// ---- bf16 split-KV decode (tensor-core scores, warp-shuffle softmax) ---------------------------
+struct DecodeParams {
+    const void *q, *k, *v;
+    void *o;
+    float *lse;
+    int32_t n_part, hq, hkv, d;
+    float scale;
+    int32_t sync;
+    int64_t cache_stride;
+    const int32_t *kv_len;
+    int32_t max_kv_len;
+    float *partial;               // scratch
+    size_t partial_bytes;
+};
+size_t decode_scratch_bytes(int n_part, int hq, int d, int sm_count);
+cudaError_t launch_decode_bf16(const Context *ctx, const DecodeParams &p, cudaStream_t s, int64_t *launches);
+
+}  // namespace fedattn

@@ -1,0 +1,291 @@
+"""GPU parity: the CUDA path, called through the C-ABI binding, against the fp64 CPU oracle on the
+same seeded inputs.  Bars: bit-exact for offsets / positions / selected indices / copied bytes;
+max-abs 1e-4 for fp32 inputs; max-abs 2e-2 for bf16 inputs with O(1) outputs."""
+import numpy as np
+import pytest
+import torch
+
+import fedattn_inputs as fi
+from helpers import TOL, Runner, check_close, dev, fa, host
+
+pytestmark = pytest.mark.gpu
+
+
+def split(x, lens):
+    return np.split(x, np.cumsum(lens)[:-1])
+
+
+def gen(seed, lens, hq, hkv, d, dtype, gain=1.0):
+    w = fi.Workload("t", seed, tuple(int(x) for x in lens), hq, hkv, d, dtype, gain)
+    return w.qkv()
+
+
+# ---------------------------------------------------------------------------------------------
+# config 1: fp32, N=2 x 128, 4 heads, d=64 -- full comparison, local and sync
+# ---------------------------------------------------------------------------------------------
+def test_cfg1_fp32_local_and_sync(oracle):
+    w = fi.cfg1()
+    q, k, v = w.qkv()
+    r = Runner(2, 4, 4, 64, "f32", 256)
+    o, lse = r.local(q, k, v, w.seqlens)
+    oo, ol = oracle.local(q, k, v, w.seqlens)
+    e1 = check_close(o, oo, TOL["f32"], "cfg1 local o")
+    check_close(lse, ol, TOL["f32"], "cfg1 local lse")
+    agg = r.aggregate(fa().AGG_CONCAT, split(k, w.seqlens), split(v, w.seqlens))
+    ka, va, pos, cu = oracle.aggregate_concat(split(k, w.seqlens), split(v, w.seqlens))
+    assert np.array_equal(agg["kv_pos"].cpu().numpy(), pos) and np.array_equal(agg["cu_kv"].cpu().numpy(), cu)
+    assert np.array_equal(host(agg["k_agg"]), ka) and np.array_equal(host(agg["v_agg"]), va)
+    o, lse = r.sync(q, agg["k_agg"], agg["v_agg"], agg["kv_pos"])
+    oo, ol = oracle.sync(q, ka, va, kv_pos=pos)
+    check_close(o, oo, TOL["f32"], "cfg1 sync o")
+    check_close(lse, ol, TOL["f32"], "cfg1 sync lse")
+    assert np.abs(oo).max() > 0.1 and e1 < TOL["f32"]
+
+
+@pytest.mark.parametrize("dtype,hq,hkv,d", [("f32", 4, 2, 32), ("f32", 2, 2, 128), ("bf16", 4, 2, 64),
+                                            ("bf16", 8, 2, 128), ("bf16", 4, 4, 128)])
+@pytest.mark.parametrize("causal", [True, False])
+def test_ragged_segments_local_and_sync(oracle, dtype, hq, hkv, d, causal):
+    """Ragged lengths incl. 1, 0 and non-multiples of the 128-row tile; several tiles per segment."""
+    lens = [1, 130, 0, 257, 64, 300]
+    q, k, v = gen(11, lens, hq, hkv, d, dtype)
+    r = Runner(len(lens), hq, hkv, d, dtype, sum(lens), causal=causal)
+    o, lse = r.local(q, k, v, lens)
+    oo, ol = oracle.local(q, k, v, lens, causal=causal)
+    check_close(o, oo, TOL[dtype], "local o")
+    check_close(lse, ol, 1e-3 if dtype == "bf16" else 1e-4, "local lse")
+    o, lse = r.sync(q, k, v)
+    oo, ol = oracle.sync(q, k, v, causal=causal)
+    check_close(o, oo, TOL[dtype], "sync o")
+    check_close(lse, ol, 1e-3 if dtype == "bf16" else 1e-4, "sync lse")
+    # twice the same call: bitwise identical
+    o2, _ = r.sync(q, k, v)
+    assert np.array_equal(o, o2)
+
+
+def test_single_participant_and_tiny(oracle):
+    for lens, hq, hkv in [([1], 4, 4), ([5], 8, 2), ([129], 4, 1), ([128, 128], 4, 2), ([127, 1, 128], 4, 2)]:
+        q, k, v = gen(5, lens, hq, hkv, 128, "bf16")
+        r = Runner(len(lens), hq, hkv, 128, "bf16", sum(lens))
+        check_close(r.local(q, k, v, lens)[0], oracle.local(q, k, v, lens)[0], TOL["bf16"], str(lens))
+        check_close(r.sync(q, k, v)[0], oracle.sync(q, k, v)[0], TOL["bf16"], str(lens))
+
+
+def test_sync_with_explicit_query_positions(oracle):
+    """One participant's rows against the global KV, positions given explicitly."""
+    lens = [100, 60, 140]
+    q, k, v = gen(6, lens, 4, 2, 128, "bf16")
+    r = Runner(3, 4, 2, 128, "bf16", 300)
+    qp = np.arange(100, 160, dtype=np.int32)
+    o, lse = r.sync(q[100:160], k, v, q_pos=qp)
+    oo, ol = oracle.sync(q[100:160], k, v, q_pos=qp)
+    check_close(o, oo, TOL["bf16"], "q_pos")
+    check_close(o, oracle.sync(q, k, v)[0][100:160], TOL["bf16"], "q_pos vs packed")
+
+
+# ---------------------------------------------------------------------------------------------
+# aggregation
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_concat_is_bit_exact(oracle, dtype):
+    lens = [3, 0, 257, 1, 1000]
+    _, k, v = gen(7, lens, 2, 2, 64, dtype)
+    r = Runner(len(lens), 2, 2, 64, dtype, sum(lens))
+    agg = r.aggregate(fa().AGG_CONCAT, split(k, lens), split(v, lens))
+    ka, va, pos, cu = oracle.aggregate_concat(split(k, lens), split(v, lens))
+    assert agg["status"] == 0
+    assert np.array_equal(host(agg["k_agg"]), ka) and np.array_equal(host(agg["v_agg"]), va)
+    assert np.array_equal(agg["kv_pos"].cpu().numpy(), pos) and np.array_equal(agg["cu_kv"].cpu().numpy(), cu)
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_topk_indices_bit_exact_with_ties(oracle, dtype):
+    lens = [300, 1, 64, 1000, 7]
+    ksel = [75, 1, 0, 250, 7]
+    hkv, d = 4, 128
+    _, k, v = gen(8, lens, hkv, hkv, d, dtype)
+    kp, vp = split(k, lens), split(v, lens)
+    kp[0][17] = kp[0][3]; kp[0][200] = kp[0][3]; kp[0][40, 1] = -kp[0][41, 1]     # planted ties
+    kp[3][:] = kp[3][0]                                                           # all equal => first k
+    r = Runner(len(lens), hkv, hkv, d, dtype, sum(lens))
+    agg = r.aggregate(fa().AGG_TOPK_KNORM, kp, vp, ksel)
+    ka, va, pos, cu, sel = oracle.aggregate_topk(kp, vp, ksel)
+    assert agg["status"] == 0
+    assert np.array_equal(agg["sel_idx"].cpu().numpy(), sel)
+    assert np.array_equal(agg["kv_pos"].cpu().numpy(), pos) and np.array_equal(agg["cu_kv"].cpu().numpy(), cu)
+    assert np.array_equal(host(agg["k_agg"]), ka) and np.array_equal(host(agg["v_agg"]), va)
+    assert list(sel[0, cu[3]:cu[4]]) == list(range(250))
+
+
+def test_indexed_aggregation_and_bad_index_status(oracle):
+    lens = [50, 20, 30]
+    ksel = [5, 0, 30]
+    hkv, d = 2, 64
+    _, k, v = gen(9, lens, hkv, hkv, d, "bf16")
+    kp, vp = split(k, lens), split(v, lens)
+    rng = np.random.default_rng(0)
+    sel = np.stack([np.concatenate([np.sort(rng.choice(50, 5, replace=False)), np.arange(30)]) for _ in range(hkv)])
+    r = Runner(3, hkv, hkv, d, "bf16", 100)
+    agg = r.aggregate(fa().AGG_INDEXED, kp, vp, ksel, sel_idx_in=sel)
+    ka, va, pos, cu = oracle.aggregate_indexed(kp, vp, ksel, sel)
+    assert agg["status"] == 0
+    assert np.array_equal(host(agg["k_agg"]), ka) and np.array_equal(host(agg["v_agg"]), va)
+    assert np.array_equal(agg["kv_pos"].cpu().numpy(), pos) and np.array_equal(agg["cu_kv"].cpu().numpy(), cu)
+    bad = sel.copy()
+    bad[1, 2] = 50                                   # out of range for participant 0 (L_0 = 50)
+    agg = r.aggregate(fa().AGG_INDEXED, kp, vp, ksel, sel_idx_in=bad)
+    assert agg["status"] == 6                        # reported, not faulted; context still usable
+    assert r.aggregate(fa().AGG_INDEXED, kp, vp, ksel, sel_idx_in=sel)["status"] == 0
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_sparse_sync_small_incl_empty_rows_and_excluded_participant(oracle, dtype):
+    lens = [140, 90, 260]
+    hq, hkv, d = 8, 2, 128
+    q, k, v = gen(10, lens, hq, hkv, d, dtype)
+    kp, vp = split(k, lens), split(v, lens)
+    r = Runner(3, hq, hkv, d, dtype, sum(lens))
+    for ksel in ([35, 23, 65], [0, 30, 100], [140, 90, 260], [0, 0, 0]):
+        agg = r.aggregate(fa().AGG_TOPK_KNORM, kp, vp, ksel)
+        ka, va, pos, cu, sel = oracle.aggregate_topk(kp, vp, ksel)
+        assert np.array_equal(agg["sel_idx"].cpu().numpy(), sel)
+        o, lse = r.sync(q, agg["k_agg"], agg["v_agg"], agg["kv_pos"], head_major=True)
+        oo, ol = oracle.sync(q, ka, va, kv_pos=pos, kv_head_major=True)
+        check_close(o, oo, TOL[dtype], "sparse sync %s" % ksel)
+        check_close(lse, ol, 1e-3, "sparse sync lse %s" % ksel)
+    # rows of the first participant see nothing when it is excluded: zeros and -inf
+    assert np.all(o[:140] == 0)
+
+
+# ---------------------------------------------------------------------------------------------
+# decode
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("dtype,d", [("bf16", 128), ("f32", 64), ("bf16", 64)])
+def test_decode_small(oracle, dtype, d):
+    n, cap, hq, hkv = 3, 200, 8, 2
+    w = fi.Workload("d", 12, (cap,) * n, hq, hkv, d, dtype)
+    _, k, v = w.qkv()
+    q = w.decode_q(0)
+    kc, vc = k.reshape(n, cap, hkv, d), v.reshape(n, cap, hkv, d)
+    r = Runner(n, hq, hkv, d, dtype, n * cap)
+    for lens in ([200, 200, 200], [1, 77, 130], [0, 200, 5]):
+        o, lse = r.decode(q, kc, vc, lens, False, max_kv_len=cap)
+        oo, ol = oracle.decode(q, kc, vc, lens, False)
+        check_close(o, oo, TOL[dtype], "decode local %s" % lens)
+        check_close(lse, ol, 1e-3, "decode local lse")
+    for T in (600, 333, 1):
+        o, lse = r.decode(q, k, v, [T], True, max_kv_len=600)
+        oo, ol = oracle.decode(q, k, v, [T], True)
+        check_close(o, oo, TOL[dtype], "decode sync %d" % T)
+        check_close(lse, ol, 1e-3, "decode sync lse")
+
+
+def test_cfg5_decode_full_size(oracle):
+    w = fi.cfg5()
+    n, cap, hq, hkv, d = 8, 4096, 32, 8, 128
+    _, k, v = w.qkv()
+    kc, vc = k.reshape(n, cap, hkv, d), v.reshape(n, cap, hkv, d)
+    r = Runner(n, hq, hkv, d, "bf16", n * cap)
+    for step in (1, 4):
+        q = w.decode_q(step)
+        if fi.is_sync_block(step, w.sync_interval):
+            o, _ = r.decode(q, k, v, [n * cap], True)
+            oo, _ = oracle.decode(q, k, v, [n * cap], True)
+        else:
+            o, _ = r.decode(q, kc, vc, [cap] * n, False)
+            oo, _ = oracle.decode(q, kc, vc, [cap] * n, False)
+        err = check_close(o, oo, TOL["bf16"], "cfg5 step %d" % step)
+        assert err / np.abs(oo).max() < 0.05
+
+
+# ---------------------------------------------------------------------------------------------
+# full-size configurations, sampled rows (rows are independent, so sampled parity is exact)
+# ---------------------------------------------------------------------------------------------
+def _full_size_local_sync(oracle, w, n_random, block=0):
+    q, k, v = w.qkv(block)
+    rows = fi.sample_rows(w.seed, w.seqlens, n_random)
+    r = Runner(w.n_participants, w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype, w.total_tokens)
+    o, lse = r.local(q, k, v, w.seqlens)
+    oo, ol = oracle.local(q, k, v, w.seqlens, rows=rows)
+    e = check_close(o[rows], oo, TOL[w.dtype], w.name + " local")
+    check_close(lse[rows], ol, 1e-3, w.name + " local lse")
+    assert e / np.abs(oo).max() < 0.05               # not vacuous: error small relative to max |o|
+    agg = r.aggregate(fa().AGG_CONCAT, split(k, w.seqlens), split(v, w.seqlens))
+    assert np.array_equal(host(agg["k_agg"]), k) and np.array_equal(host(agg["v_agg"]), v)
+    o, lse = r.sync(q, agg["k_agg"], agg["v_agg"], agg["kv_pos"])
+    oo, ol = oracle.sync(q, k, v, rows=rows)
+    e = check_close(o[rows], oo, TOL[w.dtype], w.name + " sync")
+    check_close(lse[rows], ol, 1e-3, w.name + " sync lse")
+    assert e / np.abs(oo).max() < 0.05
+
+
+def test_cfg2_full_size_sampled(oracle):
+    _full_size_local_sync(oracle, fi.cfg2(), 256)
+
+
+def test_cfg2_prescaled_reading_relative_error(oracle):
+    """Literal alternative reading of config 2 (elements already divided by sqrt(128)): outputs are
+    small, so the bound is relative to max |o|."""
+    w = fi.cfg2_prescaled().scaled(seqlens=(512,) * 4)
+    q, k, v = w.qkv()
+    r = Runner(4, 32, 8, 128, "bf16", w.total_tokens)
+    o, _ = r.sync(q, k, v)
+    oo, _ = oracle.sync(q, k, v)
+    assert np.abs(o - oo).max() / np.abs(oo).max() < 0.02
+
+
+def test_cfg3_one_block_full_size_sampled(oracle):
+    _full_size_local_sync(oracle, fi.cfg3(), 96, block=5)
+
+
+def test_cfg4_sparse_full_size(oracle):
+    w = fi.cfg4()
+    q, k, v = w.qkv()
+    kp, vp = split(k, w.seqlens), split(v, w.seqlens)
+    ksel = [w.k_sel] * w.n_participants
+    r = Runner(16, 32, 8, 128, "bf16", w.total_tokens)
+    agg = r.aggregate(fa().AGG_TOPK_KNORM, kp, vp, ksel)
+    ka, va, pos, cu, sel = oracle.aggregate_topk(kp, vp, ksel)
+    assert np.array_equal(agg["sel_idx"].cpu().numpy(), sel)            # bit-exact indices
+    assert np.array_equal(agg["kv_pos"].cpu().numpy(), pos) and np.array_equal(agg["cu_kv"].cpu().numpy(), cu)
+    assert np.array_equal(host(agg["k_agg"]), ka) and np.array_equal(host(agg["v_agg"]), va)
+    rows = fi.sample_rows(w.seed, w.seqlens, 128)
+    o, lse = r.sync(q, agg["k_agg"], agg["v_agg"], agg["kv_pos"], head_major=True)
+    oo, ol = oracle.sync(q, ka, va, kv_pos=pos, kv_head_major=True, rows=rows)
+    check_close(o[rows], oo, TOL["bf16"], "cfg4 sparse sync")
+    check_close(lse[rows], ol, 1e-3, "cfg4 sparse sync lse")
+
+
+# ---------------------------------------------------------------------------------------------
+# C-ABI argument validation: rejected on the host, nothing launched, nothing faults
+# ---------------------------------------------------------------------------------------------
+def test_invalid_arguments_are_rejected():
+    m = fa()
+    r = Runner(2, 4, 2, 128, "bf16", 64)
+    q = torch.zeros((64, 4, 128), dtype=torch.bfloat16, device="cuda")
+    kv = torch.zeros((64, 2, 128), dtype=torch.bfloat16, device="cuda")
+    o = torch.zeros_like(q)
+    before = r.ctx.launch_count()
+    with pytest.raises(m.FedAttnError) as e:
+        m.fedattn_local(r.ctx, r.shape, q, kv, kv, [0, 40, 30], o)            # non-monotone offsets
+    assert e.value.code == 1
+    with pytest.raises(m.FedAttnError):
+        m.fedattn_local(r.ctx, r.shape, q, kv, kv, [1, 40, 64], o)            # cu[0] != 0
+    with pytest.raises(m.FedAttnError):
+        m.fedattn_local(r.ctx, r.shape, None, kv, kv, [0, 40, 64], o)         # null pointer
+    with pytest.raises(m.FedAttnError):
+        m.fedattn_local(r.ctx, m.Shape(2, 4, 3, 128, m.BF16), q, kv, kv, [0, 40, 64], o)   # Hq % Hkv
+    with pytest.raises(m.FedAttnError):
+        m.fedattn_aggregate_kv(r.ctx, r.shape, m.AGG_TOPK_KNORM, [kv[:40], kv[40:]], [kv[:40], kv[40:]], [40, 24],
+                               [41, 0], None, kv, kv, None, None, None)       # k_sel > L_n
+    with pytest.raises(m.FedAttnError):
+        m.fedattn_aggregate_kv(r.ctx, r.shape, 7, [kv[:40], kv[40:]], [kv[:40], kv[40:]], [40, 24], None, None,
+                               kv, kv, None, None, None)                      # unknown mode
+    with pytest.raises(m.FedAttnError):
+        m.fedattn_sync(r.ctx, r.shape, q, None, kv, kv, None, -1, False, o)   # negative total_kv
+    with pytest.raises(m.FedAttnError):
+        m.fedattn_decode(r.ctx, r.shape, 3, q[:2], kv, kv, 0, torch.zeros(2, dtype=torch.int32, device="cuda"), 8,
+                         o[:2])                                               # unknown decode mode
+    assert r.ctx.launch_count() == before and r.poll() == 0
+    m.fedattn_local(r.ctx, r.shape, q, kv, kv, [0, 40, 64], o)                # still usable
+    assert r.poll() == 0 and r.ctx.launch_count() > before
