@@ -1,5 +1,468 @@
+// bf16 prefill attention for sm_100a: TMA-fed, tcgen05 tensor cores, accumulators in TMEM,
+// online softmax in fp32.  Serves fedattn_local (per-participant causal attention over packed
+// segments) and fedattn_sync (queries over the aggregated KV, causal on global positions).
+//
+// One CTA owns one 128-row query tile of one query head and walks the key/value tiles that its
+// rows may see; tiles the segment descriptors or the causal mask rule out are never loaded.
+// Two CTAs are resident per SM (96 KB shared memory and 256 TMEM columns each), so one CTA's
+// softmax overlaps the other's MMAs.
+//
+// Per KV tile j:   S = Q K_j^T            (tcgen05.mma, A/B from shared memory, D in TMEM)
+//                  P = exp2(S*c - m)      (128 softmax threads, one query row each, TMEM->regs)
+//                  O += P V_j             (tcgen05.mma, A = P from TMEM, B = V from shared memory)
+// O stays in TMEM for the whole tile walk and is rescaled only when a row's running maximum
+// grows by more than 2^8 (the final normalisation uses the same reference maximum, so the
+// result is exact up to rounding).
+//
+// Warp roles: warps 0-3 softmax/epilogue (TMEM lane = query row), warp 4 TMA producer (+ TMEM
+// allocation), warp 5 MMA issuer.  Every wait is bounded; on expiry the CTA sets the status word,
+// stops waiting and runs to its normal end (TMEM is always released).
+#include <cuda.h>
+
 #include "common.cuh"
+
 namespace fedattn {
-bool prefill_sm100_supported(const Context *) { return false; }
-cudaError_t launch_prefill_sm100(const Context *, const PrefillParams &, cudaStream_t, int64_t *) { return cudaErrorNotSupported; }
+
+namespace {
+
+constexpr int kTileM = 128;          // query rows per CTA
+constexpr int kTileN = 128;          // keys per KV tile
+constexpr int kD = 128;              // head dim
+constexpr int kThreads = 192;
+constexpr uint32_t kTileBytes = kTileM * kD * 2;      // 32 KB: one Q, K or V tile
+constexpr uint32_t kHalfBytes = kTileBytes / 2;       // one 64-column TMA box
+constexpr uint32_t kSmemBytes = 3 * kTileBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr uint32_t kTmemCols = 256;
+constexpr uint32_t kColS = 0, kColP = 0, kColO = 128;
+constexpr uint32_t kWaitLimit = 1u << 20;
+constexpr float kRescaleThreshold = 8.0f;
+
+struct KernelParams {
+    PrefillParams p;
+    int32_t tile_cu[kMaxP + 1];      // prefix sum of query tiles per segment
+    int32_t *status;
+};
+
+// ---- PTX wrappers ---------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
 }
+__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\t"
+                 "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+                 "selp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false (after flagging the status word once) when the limit is reached or
+// another thread of this CTA already gave up.
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag, int32_t *status)
+{
+    for (uint32_t it = 0; it < kWaitLimit; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+    }
+    *abort_flag = 1;
+    atomicMax(status, (int32_t)FEDATTN_ERR_TIMEOUT);
+    return false;
+}
+
+__device__ __forceinline__ void tma_load_3d(void *dst, const CUtensorMap *map, uint64_t *bar, int c0, int c1, int c2)
+{
+    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
+                 " [%0], [%1, {%3, %4, %5}], [%2];"
+                 ::"r"(smem_u32(dst)), "l"((uint64_t)map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2)
+                 : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint64_t *bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+// D[tmem] (+)= A[smem desc] * B[smem desc]
+__device__ __forceinline__ void umma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t acc)
+{
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                 ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc) : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem desc]
+__device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t acc)
+{
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+                 ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(acc) : "memory");
+}
+
+#define FEDATTN_TMEM_LD32(taddr, r)                                                                          \
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "                                                   \
+                 "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"                                   \
+                 "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"                  \
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]),       \
+                   "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]),   \
+                   "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]),             \
+                   "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]),             \
+                   "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])              \
+                 : "r"(taddr) : "memory")
+
+#define FEDATTN_TMEM_ST32(taddr, r)                                                                          \
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "                                             \
+                 "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"                                  \
+                 "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"                         \
+                 ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]),  \
+                   "r"(r[7]), "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]),          \
+                   "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]),       \
+                   "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]),       \
+                   "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31]) : "memory")
+
+#define FEDATTN_TMEM_ST16(taddr, r)                                                                          \
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "                                             \
+                 "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"                                 \
+                 ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]),  \
+                   "r"(r[7]), "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]),          \
+                   "r"(r[14]), "r"(r[15]) : "memory")
+
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ float ex2(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
+{
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+
+// Shared-memory matrix descriptor, 128-byte swizzle, 8-row groups 1024 bytes apart.
+//   K-major operand (Q, K): rows of 64 bf16 = 128 B; a tile is two such [128 x 64] halves.
+//   MN-major operand (V as B, N = head dim): 64 head-dim elements contiguous per key row;
+//   lbo = distance between the two 64-wide head-dim halves.
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr >> 4) & 0x3fff);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3fff) << 16;
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3fff) << 32;
+    d |= (uint64_t)1 << 46;            // descriptor version (Blackwell)
+    d |= (uint64_t)2 << 61;            // SWIZZLE_128B
+    return d;
+}
+
+// Instruction descriptor, kind::f16: D fp32, A/B bf16, M = 128, N = 128.
+constexpr uint32_t kIdescBase = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+constexpr uint32_t kIdescQK = kIdescBase;                 // A, B K-major
+constexpr uint32_t kIdescPV = kIdescBase | (1u << 16);    // B (V) MN-major
+
+// number of entries of the non-decreasing array pos[0..n) that are <= x
+__device__ __forceinline__ int count_le(const int32_t *pos, int n, int x)
+{
+    int lo = 0, hi = n;
+    while (lo < hi) {
+        const int mid = (lo + hi) >> 1;
+        if (__ldg(pos + mid) <= x) lo = mid + 1; else hi = mid;
+    }
+    return lo;
+}
+
+}  // namespace
+
+__global__ void __launch_bounds__(kThreads, 2)
+prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                     const __grid_constant__ CUtensorMap map_v, const __grid_constant__ KernelParams kp)
+{
+    extern __shared__ uint8_t smem_raw[];
+    const PrefillParams &p = kp.p;
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint8_t *sQ = smem, *sK = smem + kTileBytes, *sV = smem + 2 * kTileBytes;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + 3 * kTileBytes);
+    uint64_t *bar_q = bars + 0, *bar_k = bars + 1, *bar_v = bars + 2, *bar_s = bars + 3, *bar_p = bars + 4,
+             *bar_o = bars + 5;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 8);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(bars + 9);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+    // ---- which query tile / head ------------------------------------------------------------------
+    const int total_tiles = kp.tile_cu[p.n_seg];
+    const int tile_rank = blockIdx.x / p.hq;
+    const int h = blockIdx.x - tile_rank * p.hq;
+    const int tile_id = total_tiles - 1 - tile_rank;           // heavy (late) tiles first
+    int seg = 0;
+    while (seg + 1 < p.n_seg && tile_id >= kp.tile_cu[seg + 1]) ++seg;
+    const int q_row0 = p.cu[seg] + (tile_id - kp.tile_cu[seg]) * kTileM;
+    const int n_valid = min(kTileM, p.cu[seg + 1] - q_row0);
+    const int kvh = h / (p.hq / p.hkv);
+
+    // ---- allowed-prefix length c(row): keys kv_begin .. kv_begin + c - 1 are visible ---------------
+    const int T = (int)p.total_kv;
+    const int32_t *kvp = p.kv_pos ? p.kv_pos + (p.kv_head_major ? (int64_t)kvh * T : 0) : nullptr;
+    int kv_begin = 0;
+    auto prefix_len = [&](int r) -> int {
+        const int pos = q_row0 + r;
+        if (!p.sync) {
+            const int seg_len = p.cu[seg + 1] - p.cu[seg];
+            return p.causal ? min(pos - p.cu[seg] + 1, seg_len) : seg_len;
+        }
+        if (!p.causal) return T;
+        if (!kvp) return min(pos + 1, T);
+        return count_le(kvp, T, pos);
+    };
+    if (!p.sync) kv_begin = p.cu[seg];
+    const int c_last = prefix_len(n_valid - 1);
+    const int n_tiles = (c_last + kTileN - 1) / kTileN;
+
+    // ---- setup ------------------------------------------------------------------------------------
+    if (tid == 0) {
+        mbar_init(bar_q, 1); mbar_init(bar_k, 1); mbar_init(bar_v, 1);
+        mbar_init(bar_s, 1); mbar_init(bar_p, 128); mbar_init(bar_o, 1);
+        *abort_flag = (*reinterpret_cast<volatile int32_t *>(kp.status) == FEDATTN_ERR_TIMEOUT) ? 1 : 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 4) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 4) {
+        // ================= TMA producer =================
+        if (lane == 0 && n_tiles > 0) {
+            asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&map_q) : "memory");
+            asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&map_k) : "memory");
+            asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&map_v) : "memory");
+            mbar_expect_tx(bar_q, kTileBytes);
+            tma_load_3d(sQ, &map_q, bar_q, 0, h, q_row0);
+            tma_load_3d(sQ + kHalfBytes, &map_q, bar_q, 64, h, q_row0);
+            for (int j = 0; j < n_tiles; ++j) {
+                const int row = kv_begin + j * kTileN;
+                const int c1 = p.kv_head_major ? row : kvh, c2 = p.kv_head_major ? kvh : row;
+                if (j > 0) mbar_wait(bar_s, (j - 1) & 1, abort_flag, kp.status);     // K buffer free
+                mbar_expect_tx(bar_k, kTileBytes);
+                tma_load_3d(sK, &map_k, bar_k, 0, c1, c2);
+                tma_load_3d(sK + kHalfBytes, &map_k, bar_k, 64, c1, c2);
+                if (j > 0) mbar_wait(bar_o, (j - 1) & 1, abort_flag, kp.status);     // V buffer free
+                mbar_expect_tx(bar_v, kTileBytes);
+                tma_load_3d(sV, &map_v, bar_v, 0, c1, c2);
+                tma_load_3d(sV + kHalfBytes, &map_v, bar_v, 64, c1, c2);
+            }
+            if (*abort_flag) {
+                // give the copies still in flight a bounded chance to land before the CTA retires
+                for (uint32_t it = 0; it < 4096 && !mbar_try_wait(bar_k, (n_tiles - 1) & 1); ++it) {}
+                for (uint32_t it = 0; it < 4096 && !mbar_try_wait(bar_v, (n_tiles - 1) & 1); ++it) {}
+                for (uint32_t it = 0; it < 4096 && !mbar_try_wait(bar_q, 0); ++it) {}
+            }
+        }
+    } else if (warp == 5) {
+        // ================= MMA issuer =================
+        if (lane == 0 && n_tiles > 0) {
+            const uint32_t tS = tmem_base + kColS, tP = tmem_base + kColP, tO = tmem_base + kColO;
+            const uint32_t aQ = smem_u32(sQ), aK = smem_u32(sK), aV = smem_u32(sV);
+            mbar_wait(bar_q, 0, abort_flag, kp.status);
+            for (int j = 0; j < n_tiles; ++j) {
+                mbar_wait(bar_k, j & 1, abort_flag, kp.status);
+                tc_fence_after();
+#pragma unroll
+                for (int ks = 0; ks < kD / 16; ++ks) {
+                    const uint32_t off = (ks >> 2) * kHalfBytes + (ks & 3) * 32;
+                    umma_ss(tS, make_desc(aQ + off, 16, 1024), make_desc(aK + off, 16, 1024), kIdescQK, ks > 0);
+                }
+                tc_commit(bar_s);
+                mbar_wait(bar_p, j & 1, abort_flag, kp.status);
+                mbar_wait(bar_v, j & 1, abort_flag, kp.status);
+                tc_fence_after();
+#pragma unroll
+                for (int ks = 0; ks < kTileN / 16; ++ks)
+                    umma_ts(tO, tP + ks * 8, make_desc(aV + ks * 2048, kHalfBytes, 1024), kIdescPV, (j > 0 || ks > 0));
+                tc_commit(bar_o);
+            }
+        }
+    } else {
+        // ================= softmax + epilogue: thread = query row =================
+        const int r = tid;                                      // 0..127, TMEM lane
+        const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+        const uint32_t tS = tmem_base + lane_base + kColS, tP = tmem_base + lane_base + kColP,
+                       tO = tmem_base + lane_base + kColO;
+        const int c_r = prefix_len(r);
+        const float sl2 = p.scale * 1.4426950408889634f;
+        float m_used = 0.f, l = 0.f;
+
+        for (int j = 0; j < n_tiles; ++j) {
+            mbar_wait(bar_s, j & 1, abort_flag, kp.status);
+            tc_fence_after();
+            uint32_t s[128];
+            FEDATTN_TMEM_LD32(tS + 0, (s + 0));
+            FEDATTN_TMEM_LD32(tS + 32, (s + 32));
+            FEDATTN_TMEM_LD32(tS + 64, (s + 64));
+            FEDATTN_TMEM_LD32(tS + 96, (s + 96));
+            tmem_wait_ld();
+            const int lim = c_r - j * kTileN;                  // columns < lim are visible
+            if (lim < kTileN) {
+#pragma unroll
+                for (int c = 0; c < 128; ++c)
+                    if (c >= lim) s[c] = 0xff800000u;           // -inf
+            }
+            float mx = -INFINITY;
+#pragma unroll
+            for (int c = 0; c < 128; ++c) mx = fmaxf(mx, __uint_as_float(s[c]));
+            const float t_max = mx * sl2;
+            if (j == 0) {
+                m_used = (t_max == -INFINITY) ? 0.f : t_max;
+            } else {
+                const bool need = t_max > m_used + kRescaleThreshold;
+                if (__any_sync(0xffffffffu, need)) {
+                    const float alpha = need ? ex2(m_used - t_max) : 1.f;
+                    mbar_wait(bar_o, (j - 1) & 1, abort_flag, kp.status);   // O holds tiles 0..j-1
+                    tc_fence_after();
+#pragma unroll
+                    for (int cc = 0; cc < 4; ++cc) {
+                        uint32_t o[32];
+                        FEDATTN_TMEM_LD32(tO + cc * 32, o);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
+                        FEDATTN_TMEM_ST32(tO + cc * 32, o);
+                    }
+                    if (need) { l *= alpha; m_used = t_max; }
+                }
+            }
+            float rowsum = 0.f;
+#pragma unroll
+            for (int cc = 0; cc < 4; ++cc) {
+                uint32_t pk[16];
+#pragma unroll
+                for (int c = 0; c < 16; ++c) {
+                    const float p0 = ex2(fmaf(__uint_as_float(s[cc * 32 + 2 * c]), sl2, -m_used));
+                    const float p1 = ex2(fmaf(__uint_as_float(s[cc * 32 + 2 * c + 1]), sl2, -m_used));
+                    rowsum += p0 + p1;
+                    pk[c] = pack_bf16(p0, p1);
+                }
+                FEDATTN_TMEM_ST16(tP + cc * 16, pk);
+            }
+            l += rowsum;
+            tmem_wait_st();
+            tc_fence_before();
+            mbar_arrive(bar_p);
+        }
+
+        // ---- epilogue: O / l -> bf16 -> global -------------------------------------------------------
+        const bool valid = r < n_valid;
+        __nv_bfloat16 *orow = reinterpret_cast<__nv_bfloat16 *>(p.o) + ((int64_t)(q_row0 + r) * p.hq + h) * kD;
+        if (n_tiles > 0) {
+            mbar_wait(bar_o, (n_tiles - 1) & 1, abort_flag, kp.status);
+            tc_fence_after();
+            const float inv = l > 0.f ? 1.f / l : 0.f;
+#pragma unroll
+            for (int cc = 0; cc < 4; ++cc) {
+                uint32_t o[32];
+                FEDATTN_TMEM_LD32(tO + cc * 32, o);
+                tmem_wait_ld();
+                if (valid) {
+#pragma unroll
+                    for (int c = 0; c < 32; c += 8) {
+                        uint4 w;
+                        w.x = pack_bf16(__uint_as_float(o[c + 0]) * inv, __uint_as_float(o[c + 1]) * inv);
+                        w.y = pack_bf16(__uint_as_float(o[c + 2]) * inv, __uint_as_float(o[c + 3]) * inv);
+                        w.z = pack_bf16(__uint_as_float(o[c + 4]) * inv, __uint_as_float(o[c + 5]) * inv);
+                        w.w = pack_bf16(__uint_as_float(o[c + 6]) * inv, __uint_as_float(o[c + 7]) * inv);
+                        *reinterpret_cast<uint4 *>(orow + cc * 32 + c) = w;
+                    }
+                }
+            }
+        } else if (valid) {
+#pragma unroll
+            for (int c = 0; c < kD; c += 8) *reinterpret_cast<uint4 *>(orow + c) = make_uint4(0, 0, 0, 0);
+        }
+        if (valid && p.lse)
+            p.lse[(int64_t)(q_row0 + r) * p.hq + h] =
+                l > 0.f ? (m_used + log2f(l)) * 0.6931471805599453f : -INFINITY;
+    }
+
+    // ---- teardown -----------------------------------------------------------------------------------
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 4) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+    }
+}
+
+// ---- host ---------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+bool prefill_sm100_supported(const Context *ctx) { return ctx->encode_tiled != nullptr; }
+
+// [rows, heads, 128] bf16 (token-major) or [heads, rows, 128] (head-major); boxes of 64 columns x 128 rows.
+static bool encode_map(const Context *ctx, CUtensorMap *map, const void *base, int64_t rows, int heads, bool head_major)
+{
+    EncodeTiledFn fn = reinterpret_cast<EncodeTiledFn>(ctx->encode_tiled);
+    cuuint64_t dims[3], strides[2];
+    cuuint32_t box[3], estr[3] = {1, 1, 1};
+    dims[0] = kD;
+    if (head_major) {
+        dims[1] = (cuuint64_t)rows; dims[2] = (cuuint64_t)heads;
+        strides[0] = kD * 2; strides[1] = (cuuint64_t)rows * kD * 2;
+        box[0] = 64; box[1] = kTileN; box[2] = 1;
+    } else {
+        dims[1] = (cuuint64_t)heads; dims[2] = (cuuint64_t)rows;
+        strides[0] = kD * 2; strides[1] = (cuuint64_t)heads * kD * 2;
+        box[0] = 64; box[1] = 1; box[2] = kTileN;
+    }
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+cudaError_t launch_prefill_sm100(const Context *ctx, const PrefillParams &p, cudaStream_t s, int64_t *launches)
+{
+    static_assert(sizeof(KernelParams) < 3000, "kernel parameter block too large");
+    KernelParams kp;
+    kp.p = p;
+    kp.status = ctx->status;
+    kp.tile_cu[0] = 0;
+    for (int n = 0; n < p.n_seg; ++n)
+        kp.tile_cu[n + 1] = kp.tile_cu[n] + (p.cu[n + 1] - p.cu[n] + kTileM - 1) / kTileM;
+    const int64_t blocks = (int64_t)kp.tile_cu[p.n_seg] * p.hq;
+    if (blocks == 0) return cudaSuccess;
+    if (blocks > 0x7fffffffLL) return cudaErrorInvalidValue;
+    CUtensorMap mq, mk, mv;
+    if (!encode_map(ctx, &mq, p.q, p.n_q_rows, p.hq, false) ||
+        !encode_map(ctx, &mk, p.k, p.total_kv, p.hkv, p.kv_head_major != 0) ||
+        !encode_map(ctx, &mv, p.v, p.total_kv, p.hkv, p.kv_head_major != 0))
+        return cudaErrorInvalidValue;
+    static bool attr_set[64] = {};
+    if (!attr_set[ctx->device & 63]) {
+        cudaError_t e = cudaFuncSetAttribute(prefill_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        if (e != cudaSuccess) return e;
+        attr_set[ctx->device & 63] = true;
+    }
+    prefill_sm100_kernel<<<(unsigned)blocks, kThreads, kSmemBytes, s>>>(mq, mk, mv, kp);
+    ++*launches;
+    return cudaGetLastError();
+}
+
+}  // namespace fedattn
