@@ -1,0 +1,423 @@
+#!/usr/bin/env python
+"""Benchmark of the FedAttn attention hot path on B200.
+
+One step = one pass of the whole hot path over one batch of synthetic input with the shapes of
+the bf16 Llama-3-8B attention configuration (N=4 participants x 2048 tokens, 32 query heads /
+8 KV heads, head_dim 128):
+
+    fedattn_local                      per-participant causal attention
+    fedattn_aggregate_kv (CONCAT)      dense KV aggregation
+    fedattn_sync                       queries over the 8192-token aggregated KV
+    fedattn_aggregate_kv (TOPK_KNORM)  sparse aggregation, top 25% keys per participant and KV head
+    fedattn_sync (sparse)              queries over the selected KV, global-position mask
+    fedattn_decode (LOCAL)             one new token per participant over its own 2048-token cache
+    fedattn_decode (SYNC)              the same tokens over the shared 8192-token cache
+
+`value` is the algorithmic attention TFLOP/s of the whole step (exact unmasked (q,k) pairs x 4*d
+flop per query head, divided by the step time, inputs resident in HBM).  `e2e` is the same metric
+through the same calls with pinned HOST inputs and outputs (copies inside the timed region).
+`roofline` covers the dominant kernel (the tcgen05 prefill kernel); `calls` gives every call's
+own time and rate.  `--impl reference` times the fp64 CPU oracle on a bounded row sample.
+With --gpus N > 1 every rank runs an independent replica (the path has no exchange step on one
+device; participants are simulated per GPU) and the value is the sum over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import fedattn_inputs as fi  # noqa: E402
+
+METRIC = "fedattn_prefill_tflops"
+UNIT = "TFLOP/s"
+N_SETS = 3            # rotating input sets: ~600 MB touched per cycle, larger than the 126 MB L2
+SPARSE_RATIO_NUM, SPARSE_RATIO_DEN = 1, 4
+# dram__bytes_read.sum + dram__bytes_write.sum per prefill launch of the sync call at this
+# workload, from the ncu capture summarised under profiles/ (None until captured)
+PREFILL_SYNC_DRAM_BYTES = None
+
+
+def env_rank():
+    return (int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0")),
+            int(os.environ.get("WORLD_SIZE", "1")))
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return dict(tensor=float(d["bf16_tflops"]), tensor_sustained=float(d.get("bf16_tflops_sustained", 0.0)),
+                    hbm=float(d["hbm_gbs"]), kind="measured")
+    return dict(tensor=1590.0, tensor_sustained=1400.0, hbm=6650.0, kind="fallback")
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.thread.join(timeout=2)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for nm, val in zip(names, f[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------------------------------------
+# workload bookkeeping (algorithmic flops / bytes; no arithmetic of the method)
+# ------------------------------------------------------------------------------------------------
+def workload():
+    return fi.cfg2()
+
+
+def flops_local(w):
+    return 4.0 * w.head_dim * w.n_q_heads * sum(n * (n + 1) // 2 for n in w.seqlens)
+
+
+def flops_sync(w):
+    L = w.total_tokens
+    return 4.0 * w.head_dim * w.n_q_heads * (L * (L + 1) // 2)
+
+
+def flops_decode(w):
+    L = w.total_tokens
+    return 4.0 * w.head_dim * w.n_q_heads * L, 4.0 * w.head_dim * w.n_q_heads * w.n_participants * L
+
+
+# ------------------------------------------------------------------------------------------------
+# our arm
+# ------------------------------------------------------------------------------------------------
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    import paper_2511_02647_b200 as fa
+
+    rank, local_rank, world = env_rank()
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    w = workload()
+    N, Hq, Hkv, d, L = w.n_participants, w.n_q_heads, w.n_kv_heads, w.head_dim, w.total_tokens
+    seqlens = list(w.seqlens)
+    cu = [0] + list(np.cumsum(seqlens))
+    ksel = [n * SPARSE_RATIO_NUM // SPARSE_RATIO_DEN for n in seqlens]
+    T = sum(ksel)
+    shape = fa.Shape(N, Hq, Hkv, d, fa.BF16)
+    ctx = fa.Context(shape, L, L, device=local_rank)
+    dev = torch.device("cuda", local_rank)
+    bf = torch.bfloat16
+
+    # host inputs (pinned) -- also the e2e source
+    host_sets = []
+    for s in range(N_SETS):
+        q, k, v = w.qkv(block=s)
+        qd = w.decode_q(s)
+        host_sets.append([torch.from_numpy(x).to(bf).pin_memory() for x in (q, k, v, qd)])
+
+    class Buf:
+        pass
+
+    def make_set(hs):
+        b = Buf()
+        b.q, b.k, b.v, b.qd = [x.to(dev, non_blocking=True) for x in hs]
+        b.o_local = torch.empty_like(b.q); b.o_sync = torch.empty_like(b.q); b.o_sparse = torch.empty_like(b.q)
+        b.k_agg = torch.empty_like(b.k); b.v_agg = torch.empty_like(b.v)
+        b.kv_pos = torch.empty(L, dtype=torch.int32, device=dev)
+        b.cu_kv = torch.empty(N + 1, dtype=torch.int32, device=dev)
+        b.k_sp = torch.empty((Hkv, T, d), dtype=bf, device=dev); b.v_sp = torch.empty_like(b.k_sp)
+        b.pos_sp = torch.empty((Hkv, T), dtype=torch.int32, device=dev)
+        b.sel = torch.empty((Hkv, T), dtype=torch.int32, device=dev)
+        b.cu_sp = torch.empty(N + 1, dtype=torch.int32, device=dev)
+        b.o_dl = torch.empty_like(b.qd); b.o_ds = torch.empty_like(b.qd)
+        b.len_local = torch.tensor(seqlens, dtype=torch.int32, device=dev)
+        b.len_sync = torch.tensor([L], dtype=torch.int32, device=dev)
+        return b
+
+    sets = [make_set(hs) for hs in host_sets]
+    torch.cuda.synchronize()
+    set_mb = sum(t.numel() * t.element_size() for t in vars(sets[0]).values() if torch.is_tensor(t)) // 2 ** 20
+    stream = torch.cuda.current_stream()
+    call_names = ["local", "aggregate_concat", "sync", "aggregate_topk", "sync_sparse", "decode_local", "decode_sync"]
+
+    def step(b, ev=None):
+        def mark(i):
+            if ev is not None:
+                ev[i].record(stream)
+        kp = [b.k[cu[n]:cu[n + 1]] for n in range(N)]
+        vp = [b.v[cu[n]:cu[n + 1]] for n in range(N)]
+        mark(0)
+        fa.fedattn_local(ctx, shape, b.q, b.k, b.v, cu, b.o_local)
+        mark(1)
+        fa.fedattn_aggregate_kv(ctx, shape, fa.AGG_CONCAT, kp, vp, seqlens, None, None, b.k_agg, b.v_agg, b.kv_pos,
+                                b.cu_kv, None)
+        mark(2)
+        fa.fedattn_sync(ctx, shape, b.q, None, b.k_agg, b.v_agg, b.kv_pos, L, False, b.o_sync)
+        mark(3)
+        fa.fedattn_aggregate_kv(ctx, shape, fa.AGG_TOPK_KNORM, kp, vp, seqlens, ksel, None, b.k_sp, b.v_sp, b.pos_sp,
+                                b.cu_sp, b.sel)
+        mark(4)
+        fa.fedattn_sync(ctx, shape, b.q, None, b.k_sp, b.v_sp, b.pos_sp, T, True, b.o_sparse)
+        mark(5)
+        # decode: the prefill K/V act as the caches (local: participant n's own rows; sync: aggregated)
+        fa.fedattn_decode(ctx, shape, fa.DECODE_LOCAL, b.qd, b.k, b.v, seqlens[0] * Hkv * d, b.len_local,
+                          max(seqlens), b.o_dl)
+        mark(6)
+        fa.fedattn_decode(ctx, shape, fa.DECODE_SYNC, b.qd, b.k_agg, b.v_agg, 0, b.len_sync, L, b.o_ds)
+        mark(7)
+
+    assert len(set(seqlens)) == 1, "local decode uses a constant cache stride"
+
+    # one untimed pass to obtain the sparse pair count from the positions the library produced
+    step(sets[0])
+    assert ctx.poll() == 0
+    pos = sets[0].pos_sp.to(torch.int64)                                     # [Hkv, T], ascending per head
+    rows = torch.arange(L, device=dev, dtype=torch.int64)
+    pairs_sparse = sum(int(torch.searchsorted(pos[h].contiguous(), rows, right=True).sum().item()) for h in range(Hkv))
+    f_local, f_sync = flops_local(w), flops_sync(w)
+    f_sparse = 4.0 * d * (Hq // Hkv) * pairs_sparse
+    f_dl, f_ds = flops_decode(w)
+    step_flops = f_local + f_sync + f_sparse + f_dl + f_ds
+    eb = 2
+    kv_bytes = 2 * L * Hkv * d * eb
+    call_flops = dict(local=f_local, sync=f_sync, sync_sparse=f_sparse, decode_local=f_dl, decode_sync=f_ds)
+    call_bytes = dict(aggregate_concat=2 * kv_bytes,
+                      aggregate_topk=kv_bytes // 2 + (kv_bytes // 2) * T // L + kv_bytes * T // L,
+                      decode_local=kv_bytes + 2 * N * Hq * d * eb, decode_sync=kv_bytes + 2 * N * Hq * d * eb)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(max(args.warmup, 3)):
+        step(sets[i % N_SETS])
+    barrier()
+
+    # ---- timed region: K steps, per-call events on the launching stream ----
+    K = args.steps
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(8)] for _ in range(K)]
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    time.sleep(0.25)
+    launches0 = ctx.launch_count()
+    barrier()
+    t_start = torch.cuda.Event(enable_timing=True); t_end = torch.cuda.Event(enable_timing=True)
+    t_start.record(stream)
+    for i in range(K):
+        step(sets[i % N_SETS], evs[i])
+    t_end.record(stream)
+    barrier()
+    total_ms = t_start.elapsed_time(t_end)
+    launches = ctx.launch_count() - launches0
+    status = ctx.poll()
+    time.sleep(0.25)
+    clocks = sampler.stop()
+    if status != 0:
+        raise RuntimeError("device status %d after the timed region" % status)
+    call_ms = {nm: sum(evs[i][j].elapsed_time(evs[i][j + 1]) for i in range(K)) / K for j, nm in enumerate(call_names)}
+
+    # ---- e2e: pinned host inputs -> device, the same step, results -> pinned host ----
+    e2e_steps = max(3, min(K, 10))
+    hout = [torch.empty((L, Hq, d), dtype=bf).pin_memory() for _ in range(3)] + \
+           [torch.empty((N, Hq, d), dtype=bf).pin_memory() for _ in range(2)]
+    h2d = sum(x.numel() * x.element_size() for x in host_sets[0])
+    d2h = sum(x.numel() * x.element_size() for x in hout)
+
+    def e2e_step(i):
+        b, hs = sets[i % N_SETS], host_sets[i % N_SETS]
+        b.q.copy_(hs[0], non_blocking=True); b.k.copy_(hs[1], non_blocking=True)
+        b.v.copy_(hs[2], non_blocking=True); b.qd.copy_(hs[3], non_blocking=True)
+        step(b)
+        for dst, src in zip(hout, (b.o_local, b.o_sync, b.o_sparse, b.o_dl, b.o_ds)):
+            dst.copy_(src, non_blocking=True)
+
+    e2e_step(0)
+    barrier()
+    e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for i in range(e2e_steps):
+        e2e_step(i)
+    e1.record(stream)
+    barrier()
+    e2e_ms = e0.elapsed_time(e1) / e2e_steps
+
+    # ---- max over ranks ----
+    if world > 1:
+        t = torch.tensor([total_ms, e2e_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms, e2e_ms = float(t[0]), float(t[1])
+    ms_per_step = total_ms / K
+    value = world * step_flops / (ms_per_step * 1e-3) / 1e12
+    e2e_value = world * step_flops / (e2e_ms * 1e-3) / 1e12
+
+    if rank == 0:
+        pk = peaks()
+        pre_ms = call_ms["local"] + call_ms["sync"] + call_ms["sync_sparse"]
+        pre_flops = f_local + f_sync + f_sparse
+        achieved = pre_flops / (pre_ms * 1e-3) / 1e12
+        calls = {}
+        for nm in call_names:
+            c = {"ms": round(call_ms[nm], 5)}
+            if nm in call_flops:
+                c["tflops"] = round(call_flops[nm] / (call_ms[nm] * 1e-3) / 1e12, 3)
+            if nm in call_bytes:
+                c["gbs"] = round(call_bytes[nm] / (call_ms[nm] * 1e-3) / 1e9, 1)
+                c["frac_hbm"] = round(c["gbs"] / pk["hbm"], 4)
+            if nm in ("local", "sync", "sync_sparse"):
+                c["frac_tensor"] = round(c["tflops"] / pk["tensor"], 4)
+            calls[nm] = c
+        out = {
+            "metric": METRIC, "value": round(value, 3), "unit": UNIT, "n_gpus": world, "steps": K,
+            "warmup": max(args.warmup, 3), "ms_per_step": round(ms_per_step, 5), "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": w.name, "participants": N, "tokens_per_participant": seqlens[0],
+                       "q_heads": Hq, "kv_heads": Hkv, "head_dim": d, "sparse_keep": "1/4 per KV head",
+                       "step": "local+concat+sync+topk+sparse_sync+decode_local+decode_sync",
+                       "l2": "%d rotating input/output sets of %d MB each (> 126 MB L2), no flush" % (N_SETS, set_mb),
+                       "parallelism": "replicas" if world > 1 else "single"},
+            "clocks": clocks,
+            "e2e": {"value": round(e2e_value, 3), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "ms_per_step": round(e2e_ms, 4)},
+            "gpu_launches": int(launches),
+            "roofline": {"bound": "tensor", "kernel": "prefill_sm100_kernel (local + sync + sparse sync launches)",
+                         "achieved": round(achieved, 2), "peak": pk["tensor"], "unit": "TFLOP/s",
+                         "frac": round(achieved / pk["tensor"], 4), "peak_kind": "burst bf16, " + pk["kind"],
+                         "frac_of_sustained": round(achieved / pk["tensor_sustained"], 4) if pk["tensor_sustained"] else None,
+                         "frac_of_nominal_2250": round(achieved / 2250.0, 4),
+                         "traffic": PREFILL_SYNC_DRAM_BYTES},
+            "calls": calls,
+            "step_tflop": round(step_flops / 1e12, 5),
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            out["cpu_baseline"] = cpu_baseline(w, target_seconds=12.0)
+        print(json.dumps(out), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# ------------------------------------------------------------------------------------------------
+# CPU oracle legs
+# ------------------------------------------------------------------------------------------------
+def oracle_sample(w, q, k, v, n_rows, seed):
+    """Runs the oracle's local and sync attention on n_rows seeded rows (all heads).
+    Returns (seconds, algorithmic flops of the sample)."""
+    import oracle
+    rng = np.random.default_rng(seed)
+    rows = np.sort(rng.choice(w.total_tokens, size=n_rows, replace=False)).astype(np.int64)
+    off = np.concatenate([[0], np.cumsum(w.seqlens)])
+    seg = np.searchsorted(off, rows, side="right") - 1
+    pairs = int((rows - off[seg] + 1).sum() + (rows + 1).sum())
+    t0 = time.perf_counter()
+    oracle.local(q, k, v, w.seqlens, rows=rows)
+    oracle.sync(q, k, v, rows=rows)
+    dt = time.perf_counter() - t0
+    return dt, 4.0 * w.head_dim * w.n_q_heads * pairs
+
+
+def cpu_baseline(w, target_seconds):
+    import oracle
+    q, k, v = w.qkv(0)
+    q, k, v = (x.astype(np.float64) for x in (q, k, v))
+    dt, fl = oracle_sample(w, q, k, v, 16, 0)
+    n = int(min(w.total_tokens, max(16, 16 * target_seconds / max(dt, 1e-3))))
+    dt, fl = oracle_sample(w, q, k, v, n, 1)
+    return {"value": round(fl / dt / 1e12, 6), "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
+            "sample": "fp64 oracle local+sync attention on %d seeded query rows x %d heads of %s (%.1f s)"
+                      % (n, w.n_q_heads, w.name, dt)}
+
+
+def run_reference(args):
+    rank, _, world = env_rank()
+    if rank != 0:
+        return
+    import oracle
+    w = workload()
+    q, k, v = w.qkv(0)
+    q, k, v = (x.astype(np.float64) for x in (q, k, v))
+    dt, _ = oracle_sample(w, q, k, v, 16, 0)
+    budget = 120.0 / max(1, args.steps + max(args.warmup, 1))
+    n = int(min(w.total_tokens, max(16, 16 * min(budget, 8.0) / max(dt, 1e-3))))
+    for i in range(max(args.warmup, 1)):
+        oracle_sample(w, q, k, v, n, 10 + i)
+    tot_t, tot_f = 0.0, 0.0
+    for i in range(args.steps):
+        dt, fl = oracle_sample(w, q, k, v, n, 100 + i)
+        tot_t += dt; tot_f += fl
+    value = tot_f / tot_t / 1e12
+    sample = "fp64 oracle local+sync attention on %d seeded query rows x %d heads of %s per step" % (
+        n, w.n_q_heads, w.name)
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": round(value, 6), "unit": UNIT, "n_gpus": world,
+        "steps": args.steps, "warmup": max(args.warmup, 1), "ms_per_step": round(tot_t / args.steps * 1e3, 3),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "sample": sample},
+        "cpu_baseline": {"value": round(value, 6), "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": round(value, 6), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

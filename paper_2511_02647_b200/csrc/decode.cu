@@ -1,5 +1,317 @@
+// bf16 split-KV decode (head_dim 128): one new query token per participant over cached K/V.
+// HBM-bound: each K/V row is read once.  The query rows that share a KV head -- the g = Hq/Hkv
+// grouped heads of one participant (LOCAL), or of all participants (SYNC, one shared global
+// cache) -- are stacked into 16-row tiles so that QK^T and PV run on the tensor cores
+// (mma.sync m16n8k16), which keeps the 32 flop/byte of the sync step far below the memory time.
+// K/V tiles of 64 keys stream through a 3-stage cp.async pipeline with a 16-byte-chunk XOR
+// swizzle (conflict-free ldmatrix).  Row max / row sum are reduced with warp shuffles inside
+// each 4-lane quad.  Each CTA handles one (cache, KV head, split) and writes an unnormalised
+// partial (m, l, o); a second kernel merges the splits.
 #include "common.cuh"
+
 namespace fedattn {
-size_t decode_scratch_bytes(int, int, int, int) { return 0; }
-cudaError_t launch_decode_bf16(const Context *, const DecodeParams &, cudaStream_t, int64_t *) { return cudaErrorNotSupported; }
+
+namespace {
+
+constexpr int kD = 128;
+constexpr int kTileKeys = 64;
+constexpr int kStages = 3;
+constexpr int kTileBytes = kTileKeys * kD * 2;          // 16 KB (K or V)
+constexpr int kStageBytes = 2 * kTileBytes;             // K + V
+constexpr int kMaxSplits = 64;
+constexpr int kPartialStride = kD + 2;                  // m, l, o[128]
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, bool valid)
+{
+    const int sz = valid ? 16 : 0;      // src-size 0 => zero fill
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(sz) : "memory");
 }
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t addr)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
+{
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ float ex2(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
+{
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+
+// byte offset of 16-byte chunk `chunk` (0..15) of key row `row` inside a swizzled [64][128] bf16 tile
+__device__ __forceinline__ uint32_t swz(int row, int chunk) { return (uint32_t)(row * 256 + ((chunk ^ (row & 7)) << 4)); }
+
+}  // namespace
+
+// grid: x = split, y = KV head, z = cache * n_chunks + chunk   (cache = participant for LOCAL, 0 for SYNC)
+// block: 128 * kMTiles threads.  Warp w: M-tile w % kMTiles, key slice w / kMTiles (16 keys of every tile).
+template <int kMTiles>
+__global__ void __launch_bounds__(128 * kMTiles, 2)
+decode_split_kernel(const DecodeParams p, int n_splits, int n_chunks)
+{
+    extern __shared__ __align__(1024) uint8_t smem[];
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int mt = warp % kMTiles, slice = warp / kMTiles;
+    const int split = blockIdx.x, kvh = blockIdx.y;
+    const int cache = blockIdx.z / n_chunks, chunk = blockIdx.z - cache * n_chunks;
+    const int g = p.hq / p.hkv;
+    const int rows_total = p.sync ? p.n_part * g : g;          // query rows sharing this cache + KV head
+    const int row_base = (chunk * kMTiles + mt) * 16;           // first stacked row of this warp's M-tile
+
+    const int len = p.sync ? p.kv_len[0] : p.kv_len[cache];
+    const int tiles_total = (len + kTileKeys - 1) / kTileKeys;
+    const int tiles_per_split = (tiles_total + n_splits - 1) / n_splits;
+    const int tile_lo = min(split * tiles_per_split, tiles_total);
+    const int tile_hi = min(tile_lo + tiles_per_split, tiles_total);
+    const int n_tiles = tile_hi - tile_lo;
+
+    const size_t tok_stride = (size_t)p.hkv * kD;              // elements
+    const __nv_bfloat16 *Kb = reinterpret_cast<const __nv_bfloat16 *>(p.k) +
+                              (p.sync ? 0 : (size_t)cache * p.cache_stride) + (size_t)kvh * kD;
+    const __nv_bfloat16 *Vb = reinterpret_cast<const __nv_bfloat16 *>(p.v) +
+                              (p.sync ? 0 : (size_t)cache * p.cache_stride) + (size_t)kvh * kD;
+
+    // stacked row -> (participant, query head)
+    auto q_ptr = [&](int srow) -> const __nv_bfloat16 * {
+        if (srow >= rows_total) return nullptr;
+        const int part = p.sync ? srow / g : cache;
+        const int head = kvh * g + (p.sync ? srow % g : srow);
+        return reinterpret_cast<const __nv_bfloat16 *>(p.q) + ((size_t)part * p.hq + head) * kD;
+    };
+
+    // Q fragments (A operand, 16 x 128): 8 k-steps x 4 registers
+    uint32_t qf[8][4];
+    {
+        const __nv_bfloat16 *r0 = q_ptr(row_base + (lane >> 2)), *r1 = q_ptr(row_base + (lane >> 2) + 8);
+        const int c = (lane & 3) * 2;
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+            qf[ks][0] = r0 ? *reinterpret_cast<const uint32_t *>(r0 + ks * 16 + c) : 0u;
+            qf[ks][1] = r1 ? *reinterpret_cast<const uint32_t *>(r1 + ks * 16 + c) : 0u;
+            qf[ks][2] = r0 ? *reinterpret_cast<const uint32_t *>(r0 + ks * 16 + c + 8) : 0u;
+            qf[ks][3] = r1 ? *reinterpret_cast<const uint32_t *>(r1 + ks * 16 + c + 8) : 0u;
+        }
+    }
+
+    auto load_tile = [&](int t, int stage) {
+        // K and V tiles: 64 rows x 16 chunks each; rows past `len` are zero-filled
+        const int key0 = (tile_lo + t) * kTileKeys;
+        const uint32_t sK = smem_u32(smem) + stage * kStageBytes, sV = sK + kTileBytes;
+#pragma unroll
+        for (int i = tid; i < kTileKeys * 16; i += 128 * kMTiles) {
+            const int row = i >> 4, ch = i & 15;
+            const bool ok = key0 + row < len;
+            const size_t off = (size_t)(ok ? key0 + row : 0) * tok_stride + ch * 8;
+            cp_async16(sK + swz(row, ch), Kb + off, ok);
+            cp_async16(sV + swz(row, ch), Vb + off, ok);
+        }
+    };
+
+    const float sl2 = p.scale * 1.4426950408889634f;
+    float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;   // rows lane/4 and lane/4 + 8
+    float acc[16][4];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) acc[i][0] = acc[i][1] = acc[i][2] = acc[i][3] = 0.f;
+
+#pragma unroll
+    for (int s = 0; s < kStages - 1; ++s) {
+        if (s < n_tiles) load_tile(s, s);
+        cp_async_commit();
+    }
+    for (int t = 0; t < n_tiles; ++t) {
+        cp_async_wait<kStages - 2>();
+        __syncthreads();
+        if (t + kStages - 1 < n_tiles) load_tile(t + kStages - 1, (t + kStages - 1) % kStages);
+        cp_async_commit();
+
+        const uint32_t sK = smem_u32(smem) + (t % kStages) * kStageBytes, sV = sK + kTileBytes;
+        const int krow0 = slice * 16;
+        // ---- S = Q K^T for this warp's 16 keys: two n-tiles of 8 keys ----
+        float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+            // matrices: (keys 0-7, d 0-7) (keys 0-7, d 8-15) (keys 8-15, d 0-7) (keys 8-15, d 8-15)
+            const int row = krow0 + (lane & 7) + ((lane >> 4) << 3);
+            const int ch = ks * 2 + ((lane >> 3) & 1);
+            uint32_t b[4];
+            ldmatrix_x4(b, sK + swz(row, ch));
+            mma_bf16(s0, qf[ks], b[0], b[1]);
+            mma_bf16(s1, qf[ks], b[2], b[3]);
+        }
+        // ---- mask keys past the end, online softmax (rows lane/4 and lane/4+8) ----
+        const int key = (tile_lo + t) * kTileKeys + krow0 + (lane & 3) * 2;
+        float v[8] = {s0[0], s0[1], s1[0], s1[1], s0[2], s0[3], s1[2], s1[3]};   // row0: v[0..3], row1: v[4..7]
+        const bool ok[4] = {key < len, key + 1 < len, key + 8 < len, key + 9 < len};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            v[i] = ok[i] ? v[i] * sl2 : -INFINITY;
+            v[i + 4] = ok[i] ? v[i + 4] * sl2 : -INFINITY;
+        }
+        float mx0 = fmaxf(fmaxf(v[0], v[1]), fmaxf(v[2], v[3])), mx1 = fmaxf(fmaxf(v[4], v[5]), fmaxf(v[6], v[7]));
+        mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1)); mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
+        mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1)); mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
+        const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);
+        const float ms0 = mn0 == -INFINITY ? 0.f : mn0, ms1 = mn1 == -INFINITY ? 0.f : mn1;
+        const float a0 = ex2(m0 - ms0), a1 = ex2(m1 - ms1);
+        m0 = mn0; m1 = mn1;
+        float ps0 = 0.f, ps1 = 0.f;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            v[i] = ex2(v[i] - ms0); ps0 += v[i];
+            v[i + 4] = ex2(v[i + 4] - ms1); ps1 += v[i + 4];
+        }
+        l0 = l0 * a0 + ps0; l1 = l1 * a1 + ps1;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) { acc[i][0] *= a0; acc[i][1] *= a0; acc[i][2] *= a1; acc[i][3] *= a1; }
+        // P as A operand (16 rows x 16 keys)
+        uint32_t pf[4] = {pack_bf16(v[0], v[1]), pack_bf16(v[4], v[5]), pack_bf16(v[2], v[3]), pack_bf16(v[6], v[7])};
+        // ---- O += P V ----
+#pragma unroll
+        for (int nd = 0; nd < 8; ++nd) {
+            // matrices: (keys 0-7, d 0-7) (keys 8-15, d 0-7) (keys 0-7, d 8-15) (keys 8-15, d 8-15) of d block nd*16
+            const int row = krow0 + (lane & 7) + (((lane >> 3) & 1) << 3);
+            const int ch = nd * 2 + (lane >> 4);
+            uint32_t b[4];
+            ldmatrix_x4_trans(b, sV + swz(row, ch));
+            mma_bf16(acc[2 * nd], pf, b[0], b[1]);
+            mma_bf16(acc[2 * nd + 1], pf, b[2], b[3]);
+        }
+    }
+    cp_async_wait<0>();
+    __syncthreads();
+
+    // ---- merge the four key slices of each M-tile through shared memory ----
+    float *red = reinterpret_cast<float *>(smem);              // [warp][16 rows][kPartialStride]
+    {
+        // quad-reduce l (each lane of a quad summed different keys)
+        l0 += __shfl_xor_sync(0xffffffffu, l0, 1); l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
+        l1 += __shfl_xor_sync(0xffffffffu, l1, 1); l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
+        float *w0 = red + ((size_t)warp * 16 + (lane >> 2)) * kPartialStride;
+        float *w1 = w0 + 8 * kPartialStride;
+        if ((lane & 3) == 0) { w0[0] = m0; w0[1] = l0; w1[0] = m1; w1[1] = l1; }
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const int c = i * 8 + (lane & 3) * 2;
+            w0[2 + c] = acc[i][0]; w0[2 + c + 1] = acc[i][1];
+            w1[2 + c] = acc[i][2]; w1[2 + c + 1] = acc[i][3];
+        }
+    }
+    __syncthreads();
+    // thread -> (M-tile, row, 4 consecutive columns... ) : 16 * kMTiles rows x 128 columns
+    for (int idx = tid; idx < 16 * kMTiles * kD; idx += 128 * kMTiles) {
+        const int c = idx % kD, rr = idx / kD;                 // rr: row within CTA (mt' * 16 + r)
+        const int mtp = rr >> 4, r = rr & 15;
+        const int srow = (chunk * kMTiles + mtp) * 16 + r;
+        if (srow >= rows_total) continue;
+        float mm = -INFINITY;
+#pragma unroll
+        for (int sl = 0; sl < 4; ++sl) mm = fmaxf(mm, red[((size_t)(sl * kMTiles + mtp) * 16 + r) * kPartialStride]);
+        const float ms = mm == -INFINITY ? 0.f : mm;
+        float ll = 0.f, oo = 0.f;
+#pragma unroll
+        for (int sl = 0; sl < 4; ++sl) {
+            const float *w = red + ((size_t)(sl * kMTiles + mtp) * 16 + r) * kPartialStride;
+            const float sc = ex2(w[0] - ms);
+            ll += w[1] * sc;
+            oo += w[2 + c] * sc;
+        }
+        const int part = p.sync ? srow / g : cache;
+        const int head = kvh * g + (p.sync ? srow % g : srow);
+        const size_t orow = (size_t)part * p.hq + head;
+        if (n_splits == 1) {
+            reinterpret_cast<__nv_bfloat16 *>(p.o)[orow * kD + c] = __float2bfloat16_rn(ll > 0.f ? oo / ll : 0.f);
+            if (c == 0 && p.lse) p.lse[orow] = ll > 0.f ? (mm + log2f(ll)) * 0.6931471805599453f : -INFINITY;
+        } else {
+            float *dst = p.partial + (orow * n_splits + split) * kPartialStride;
+            dst[2 + c] = oo;
+            if (c == 0) { dst[0] = mm; dst[1] = ll; }
+        }
+    }
+}
+
+// grid: one CTA per output row (participant, query head); 128 threads = head dim.
+__global__ void __launch_bounds__(kD)
+decode_combine_kernel(const DecodeParams p, int n_splits)
+{
+    const size_t orow = blockIdx.x;
+    const int c = threadIdx.x;
+    const float *src = p.partial + orow * n_splits * kPartialStride;
+    float mm = -INFINITY;
+    for (int s = 0; s < n_splits; ++s) mm = fmaxf(mm, src[s * kPartialStride]);
+    const float ms = mm == -INFINITY ? 0.f : mm;
+    float ll = 0.f, oo = 0.f;
+    for (int s = 0; s < n_splits; ++s) {
+        const float sc = ex2(src[s * kPartialStride] - ms);
+        ll += src[s * kPartialStride + 1] * sc;
+        oo += src[s * kPartialStride + 2 + c] * sc;
+    }
+    reinterpret_cast<__nv_bfloat16 *>(p.o)[orow * kD + c] = __float2bfloat16_rn(ll > 0.f ? oo / ll : 0.f);
+    if (c == 0 && p.lse) p.lse[orow] = ll > 0.f ? (mm + log2f(ll)) * 0.6931471805599453f : -INFINITY;
+}
+
+size_t decode_scratch_bytes(int n_part, int hq, int d, int /*sm_count*/)
+{
+    if (d != kD) return 0;
+    return (size_t)n_part * hq * kMaxSplits * kPartialStride * sizeof(float);
+}
+
+cudaError_t launch_decode_bf16(const Context *ctx, const DecodeParams &p, cudaStream_t s, int64_t *launches)
+{
+    const int g = p.hq / p.hkv;
+    const int rows_total = p.sync ? p.n_part * g : g;
+    const int m_tiles = rows_total > 16 ? 2 : 1;
+    const int n_chunks = (rows_total + 16 * m_tiles - 1) / (16 * m_tiles);
+    const int caches = p.sync ? 1 : p.n_part;
+    const int sources = caches * p.hkv * n_chunks;
+    const int tiles = (p.max_kv_len + kTileKeys - 1) / kTileKeys;
+    int n_splits = (2 * ctx->sm_count + sources - 1) / sources;
+    if (n_splits > tiles / 2) n_splits = tiles / 2;            // at least two tiles per split
+    if (n_splits > kMaxSplits) n_splits = kMaxSplits;
+    if (n_splits < 1) n_splits = 1;
+    if (n_splits > 1 && (size_t)p.n_part * p.hq * n_splits * kPartialStride * sizeof(float) > p.partial_bytes)
+        return cudaErrorInvalidValue;
+    const int smem = kStages * kStageBytes;                    // 96 KB (also covers the merge buffer)
+    static bool attr_set[64] = {};
+    if (!attr_set[ctx->device & 63]) {
+        cudaError_t e = cudaFuncSetAttribute(decode_split_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(decode_split_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e != cudaSuccess) return e;
+        attr_set[ctx->device & 63] = true;
+    }
+    const dim3 grid(n_splits, p.hkv, caches * n_chunks);
+    if (m_tiles == 1)
+        decode_split_kernel<1><<<grid, 128, smem, s>>>(p, n_splits, n_chunks);
+    else
+        decode_split_kernel<2><<<grid, 256, smem, s>>>(p, n_splits, n_chunks);
+    ++*launches;
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess || n_splits == 1) return e;
+    decode_combine_kernel<<<p.n_part * p.hq, kD, 0, s>>>(p, n_splits);
+    ++*launches;
+    return cudaGetLastError();
+}
+
+}  // namespace fedattn
