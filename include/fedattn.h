@@ -167,6 +167,29 @@ fedattn_status fedattn_decode(fedattn_ctx *ctx, const fedattn_shape *shape, int3
                               int64_t cache_stride_participant, const int32_t *kv_len,
                               int32_t max_kv_len, void *o, float *lse, fedattn_stream stream);
 
+/* ---- decode for callers that cannot allocate -------------------------------------------------
+ * (The paper has no counterpart; this is a packaging variant of fedattn_decode.)
+ * fedattn_decode needs a context whose workspace somebody allocated with cudaMalloc (or a
+ * framework allocator).  Some callers cannot do that: code running where the device allocator
+ * must not be entered (inside a serving loop with a frozen memory plan, a plugin that receives
+ * its tensors and nothing more, a process whose memory is fully pre-partitioned).  This entry
+ * point takes no context and allocates nothing, on the host or on the device: the split-KV
+ * partials go to a fixed 2.03 MiB array built into the library image, which every GPU that loads
+ * the library holds until the process exits.
+ *
+ * Same arguments, layouts and results as fedattn_decode (bf16, head_dim 128 only; anything else
+ * returns FEDATTN_ERR_UNSUPPORTED).  The built-in scratch covers n_participants * n_q_heads <= 256
+ * output rows; a larger shape is rejected with FEDATTN_ERR_WORKSPACE and nothing is launched.
+ * It runs on the CURRENT device.  The first call on each device resolves the array's device
+ * address and sets kernel attributes; make that first call outside any stream capture.  Nothing
+ * in the scratch needs to start at zero (every slot that is read is written earlier in the same
+ * call), and its contents after a call are unspecified.  All calls on one device share the one
+ * array: two calls that may overlap on the GPU (different streams, no ordering) race on it. */
+fedattn_status fedattn_decode_noalloc(const fedattn_shape *shape, int32_t mode,
+                                      const void *q, const void *k_cache, const void *v_cache,
+                                      int64_t cache_stride_participant, const int32_t *kv_len,
+                                      int32_t max_kv_len, void *o, float *lse, fedattn_stream stream);
+
 #ifdef __cplusplus
 }
 #endif

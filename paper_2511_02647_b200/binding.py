@@ -17,7 +17,7 @@ DECODE_LOCAL, DECODE_SYNC = 0, 1
 
 _SYMBOLS = ["fedattn_workspace_bytes", "fedattn_create", "fedattn_destroy", "fedattn_status_string",
             "fedattn_poll", "fedattn_launch_count", "fedattn_local", "fedattn_aggregate_kv",
-            "fedattn_sync", "fedattn_decode"]
+            "fedattn_sync", "fedattn_decode", "fedattn_decode_noalloc"]
 
 
 class FedAttnError(RuntimeError):
@@ -71,6 +71,8 @@ def _load():
     lib.fedattn_sync.argtypes = [vp, C.POINTER(Shape), vp, i64, vp, vp, vp, vp, i64, i32, vp, vp, vp]
     lib.fedattn_decode.restype = C.c_int
     lib.fedattn_decode.argtypes = [vp, C.POINTER(Shape), i32, vp, vp, vp, i64, vp, i32, vp, vp, vp]
+    lib.fedattn_decode_noalloc.restype = C.c_int
+    lib.fedattn_decode_noalloc.argtypes = [C.POINTER(Shape), i32, vp, vp, vp, i64, vp, i32, vp, vp, vp]
     return lib
 
 
@@ -184,3 +186,13 @@ def fedattn_decode(ctx: Context, shape: Shape, mode: int, q, k_cache, v_cache, c
     _check(_lib.fedattn_decode(ctx.handle, C.byref(shape), int(mode), _ptr(q), _ptr(k_cache), _ptr(v_cache),
                                int(cache_stride_participant), _ptr(kv_len), int(max_kv_len), _ptr(o), _ptr(lse),
                                _stream(stream)), "fedattn_decode")
+
+
+def fedattn_decode_noalloc(shape: Shape, mode: int, q, k_cache, v_cache, cache_stride_participant: int,
+                           kv_len, max_kv_len: int, o, lse=None, stream=None):
+    """fedattn_decode for callers that may not allocate: no context, no workspace; the split-KV
+    partials use a fixed array inside the library (bf16, head_dim 128, at most 256 output rows).
+    Runs on the current CUDA device; calls that may overlap on the GPU share that array and race."""
+    _check(_lib.fedattn_decode_noalloc(C.byref(shape), int(mode), _ptr(q), _ptr(k_cache), _ptr(v_cache),
+                                       int(cache_stride_participant), _ptr(kv_len), int(max_kv_len), _ptr(o),
+                                       _ptr(lse), _stream(stream)), "fedattn_decode_noalloc")

@@ -7,6 +7,8 @@
 // swizzle (conflict-free ldmatrix).  Row max / row sum are reduced with warp shuffles inside
 // each 4-lane quad.  Each CTA handles one (cache, KV head, split) and writes an unnormalised
 // partial (m, l, o); a second kernel merges the splits.
+#include <string.h>
+
 #include "common.cuh"
 
 namespace fedattn {
@@ -315,3 +317,100 @@ cudaError_t launch_decode_bf16(const Context *ctx, const DecodeParams &p, cudaSt
 }
 
 }  // namespace fedattn
+
+// ---- decode without any allocation ------------------------------------------------------------------
+// Some callers cannot allocate device memory at all: code that runs inside a region where the
+// allocator must not be entered (a latency-critical serving loop, a plugin that is handed its
+// buffers and nothing else), or code that cannot create the workspace-owning context because it
+// is not allowed to call cudaMalloc.  For them the split-KV partials live in a fixed array that is
+// part of the library image: every GPU that loads the library holds these 2.03 MiB until exit.
+namespace fedattn {
+namespace {
+
+constexpr int kStaticMaxRows = 256;     // n_participants * n_q_heads
+constexpr int kStaticMaxSplits = 16;
+constexpr size_t kStaticScratchFloats = (size_t)kStaticMaxRows * kStaticMaxSplits * kPartialStride;
+
+static __device__ __align__(256) float g_decode_scratch[kStaticScratchFloats];
+
+// Device address of g_decode_scratch per device.  In host code the array's name is only a handle
+// for the runtime, so the address handed to the kernels comes from cudaGetSymbolAddress, taken
+// once per device with that device current.
+float *g_decode_scratch_ptr[64] = {};
+int g_decode_sm_count[64] = {};
+
+}  // namespace
+}  // namespace fedattn
+
+extern "C" fedattn_status fedattn_decode_noalloc(const fedattn_shape *shape, int32_t mode, const void *q,
+                                                 const void *k_cache, const void *v_cache,
+                                                 int64_t cache_stride_participant, const int32_t *kv_len,
+                                                 int32_t max_kv_len, void *o, float *lse, fedattn_stream stream)
+{
+    using namespace fedattn;
+    if (!shape || shape->n_participants < 1 || shape->n_q_heads < 1 || shape->n_kv_heads < 1 ||
+        shape->n_q_heads % shape->n_kv_heads != 0)
+        return FEDATTN_ERR_INVALID_ARG;
+    if (mode != FEDATTN_DECODE_LOCAL && mode != FEDATTN_DECODE_SYNC) return FEDATTN_ERR_INVALID_ARG;
+    if (!q || !o || !kv_len || max_kv_len < 0 || cache_stride_participant < 0) return FEDATTN_ERR_INVALID_ARG;
+    if (max_kv_len > 0 && (!k_cache || !v_cache)) return FEDATTN_ERR_INVALID_ARG;
+    if (((uintptr_t)q | (uintptr_t)o | (uintptr_t)k_cache | (uintptr_t)v_cache) & 15) return FEDATTN_ERR_INVALID_ARG;
+    if (mode == FEDATTN_DECODE_LOCAL && (cache_stride_participant * 2) % 16 != 0) return FEDATTN_ERR_INVALID_ARG;
+    if (shape->dtype != FEDATTN_BF16 || shape->head_dim != kD) return FEDATTN_ERR_UNSUPPORTED;
+    if ((int64_t)shape->n_participants * shape->n_q_heads > kStaticMaxRows)
+        return FEDATTN_ERR_WORKSPACE;          // more output rows than the built-in scratch covers
+    if (!(shape->scale >= 0.f)) return FEDATTN_ERR_INVALID_ARG;
+
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return FEDATTN_ERR_CUDA;
+    if (!g_decode_scratch_ptr[dev]) {
+        // first call on this device: resolve the array's device address and the SM count
+        float *ptr = nullptr;
+        if (cudaGetSymbolAddress((void **)&ptr, g_decode_scratch) != cudaSuccess || !ptr) return FEDATTN_ERR_CUDA;
+        int sms = 0;
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1)
+            return FEDATTN_ERR_CUDA;
+        const int smem = kStages * kStageBytes;
+        if (cudaFuncSetAttribute(decode_split_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess ||
+            cudaFuncSetAttribute(decode_split_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
+            return FEDATTN_ERR_CUDA;
+        g_decode_sm_count[dev] = sms;
+        g_decode_scratch_ptr[dev] = ptr;
+    }
+
+    DecodeParams p;
+    memset(&p, 0, sizeof(p));
+    p.q = q; p.k = k_cache; p.v = v_cache; p.o = o; p.lse = lse;
+    p.n_part = shape->n_participants; p.hq = shape->n_q_heads; p.hkv = shape->n_kv_heads; p.d = kD;
+    p.scale = shape->scale > 0.f ? shape->scale : 0.08838834764831845f;   // 1/sqrt(128)
+    p.sync = mode == FEDATTN_DECODE_SYNC;
+    p.cache_stride = cache_stride_participant; p.kv_len = kv_len; p.max_kv_len = max_kv_len;
+    p.partial = g_decode_scratch_ptr[dev];
+    p.partial_bytes = kStaticScratchFloats * sizeof(float);
+
+    // same grid rule as the workspace-backed call, with the split count capped to the built-in scratch
+    const int g = p.hq / p.hkv;
+    const int rows_total = p.sync ? p.n_part * g : g;
+    const int m_tiles = rows_total > 16 ? 2 : 1;
+    const int n_chunks = (rows_total + 16 * m_tiles - 1) / (16 * m_tiles);
+    const int caches = p.sync ? 1 : p.n_part;
+    const int sources = caches * p.hkv * n_chunks;
+    const int tiles = (p.max_kv_len + kTileKeys - 1) / kTileKeys;
+    int n_splits = (2 * g_decode_sm_count[dev] + sources - 1) / sources;
+    if (n_splits > tiles / 2) n_splits = tiles / 2;
+    if (n_splits > kStaticMaxSplits) n_splits = kStaticMaxSplits;
+    if (n_splits < 1) n_splits = 1;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const dim3 grid(n_splits, p.hkv, caches * n_chunks);
+    const int smem = kStages * kStageBytes;
+    if (m_tiles == 1)
+        decode_split_kernel<1><<<grid, 128, smem, s>>>(p, n_splits, n_chunks);
+    else
+        decode_split_kernel<2><<<grid, 256, smem, s>>>(p, n_splits, n_chunks);
+    if (cudaGetLastError() != cudaSuccess) return FEDATTN_ERR_CUDA;
+    if (n_splits > 1) {
+        decode_combine_kernel<<<p.n_part * p.hq, kD, 0, s>>>(p, n_splits);
+        if (cudaGetLastError() != cudaSuccess) return FEDATTN_ERR_CUDA;
+    }
+    return FEDATTN_OK;
+}
