@@ -155,9 +155,10 @@ def run_ours(args):
     dev = torch.device("cuda", local_rank)
     bf = torch.bfloat16
 
+    n_sets = max(1, args.sets)
     # host inputs (pinned) -- also the e2e source
     host_sets = []
-    for s in range(N_SETS):
+    for s in range(n_sets):
         q, k, v = w.qkv(block=s)
         qd = w.decode_q(s)
         host_sets.append([torch.from_numpy(x).to(bf).pin_memory() for x in (q, k, v, qd)])
@@ -238,7 +239,7 @@ def run_ours(args):
         torch.cuda.synchronize()
 
     for i in range(max(args.warmup, 3)):
-        step(sets[i % N_SETS])
+        step(sets[i % n_sets])
     barrier()
 
     # ---- timed region: K steps, per-call events on the launching stream ----
@@ -252,7 +253,7 @@ def run_ours(args):
     t_start = torch.cuda.Event(enable_timing=True); t_end = torch.cuda.Event(enable_timing=True)
     t_start.record(stream)
     for i in range(K):
-        step(sets[i % N_SETS], evs[i])
+        step(sets[i % n_sets], evs[i])
     t_end.record(stream)
     barrier()
     total_ms = t_start.elapsed_time(t_end)
@@ -272,7 +273,7 @@ def run_ours(args):
     d2h = sum(x.numel() * x.element_size() for x in hout)
 
     def e2e_step(i):
-        b, hs = sets[i % N_SETS], host_sets[i % N_SETS]
+        b, hs = sets[i % n_sets], host_sets[i % n_sets]
         b.q.copy_(hs[0], non_blocking=True); b.k.copy_(hs[1], non_blocking=True)
         b.v.copy_(hs[2], non_blocking=True); b.qd.copy_(hs[3], non_blocking=True)
         step(b)
@@ -321,7 +322,7 @@ def run_ours(args):
             "config": {"workload": w.name, "participants": N, "tokens_per_participant": seqlens[0],
                        "q_heads": Hq, "kv_heads": Hkv, "head_dim": d, "sparse_keep": "1/4 per KV head",
                        "step": "local+concat+sync+topk+sparse_sync+decode_local+decode_sync",
-                       "l2": "%d rotating input/output sets of %d MB each (> 126 MB L2), no flush" % (N_SETS, set_mb),
+                       "l2": "%d rotating input/output sets of %d MB each (> 126 MB L2), no flush" % (n_sets, set_mb),
                        "parallelism": "replicas" if world > 1 else "single"},
             "clocks": clocks,
             "e2e": {"value": round(e2e_value, 3), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
@@ -412,6 +413,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sets", type=int, default=N_SETS,
+                    help="rotating input sets (1 keeps device memory small for a profiler capture)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

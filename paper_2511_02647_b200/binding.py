@@ -9,7 +9,8 @@ from typing import Optional, Sequence
 import torch
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
-_LIB_PATH = os.path.join(_PKG, "lib", "libfedattn.so")
+# FEDATTN_LIBRARY overrides the path of the shared library (e.g. an instrumented build).
+_LIB_PATH = os.environ.get("FEDATTN_LIBRARY") or os.path.join(_PKG, "lib", "libfedattn.so")
 
 F32, BF16 = 0, 1
 AGG_CONCAT, AGG_TOPK_KNORM, AGG_INDEXED = 0, 1, 2

@@ -28,12 +28,13 @@ namespace {
 constexpr int kTileM = 128;          // query rows per CTA
 constexpr int kTileN = 128;          // keys per KV tile
 constexpr int kD = 128;              // head dim
-constexpr int kThreads = 192;
+constexpr int kThreads = 320;         // warps 0-3 / 4-7: softmax warpgroups, 8: TMA producer, 9: MMA issuer
+constexpr int kProducerWarp = 8, kMmaWarp = 9;
 constexpr uint32_t kTileBytes = kTileM * kD * 2;      // 32 KB: one Q, K or V tile
 constexpr uint32_t kHalfBytes = kTileBytes / 2;       // one 64-column TMA box
-constexpr uint32_t kSmemBytes = 3 * kTileBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
-constexpr uint32_t kTmemCols = 256;
-constexpr uint32_t kColS = 0, kColP = 0, kColO = 128;
+constexpr uint32_t kSmemBytes = 6 * kTileBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr uint32_t kTmemCols = 512;
+constexpr uint32_t kColS = 0, kColO = 256;   // S (and P, aliased) of sub-tile t at kColS + 128 t; O at kColO + 128 t
 constexpr uint32_t kWaitLimit = 1u << 20;
 constexpr float kRescaleThreshold = 8.0f;
 
@@ -42,6 +43,14 @@ struct KernelParams {
     int32_t tile_cu[kMaxP + 1];      // prefix sum of query tiles per segment
     int32_t *status;
 };
+
+#ifdef FEDATTN_TRACE
+// Debug build only: cycle stamps of one CTA's pipeline events, [tile][event].
+__device__ long long g_trace[64 * 8];
+#define TRACE(j, e) do { if (blockIdx.x == gridDim.x / 2 && (j) < 64) g_trace[(j) * 8 + (e)] = clock64(); } while (0)
+#else
+#define TRACE(j, e) do { } while (0)
+#endif
 
 // ---- PTX wrappers ---------------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -137,6 +146,14 @@ __device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64
                    "r"(r[7]), "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]),          \
                    "r"(r[14]), "r"(r[15]) : "memory")
 
+#define FEDATTN_TMEM_LD16(taddr, r)                                                                          \
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 "                                                   \
+                 "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"                           \
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]),       \
+                   "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]),   \
+                   "=r"(r[14]), "=r"(r[15])                                                                  \
+                 : "r"(taddr) : "memory")
+
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
@@ -150,6 +167,35 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 {
     uint32_t r;
     asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+
+__device__ __forceinline__ uint64_t pack_f32x2(float lo, float hi)
+{
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack_f32x2(uint64_t v, float &lo, float &hi)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma_f32x2(uint64_t a, uint64_t b, uint64_t c)
+{
+    uint64_t r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+__device__ __forceinline__ uint64_t add_f32x2(uint64_t a, uint64_t b)
+{
+    uint64_t r;
+    asm("add.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ float max3(float a, float b, float c)
+{
+    float r;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
     return r;
 }
 
@@ -186,32 +232,40 @@ __device__ __forceinline__ int count_le(const int32_t *pos, int n, int x)
 
 }  // namespace
 
-__global__ void __launch_bounds__(kThreads, 2)
+__global__ void __launch_bounds__(kThreads, 1)
 prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                      const __grid_constant__ CUtensorMap map_v, const __grid_constant__ KernelParams kp)
 {
     extern __shared__ uint8_t smem_raw[];
     const PrefillParams &p = kp.p;
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    uint8_t *sQ = smem, *sK = smem + kTileBytes, *sV = smem + 2 * kTileBytes;
-    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + 3 * kTileBytes);
-    uint64_t *bar_q = bars + 0, *bar_k = bars + 1, *bar_v = bars + 2, *bar_s = bars + 3, *bar_p = bars + 4,
-             *bar_o = bars + 5;
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 8);
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(bars + 9);
+    uint8_t *sQ = smem;                                  // [2 sub-tiles][32 KB]
+    uint8_t *sK = smem + 2 * kTileBytes;                 // [2 stages][32 KB]
+    uint8_t *sV = smem + 4 * kTileBytes;                 // [2 stages][32 KB]
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + 6 * kTileBytes);
+    uint64_t *bar_q = bars + 0;
+    uint64_t *k_full = bars + 1, *k_empty = bars + 3, *v_full = bars + 5, *v_empty = bars + 7;
+    uint64_t *s_full = bars + 9, *p_full = bars + 11, *o_done = bars + 13;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 16);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(bars + 17);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
-    // ---- which query tile / head ------------------------------------------------------------------
+    // ---- which query tile / KV head / head pair ------------------------------------------------------
+    const int g = p.hq / p.hkv;
+    const int ppg = (g + 1) >> 1;                               // head pairs per KV head
     const int total_tiles = kp.tile_cu[p.n_seg];
-    const int tile_rank = blockIdx.x / p.hq;
-    const int h = blockIdx.x - tile_rank * p.hq;
-    const int tile_id = total_tiles - 1 - tile_rank;           // heavy (late) tiles first
+    const int per_tile = p.hkv * ppg;
+    const int tile_rank = blockIdx.x / per_tile;
+    const int rem = blockIdx.x - tile_rank * per_tile;
+    const int kvh = rem / ppg, pair = rem - kvh * ppg;
+    const int head0 = kvh * g + 2 * pair;                       // sub-tile t works on head0 + t
+    const bool valid1 = 2 * pair + 1 < g;                       // second head exists (g odd: last pair is single)
+    const int tile_id = total_tiles - 1 - tile_rank;            // heavy (late) tiles first
     int seg = 0;
     while (seg + 1 < p.n_seg && tile_id >= kp.tile_cu[seg + 1]) ++seg;
     const int q_row0 = p.cu[seg] + (tile_id - kp.tile_cu[seg]) * kTileM;
     const int n_valid = min(kTileM, p.cu[seg + 1] - q_row0);
-    const int kvh = h / (p.hq / p.hkv);
 
     // ---- allowed-prefix length c(row): keys kv_begin .. kv_begin + c - 1 are visible ---------------
     const int T = (int)p.total_kv;
@@ -233,12 +287,15 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
 
     // ---- setup ------------------------------------------------------------------------------------
     if (tid == 0) {
-        mbar_init(bar_q, 1); mbar_init(bar_k, 1); mbar_init(bar_v, 1);
-        mbar_init(bar_s, 1); mbar_init(bar_p, 128); mbar_init(bar_o, 1);
+        mbar_init(bar_q, 1);
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(k_full + i, 1); mbar_init(k_empty + i, 1); mbar_init(v_full + i, 1); mbar_init(v_empty + i, 1);
+            mbar_init(s_full + i, 1); mbar_init(p_full + i, 128); mbar_init(o_done + i, 1);
+        }
         *abort_flag = (*reinterpret_cast<volatile int32_t *>(kp.status) == FEDATTN_ERR_TIMEOUT) ? 1 : 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 4) {
+    if (warp == kProducerWarp) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                      ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -248,123 +305,196 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-    if (warp == 4) {
+    if (warp == kProducerWarp) {
         // ================= TMA producer =================
         if (lane == 0 && n_tiles > 0) {
             asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&map_q) : "memory");
             asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&map_k) : "memory");
             asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&map_v) : "memory");
-            mbar_expect_tx(bar_q, kTileBytes);
-            tma_load_3d(sQ, &map_q, bar_q, 0, h, q_row0);
-            tma_load_3d(sQ + kHalfBytes, &map_q, bar_q, 64, h, q_row0);
+            mbar_expect_tx(bar_q, valid1 ? 2 * kTileBytes : kTileBytes);
+            tma_load_3d(sQ, &map_q, bar_q, 0, head0, q_row0);
+            tma_load_3d(sQ + kHalfBytes, &map_q, bar_q, 64, head0, q_row0);
+            if (valid1) {
+                tma_load_3d(sQ + kTileBytes, &map_q, bar_q, 0, head0 + 1, q_row0);
+                tma_load_3d(sQ + kTileBytes + kHalfBytes, &map_q, bar_q, 64, head0 + 1, q_row0);
+            }
             for (int j = 0; j < n_tiles; ++j) {
+                const int st = j & 1, use = j >> 1;
                 const int row = kv_begin + j * kTileN;
                 const int c1 = p.kv_head_major ? row : kvh, c2 = p.kv_head_major ? kvh : row;
-                if (j > 0) mbar_wait(bar_s, (j - 1) & 1, abort_flag, kp.status);     // K buffer free
-                mbar_expect_tx(bar_k, kTileBytes);
-                tma_load_3d(sK, &map_k, bar_k, 0, c1, c2);
-                tma_load_3d(sK + kHalfBytes, &map_k, bar_k, 64, c1, c2);
-                if (j > 0) mbar_wait(bar_o, (j - 1) & 1, abort_flag, kp.status);     // V buffer free
-                mbar_expect_tx(bar_v, kTileBytes);
-                tma_load_3d(sV, &map_v, bar_v, 0, c1, c2);
-                tma_load_3d(sV + kHalfBytes, &map_v, bar_v, 64, c1, c2);
+                if (j >= 2) mbar_wait(k_empty + st, (use - 1) & 1, abort_flag, kp.status);
+                TRACE(j, 7);
+                mbar_expect_tx(k_full + st, kTileBytes);
+                tma_load_3d(sK + st * kTileBytes, &map_k, k_full + st, 0, c1, c2);
+                tma_load_3d(sK + st * kTileBytes + kHalfBytes, &map_k, k_full + st, 64, c1, c2);
+                if (j >= 2) mbar_wait(v_empty + st, (use - 1) & 1, abort_flag, kp.status);
+                mbar_expect_tx(v_full + st, kTileBytes);
+                tma_load_3d(sV + st * kTileBytes, &map_v, v_full + st, 0, c1, c2);
+                tma_load_3d(sV + st * kTileBytes + kHalfBytes, &map_v, v_full + st, 64, c1, c2);
             }
             if (*abort_flag) {
                 // give the copies still in flight a bounded chance to land before the CTA retires
-                for (uint32_t it = 0; it < 4096 && !mbar_try_wait(bar_k, (n_tiles - 1) & 1); ++it) {}
-                for (uint32_t it = 0; it < 4096 && !mbar_try_wait(bar_v, (n_tiles - 1) & 1); ++it) {}
+                for (int j = max(0, n_tiles - 2); j < n_tiles; ++j) {
+                    for (uint32_t it = 0; it < 4096 && !mbar_try_wait(k_full + (j & 1), (j >> 1) & 1); ++it) {}
+                    for (uint32_t it = 0; it < 4096 && !mbar_try_wait(v_full + (j & 1), (j >> 1) & 1); ++it) {}
+                }
                 for (uint32_t it = 0; it < 4096 && !mbar_try_wait(bar_q, 0); ++it) {}
             }
         }
-    } else if (warp == 5) {
+    } else if (warp == kMmaWarp) {
         // ================= MMA issuer =================
+        // Issue order  S0(0) S1(0) | PV0(0) S0(1) | PV1(0) S1(1) | PV0(1) S0(2) | ...  : while one sub-tile's
+        // softmax runs, the tensor pipe works on the other sub-tile.
         if (lane == 0 && n_tiles > 0) {
-            const uint32_t tS = tmem_base + kColS, tP = tmem_base + kColP, tO = tmem_base + kColO;
             const uint32_t aQ = smem_u32(sQ), aK = smem_u32(sK), aV = smem_u32(sV);
-            mbar_wait(bar_q, 0, abort_flag, kp.status);
-            for (int j = 0; j < n_tiles; ++j) {
-                mbar_wait(bar_k, j & 1, abort_flag, kp.status);
-                tc_fence_after();
+            const int n_sub = valid1 ? 2 : 1;
+            auto issue_s = [&](int t, int st) {
 #pragma unroll
                 for (int ks = 0; ks < kD / 16; ++ks) {
                     const uint32_t off = (ks >> 2) * kHalfBytes + (ks & 3) * 32;
-                    umma_ss(tS, make_desc(aQ + off, 16, 1024), make_desc(aK + off, 16, 1024), kIdescQK, ks > 0);
+                    umma_ss(tmem_base + kColS + t * 128, make_desc(aQ + t * kTileBytes + off, 16, 1024),
+                            make_desc(aK + st * kTileBytes + off, 16, 1024), kIdescQK, ks > 0);
                 }
-                tc_commit(bar_s);
-                mbar_wait(bar_p, j & 1, abort_flag, kp.status);
-                mbar_wait(bar_v, j & 1, abort_flag, kp.status);
-                tc_fence_after();
+            };
+            mbar_wait(bar_q, 0, abort_flag, kp.status);
+            mbar_wait(k_full + 0, 0, abort_flag, kp.status);
+            tc_fence_after();
+            for (int t = 0; t < n_sub; ++t) {
+                issue_s(t, 0);
+                tc_commit(s_full + t);
+            }
+            tc_commit(k_empty + 0);
+            for (int j = 0; j < n_tiles; ++j) {
+                const int st = j & 1, ph = (j >> 1) & 1;
+                const int st1 = (j + 1) & 1, ph1 = ((j + 1) >> 1) & 1;
+                for (int t = 0; t < n_sub; ++t) {
+                    mbar_wait(p_full + t, j & 1, abort_flag, kp.status);
+                    if (t == 0) mbar_wait(v_full + st, ph, abort_flag, kp.status);
+                    TRACE(j, 2 + t);
+                    tc_fence_after();
 #pragma unroll
-                for (int ks = 0; ks < kTileN / 16; ++ks)
-                    umma_ts(tO, tP + ks * 8, make_desc(aV + ks * 2048, kHalfBytes, 1024), kIdescPV, (j > 0 || ks > 0));
-                tc_commit(bar_o);
+                    for (int ks = 0; ks < kTileN / 16; ++ks)
+                        umma_ts(tmem_base + kColO + t * 128, tmem_base + kColS + t * 128 + ks * 8,
+                                make_desc(aV + st * kTileBytes + ks * 2048, kHalfBytes, 1024), kIdescPV,
+                                (j > 0 || ks > 0));
+                    tc_commit(o_done + t);
+                    if (t == n_sub - 1) tc_commit(v_empty + st);
+                    if (j + 1 < n_tiles) {
+                        if (t == 0) mbar_wait(k_full + st1, ph1, abort_flag, kp.status);
+                        issue_s(t, st1);
+                        tc_commit(s_full + t);
+                        if (t == n_sub - 1) tc_commit(k_empty + st1);
+                    }
+                    TRACE(j, 4 + 0 * t);
+                }
             }
         }
-    } else {
-        // ================= softmax + epilogue: thread = query row =================
-        const int r = tid;                                      // 0..127, TMEM lane
-        const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
-        const uint32_t tS = tmem_base + lane_base + kColS, tP = tmem_base + lane_base + kColP,
-                       tO = tmem_base + lane_base + kColO;
+    } else if (warp < 4 || valid1) {
+        // ================= softmax + epilogue: warpgroup = sub-tile, thread = query row =================
+        const int t = warp >> 2;                                // sub-tile 0 or 1
+        const int r = tid & 127;                                // query row = TMEM lane
+        const int h = head0 + t;
+        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+        const uint32_t tS = tmem_base + lane_base + kColS + t * 128, tP = tS,
+                       tO = tmem_base + lane_base + kColO + t * 128;
+        uint64_t *bar_s = s_full + t, *bar_p = p_full + t, *bar_o = o_done + t;
         const int c_r = prefix_len(r);
         const float sl2 = p.scale * 1.4426950408889634f;
+        const uint64_t sl2_2 = pack_f32x2(sl2, sl2);
         float m_used = 0.f, l = 0.f;
 
-        for (int j = 0; j < n_tiles; ++j) {
-            mbar_wait(bar_s, j & 1, abort_flag, kp.status);
-            tc_fence_after();
-            uint32_t s[128];
-            FEDATTN_TMEM_LD32(tS + 0, (s + 0));
-            FEDATTN_TMEM_LD32(tS + 32, (s + 32));
-            FEDATTN_TMEM_LD32(tS + 64, (s + 64));
-            FEDATTN_TMEM_LD32(tS + 96, (s + 96));
-            tmem_wait_ld();
-            const int lim = c_r - j * kTileN;                  // columns < lim are visible
-            if (lim < kTileN) {
+        // One chunk = 32 keys.  The exponent reference m_used is kept from earlier chunks; a chunk
+        // whose maximum exceeds it by more than 2^8 takes the slow path, which rescales what this
+        // row has accumulated so far (O in TMEM, the P chunks of this tile, l) to the new reference.
+        auto softmax_chunk = [&](int j, int cc, uint32_t (&s)[32], uint64_t &rowsum2) {
+            const int lim = c_r - j * kTileN - cc * 32;         // columns < lim of this chunk are visible
+            if (lim < 32) {
 #pragma unroll
-                for (int c = 0; c < 128; ++c)
+                for (int c = 0; c < 32; ++c)
                     if (c >= lim) s[c] = 0xff800000u;           // -inf
             }
             float mx = -INFINITY;
 #pragma unroll
-            for (int c = 0; c < 128; ++c) mx = fmaxf(mx, __uint_as_float(s[c]));
+            for (int c = 0; c < 32; c += 2) mx = max3(mx, __uint_as_float(s[c]), __uint_as_float(s[c + 1]));
             const float t_max = mx * sl2;
-            if (j == 0) {
+            if (j == 0 && cc == 0) {
                 m_used = (t_max == -INFINITY) ? 0.f : t_max;
             } else {
                 const bool need = t_max > m_used + kRescaleThreshold;
                 if (__any_sync(0xffffffffu, need)) {
                     const float alpha = need ? ex2(m_used - t_max) : 1.f;
-                    mbar_wait(bar_o, (j - 1) & 1, abort_flag, kp.status);   // O holds tiles 0..j-1
-                    tc_fence_after();
+                    if (j > 0) {
+                        mbar_wait(bar_o, (j - 1) & 1, abort_flag, kp.status);   // O holds tiles 0..j-1
+                        tc_fence_after();
+#pragma unroll 1
+                        for (int oc = 0; oc < 4; ++oc) {
+                            uint32_t o[32];
+                            FEDATTN_TMEM_LD32(tO + oc * 32, o);
+                            tmem_wait_ld();
 #pragma unroll
-                    for (int cc = 0; cc < 4; ++cc) {
-                        uint32_t o[32];
-                        FEDATTN_TMEM_LD32(tO + cc * 32, o);
+                            for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
+                            FEDATTN_TMEM_ST32(tO + oc * 32, o);
+                        }
+                    }
+#pragma unroll 1
+                    for (int pc = 0; pc < cc; ++pc) {           // P chunks of this tile written so far
+                        uint32_t pk[16];
+                        tmem_wait_st();
+                        FEDATTN_TMEM_LD16(tP + pc * 16, pk);
                         tmem_wait_ld();
 #pragma unroll
-                        for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
-                        FEDATTN_TMEM_ST32(tO + cc * 32, o);
+                        for (int c = 0; c < 16; ++c)
+                            pk[c] = pack_bf16(__uint_as_float(pk[c] << 16) * alpha,
+                                              __uint_as_float(pk[c] & 0xffff0000u) * alpha);
+                        FEDATTN_TMEM_ST16(tP + pc * 16, pk);
                     }
-                    if (need) { l *= alpha; m_used = t_max; }
+                    if (need) {
+                        float r0, r1;
+                        unpack_f32x2(rowsum2, r0, r1);
+                        rowsum2 = pack_f32x2(r0 * alpha, r1 * alpha);
+                        l *= alpha;
+                        m_used = t_max;
+                    }
                 }
             }
-            float rowsum = 0.f;
+            uint32_t pk[16];
+            const uint64_t negm2 = pack_f32x2(-m_used, -m_used);
 #pragma unroll
-            for (int cc = 0; cc < 4; ++cc) {
-                uint32_t pk[16];
-#pragma unroll
-                for (int c = 0; c < 16; ++c) {
-                    const float p0 = ex2(fmaf(__uint_as_float(s[cc * 32 + 2 * c]), sl2, -m_used));
-                    const float p1 = ex2(fmaf(__uint_as_float(s[cc * 32 + 2 * c + 1]), sl2, -m_used));
-                    rowsum += p0 + p1;
-                    pk[c] = pack_bf16(p0, p1);
-                }
-                FEDATTN_TMEM_ST16(tP + cc * 16, pk);
+            for (int c = 0; c < 16; ++c) {
+                float x0, x1;
+                unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(s[2 * c]), __uint_as_float(s[2 * c + 1])), sl2_2, negm2),
+                             x0, x1);
+                const float p0 = ex2(x0), p1 = ex2(x1);
+                rowsum2 = add_f32x2(rowsum2, pack_f32x2(p0, p1));
+                pk[c] = pack_bf16(p0, p1);
             }
-            l += rowsum;
+            FEDATTN_TMEM_ST16(tP + cc * 16, pk);
+        };
+
+        for (int j = 0; j < n_tiles; ++j) {
+            mbar_wait(bar_s, j & 1, abort_flag, kp.status);
+            if ((tid & 127) == 0) TRACE(j, 5 + 0 * t);
+            tc_fence_after();
+            uint32_t sa[32], sb[32];
+            uint64_t rowsum2 = 0;
+            FEDATTN_TMEM_LD32(tS + 0, sa);
+            tmem_wait_ld();
+            FEDATTN_TMEM_LD32(tS + 32, sb);
+            softmax_chunk(j, 0, sa, rowsum2);
+            tmem_wait_ld();
+            FEDATTN_TMEM_LD32(tS + 64, sa);
+            softmax_chunk(j, 1, sb, rowsum2);
+            tmem_wait_ld();
+            FEDATTN_TMEM_LD32(tS + 96, sb);
+            softmax_chunk(j, 2, sa, rowsum2);
+            tmem_wait_ld();
+            softmax_chunk(j, 3, sb, rowsum2);
+            float r0, r1;
+            unpack_f32x2(rowsum2, r0, r1);
+            l += r0 + r1;
             tmem_wait_st();
             tc_fence_before();
+            if ((tid & 127) == 0) TRACE(j, 6);
             mbar_arrive(bar_p);
         }
 
@@ -404,7 +534,7 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     // ---- teardown -----------------------------------------------------------------------------------
     tc_fence_before();
     __syncthreads();
-    if (warp == 4) {
+    if (warp == kProducerWarp) {
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
     }
 }
@@ -413,6 +543,13 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+#ifdef FEDATTN_TRACE
+extern "C" int fedattn_debug_read_trace(long long *host, int n)
+{
+    return (int)cudaMemcpyFromSymbol(host, g_trace, sizeof(long long) * n);
+}
+#endif
 
 bool prefill_sm100_supported(const Context *ctx) { return ctx->encode_tiled != nullptr; }
 
@@ -446,7 +583,8 @@ cudaError_t launch_prefill_sm100(const Context *ctx, const PrefillParams &p, cud
     kp.tile_cu[0] = 0;
     for (int n = 0; n < p.n_seg; ++n)
         kp.tile_cu[n + 1] = kp.tile_cu[n] + (p.cu[n + 1] - p.cu[n] + kTileM - 1) / kTileM;
-    const int64_t blocks = (int64_t)kp.tile_cu[p.n_seg] * p.hq;
+    const int g = p.hq / p.hkv;
+    const int64_t blocks = (int64_t)kp.tile_cu[p.n_seg] * p.hkv * ((g + 1) / 2);
     if (blocks == 0) return cudaSuccess;
     if (blocks > 0x7fffffffLL) return cudaErrorInvalidValue;
     CUtensorMap mq, mk, mv;

@@ -71,6 +71,26 @@ def test_single_participant_and_tiny(oracle):
         check_close(r.sync(q, k, v)[0], oracle.sync(q, k, v)[0], TOL["bf16"], str(lens))
 
 
+def test_growing_logits_exercise_the_rescale_path(oracle):
+    """Logits that grow along the key axis force the running-maximum reference to move many times
+    (within a tile and across tiles), so O, P and l are rescaled on the way."""
+    lens = [300, 260]
+    q, k, v = gen(13, lens, 4, 2, 128, "bf16")
+    ramp = (np.arange(sum(lens), dtype=np.float32) % 300 / 6.0)[:, None, None]
+    q = fi.round_to_bf16(np.abs(q))
+    k = fi.round_to_bf16(np.abs(k) * ramp)           # logits ~ +ramp * O(10): far beyond 2^8 per chunk
+    r = Runner(2, 4, 2, 128, "bf16", sum(lens))
+    o, lse = r.local(q, k, v, lens)
+    oo, ol = oracle.local(q, k, v, lens)
+    check_close(o, oo, TOL["bf16"], "rescale local")
+    assert np.abs(lse - ol).max() / np.abs(ol).max() < 1e-3
+    o, _ = r.sync(q, k, v)
+    check_close(o, oracle.sync(q, k, v)[0], TOL["bf16"], "rescale sync")
+    # and the opposite: the first keys dominate, later chunks underflow
+    k2 = fi.round_to_bf16(np.abs(k[::-1].copy()))
+    check_close(r.sync(q, k2, v)[0], oracle.sync(q, k2, v)[0], TOL["bf16"], "falling logits")
+
+
 def test_sync_with_explicit_query_positions(oracle):
     """One participant's rows against the global KV, positions given explicitly."""
     lens = [100, 60, 140]
