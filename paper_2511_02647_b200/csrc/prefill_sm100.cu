@@ -385,7 +385,7 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                         tc_commit(s_full + t);
                         if (t == n_sub - 1) tc_commit(k_empty + st1);
                     }
-                    TRACE(j, 4 + 0 * t);
+                    if (t == 1) TRACE(j, 4);
                 }
             }
         }
@@ -403,98 +403,77 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         const uint64_t sl2_2 = pack_f32x2(sl2, sl2);
         float m_used = 0.f, l = 0.f;
 
-        // One chunk = 32 keys.  The exponent reference m_used is kept from earlier chunks; a chunk
-        // whose maximum exceeds it by more than 2^8 takes the slow path, which rescales what this
-        // row has accumulated so far (O in TMEM, the P chunks of this tile, l) to the new reference.
-        auto softmax_chunk = [&](int j, int cc, uint32_t (&s)[32], uint64_t &rowsum2) {
-            const int lim = c_r - j * kTileN - cc * 32;         // columns < lim of this chunk are visible
-            if (lim < 32) {
+        for (int j = 0; j < n_tiles; ++j) {
+            mbar_wait(bar_s, j & 1, abort_flag, kp.status);
+            if ((tid & 127) == 0) TRACE(j, t ? 5 : 0);
+            tc_fence_after();
+            uint32_t s[128];
+            FEDATTN_TMEM_LD32(tS + 0, (s + 0));
+            FEDATTN_TMEM_LD32(tS + 32, (s + 32));
+            FEDATTN_TMEM_LD32(tS + 64, (s + 64));
+            FEDATTN_TMEM_LD32(tS + 96, (s + 96));
+            tmem_wait_ld();
+            const int lim = c_r - j * kTileN;                  // columns < lim are visible
+            if (lim < kTileN) {
 #pragma unroll
-                for (int c = 0; c < 32; ++c)
+                for (int c = 0; c < 128; ++c)
                     if (c >= lim) s[c] = 0xff800000u;           // -inf
             }
-            float mx = -INFINITY;
+            // row maximum: 8 independent chains, then a tree
+            float mx[8];
 #pragma unroll
-            for (int c = 0; c < 32; c += 2) mx = max3(mx, __uint_as_float(s[c]), __uint_as_float(s[c + 1]));
-            const float t_max = mx * sl2;
-            if (j == 0 && cc == 0) {
+            for (int i = 0; i < 8; ++i) mx[i] = fmaxf(__uint_as_float(s[2 * i]), __uint_as_float(s[2 * i + 1]));
+#pragma unroll
+            for (int c = 16; c < 128; c += 16)
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+                    mx[i] = max3(mx[i], __uint_as_float(s[c + 2 * i]), __uint_as_float(s[c + 2 * i + 1]));
+            const float t_max = fmaxf(max3(mx[0], mx[1], mx[2]), fmaxf(max3(mx[3], mx[4], mx[5]), fmaxf(mx[6], mx[7]))) * sl2;
+            if (j == 0) {
                 m_used = (t_max == -INFINITY) ? 0.f : t_max;
             } else {
+                // The exponent reference moves only when the maximum grew by more than 2^8; then what
+                // this row has accumulated so far (O in TMEM, l) is rescaled to the new reference.
                 const bool need = t_max > m_used + kRescaleThreshold;
                 if (__any_sync(0xffffffffu, need)) {
                     const float alpha = need ? ex2(m_used - t_max) : 1.f;
-                    if (j > 0) {
-                        mbar_wait(bar_o, (j - 1) & 1, abort_flag, kp.status);   // O holds tiles 0..j-1
-                        tc_fence_after();
+                    mbar_wait(bar_o, (j - 1) & 1, abort_flag, kp.status);   // O holds tiles 0..j-1
+                    tc_fence_after();
 #pragma unroll 1
-                        for (int oc = 0; oc < 4; ++oc) {
-                            uint32_t o[32];
-                            FEDATTN_TMEM_LD32(tO + oc * 32, o);
-                            tmem_wait_ld();
-#pragma unroll
-                            for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
-                            FEDATTN_TMEM_ST32(tO + oc * 32, o);
-                        }
-                    }
-#pragma unroll 1
-                    for (int pc = 0; pc < cc; ++pc) {           // P chunks of this tile written so far
-                        uint32_t pk[16];
-                        tmem_wait_st();
-                        FEDATTN_TMEM_LD16(tP + pc * 16, pk);
+                    for (int oc = 0; oc < 4; ++oc) {
+                        uint32_t o[32];
+                        FEDATTN_TMEM_LD32(tO + oc * 32, o);
                         tmem_wait_ld();
 #pragma unroll
-                        for (int c = 0; c < 16; ++c)
-                            pk[c] = pack_bf16(__uint_as_float(pk[c] << 16) * alpha,
-                                              __uint_as_float(pk[c] & 0xffff0000u) * alpha);
-                        FEDATTN_TMEM_ST16(tP + pc * 16, pk);
+                        for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
+                        FEDATTN_TMEM_ST32(tO + oc * 32, o);
                     }
-                    if (need) {
-                        float r0, r1;
-                        unpack_f32x2(rowsum2, r0, r1);
-                        rowsum2 = pack_f32x2(r0 * alpha, r1 * alpha);
-                        l *= alpha;
-                        m_used = t_max;
-                    }
+                    if (need) { l *= alpha; m_used = t_max; }
                 }
             }
-            uint32_t pk[16];
             const uint64_t negm2 = pack_f32x2(-m_used, -m_used);
+            uint64_t sum2[4] = {0, 0, 0, 0};
 #pragma unroll
-            for (int c = 0; c < 16; ++c) {
-                float x0, x1;
-                unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(s[2 * c]), __uint_as_float(s[2 * c + 1])), sl2_2, negm2),
-                             x0, x1);
-                const float p0 = ex2(x0), p1 = ex2(x1);
-                rowsum2 = add_f32x2(rowsum2, pack_f32x2(p0, p1));
-                pk[c] = pack_bf16(p0, p1);
+            for (int cc = 0; cc < 4; ++cc) {
+                uint32_t pk[16];
+#pragma unroll
+                for (int c = 0; c < 16; ++c) {
+                    float x0, x1;
+                    unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(s[cc * 32 + 2 * c]),
+                                                      __uint_as_float(s[cc * 32 + 2 * c + 1])), sl2_2, negm2), x0, x1);
+                    const float p0 = ex2(x0), p1 = ex2(x1);
+                    sum2[c & 3] = add_f32x2(sum2[c & 3], pack_f32x2(p0, p1));
+                    pk[c] = pack_bf16(p0, p1);
+                }
+                FEDATTN_TMEM_ST16(tP + cc * 16, pk);
             }
-            FEDATTN_TMEM_ST16(tP + cc * 16, pk);
-        };
-
-        for (int j = 0; j < n_tiles; ++j) {
-            mbar_wait(bar_s, j & 1, abort_flag, kp.status);
-            if ((tid & 127) == 0) TRACE(j, 5 + 0 * t);
-            tc_fence_after();
-            uint32_t sa[32], sb[32];
-            uint64_t rowsum2 = 0;
-            FEDATTN_TMEM_LD32(tS + 0, sa);
-            tmem_wait_ld();
-            FEDATTN_TMEM_LD32(tS + 32, sb);
-            softmax_chunk(j, 0, sa, rowsum2);
-            tmem_wait_ld();
-            FEDATTN_TMEM_LD32(tS + 64, sa);
-            softmax_chunk(j, 1, sb, rowsum2);
-            tmem_wait_ld();
-            FEDATTN_TMEM_LD32(tS + 96, sb);
-            softmax_chunk(j, 2, sa, rowsum2);
-            tmem_wait_ld();
-            softmax_chunk(j, 3, sb, rowsum2);
-            float r0, r1;
-            unpack_f32x2(rowsum2, r0, r1);
+            float r0, r1, r2, r3;
+            unpack_f32x2(add_f32x2(add_f32x2(sum2[0], sum2[1]), add_f32x2(sum2[2], sum2[3])), r0, r1);
+            (void)r2; (void)r3;
             l += r0 + r1;
             tmem_wait_st();
             tc_fence_before();
-            if ((tid & 127) == 0) TRACE(j, 6);
+            if ((tid & 127) == 0) TRACE(j, t ? 6 : 1);
             mbar_arrive(bar_p);
         }
 
