@@ -40,7 +40,10 @@ constexpr float kRescaleThreshold = 8.0f;
 
 struct KernelParams {
     PrefillParams p;
-    int32_t tile_cu[kMaxP + 1];      // prefix sum of query tiles per segment
+    int32_t ord_seg[kMaxP];          // segments sorted by query-tile count, descending
+    int32_t ord_nt[kMaxP];           // their query-tile counts
+    int32_t n_qtiles;                // total query tiles
+    int32_t n_items;                 // query tiles x KV heads x head pairs
     int32_t *status;
 };
 
@@ -232,6 +235,67 @@ __device__ __forceinline__ int count_le(const int32_t *pos, int n, int x)
 
 }  // namespace
 
+// One unit of work: a 128-row query tile x one pair of query heads that share a KV head.
+struct Item {
+    int kvh, head0, q_row0, n_valid, seg, kv_begin, n_tiles;
+    bool valid1;                       // the pair's second head exists (odd group size: last pair is single)
+    const int32_t *kvp;                // positions of this KV head's aggregated rows (sparse sync), or null
+};
+
+// allowed-prefix length c(row): keys kv_begin .. kv_begin + c - 1 are visible to query row r of the tile
+__device__ __forceinline__ int prefix_len(const PrefillParams &p, const Item &it, int r)
+{
+    const int pos = it.q_row0 + r;
+    const int T = (int)p.total_kv;
+    if (!p.sync) {
+        const int seg_len = p.cu[it.seg + 1] - p.cu[it.seg];
+        return p.causal ? min(pos - p.cu[it.seg] + 1, seg_len) : seg_len;
+    }
+    if (!p.causal) return T;
+    if (!it.kvp) return min(pos + 1, T);
+    return count_le(it.kvp, T, pos);
+}
+
+__device__ __forceinline__ Item decode_item(const KernelParams &kp, int item)
+{
+    const PrefillParams &p = kp.p;
+    Item it;
+    const int g = p.hq / p.hkv;
+    const int ppg = (g + 1) >> 1;                               // head pairs per KV head
+    const int per_tile = p.hkv * ppg;
+    const int tile_rank = item / per_tile;
+    const int rem = item - tile_rank * per_tile;
+    it.kvh = rem / ppg;
+    const int pair = rem - it.kvh * ppg;
+    it.head0 = it.kvh * g + 2 * pair;
+    it.valid1 = 2 * pair + 1 < g;
+    // Heavy tiles first: query tiles are ranked by their index inside their segment, descending
+    // (a causal tile's KV-tile count is that index + 1).  Level lv holds tile lv-1 of every segment
+    // that has at least lv tiles; above(lv) = number of tiles on higher levels.
+    auto above = [&](int lv) {
+        int a = 0;
+        for (int i = 0; i < p.n_seg && kp.ord_nt[i] > lv; ++i) a += kp.ord_nt[i] - lv;
+        return a;
+    };
+    int lo = 1, hi = kp.ord_nt[0];                              // largest lv with above(lv) <= tile_rank ... search
+    while (lo < hi) {                                           // smallest lv with above(lv) <= tile_rank
+        const int mid = (lo + hi) >> 1;
+        if (above(mid) <= tile_rank) hi = mid; else lo = mid + 1;
+    }
+    const int seg = kp.ord_seg[tile_rank - above(lo)];
+    it.seg = seg;
+    it.q_row0 = p.cu[seg] + (lo - 1) * kTileM;
+    it.n_valid = min(kTileM, p.cu[seg + 1] - it.q_row0);
+    it.kvp = p.kv_pos ? p.kv_pos + (p.kv_head_major ? (int64_t)it.kvh * p.total_kv : 0) : nullptr;
+    it.kv_begin = p.sync ? 0 : p.cu[seg];
+    it.n_tiles = (prefix_len(p, it, it.n_valid - 1) + kTileN - 1) / kTileN;
+    return it;
+}
+
+// Persistent kernel: one CTA per SM walks the work items item = blockIdx.x, blockIdx.x + gridDim.x, ...
+// Barrier phases run on: per-CTA counters of KV tiles (git) and of non-empty items (qn) give stages
+// and parities, so the producer prefetches the next item's K/V and Q while the current item's last
+// tiles and its epilogue are still in flight.
 __global__ void __launch_bounds__(kThreads, 1)
 prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                      const __grid_constant__ CUtensorMap map_v, const __grid_constant__ KernelParams kp)
@@ -243,54 +307,28 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     uint8_t *sK = smem + 2 * kTileBytes;                 // [2 stages][32 KB]
     uint8_t *sV = smem + 4 * kTileBytes;                 // [2 stages][32 KB]
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + 6 * kTileBytes);
-    uint64_t *bar_q = bars + 0;
-    uint64_t *k_full = bars + 1, *k_empty = bars + 3, *v_full = bars + 5, *v_empty = bars + 7;
-    uint64_t *s_full = bars + 9, *p_full = bars + 11, *o_done = bars + 13;
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 16);
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(bars + 17);
+    uint64_t *q_full = bars + 0, *q_empty = bars + 1;
+    uint64_t *k_full = bars + 2, *k_empty = bars + 4, *v_full = bars + 6, *v_empty = bars + 8;
+    uint64_t *s_full = bars + 10, *p_full = bars + 12, *o_done = bars + 14, *o_free = bars + 16;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 18);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(bars + 19);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-
-    // ---- which query tile / KV head / head pair ------------------------------------------------------
-    const int g = p.hq / p.hkv;
-    const int ppg = (g + 1) >> 1;                               // head pairs per KV head
-    const int total_tiles = kp.tile_cu[p.n_seg];
-    const int per_tile = p.hkv * ppg;
-    const int tile_rank = blockIdx.x / per_tile;
-    const int rem = blockIdx.x - tile_rank * per_tile;
-    const int kvh = rem / ppg, pair = rem - kvh * ppg;
-    const int head0 = kvh * g + 2 * pair;                       // sub-tile t works on head0 + t
-    const bool valid1 = 2 * pair + 1 < g;                       // second head exists (g odd: last pair is single)
-    const int tile_id = total_tiles - 1 - tile_rank;            // heavy (late) tiles first
-    int seg = 0;
-    while (seg + 1 < p.n_seg && tile_id >= kp.tile_cu[seg + 1]) ++seg;
-    const int q_row0 = p.cu[seg] + (tile_id - kp.tile_cu[seg]) * kTileM;
-    const int n_valid = min(kTileM, p.cu[seg + 1] - q_row0);
-
-    // ---- allowed-prefix length c(row): keys kv_begin .. kv_begin + c - 1 are visible ---------------
-    const int T = (int)p.total_kv;
-    const int32_t *kvp = p.kv_pos ? p.kv_pos + (p.kv_head_major ? (int64_t)kvh * T : 0) : nullptr;
-    int kv_begin = 0;
-    auto prefix_len = [&](int r) -> int {
-        const int pos = q_row0 + r;
-        if (!p.sync) {
-            const int seg_len = p.cu[seg + 1] - p.cu[seg];
-            return p.causal ? min(pos - p.cu[seg] + 1, seg_len) : seg_len;
-        }
-        if (!p.causal) return T;
-        if (!kvp) return min(pos + 1, T);
-        return count_le(kvp, T, pos);
+    const int n_items = kp.n_items;
+    const int n_rounds = (n_items + (int)gridDim.x - 1) / (int)gridDim.x;
+    // Static schedule: round k hands item k*G + c to CTA c, in reversed CTA order on odd rounds, so
+    // that with items sorted by cost every CTA gets a similar total.
+    auto item_of = [&](int k) -> int {
+        const int c = (k & 1) ? (int)gridDim.x - 1 - (int)blockIdx.x : (int)blockIdx.x;
+        return k * (int)gridDim.x + c;
     };
-    if (!p.sync) kv_begin = p.cu[seg];
-    const int c_last = prefix_len(n_valid - 1);
-    const int n_tiles = (c_last + kTileN - 1) / kTileN;
 
     // ---- setup ------------------------------------------------------------------------------------
     if (tid == 0) {
-        mbar_init(bar_q, 1);
+        mbar_init(q_full, 1); mbar_init(q_empty, 1);
         for (int i = 0; i < 2; ++i) {
             mbar_init(k_full + i, 1); mbar_init(k_empty + i, 1); mbar_init(v_full + i, 1); mbar_init(v_empty + i, 1);
-            mbar_init(s_full + i, 1); mbar_init(p_full + i, 128); mbar_init(o_done + i, 1);
+            mbar_init(s_full + i, 1); mbar_init(p_full + i, 128); mbar_init(o_done + i, 1); mbar_init(o_free + i, 128);
         }
         *abort_flag = (*reinterpret_cast<volatile int32_t *>(kp.status) == FEDATTN_ERR_TIMEOUT) ? 1 : 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -307,47 +345,57 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
 
     if (warp == kProducerWarp) {
         // ================= TMA producer =================
-        if (lane == 0 && n_tiles > 0) {
+        if (lane == 0) {
             asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&map_q) : "memory");
             asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&map_k) : "memory");
             asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&map_v) : "memory");
-            mbar_expect_tx(bar_q, valid1 ? 2 * kTileBytes : kTileBytes);
-            tma_load_3d(sQ, &map_q, bar_q, 0, head0, q_row0);
-            tma_load_3d(sQ + kHalfBytes, &map_q, bar_q, 64, head0, q_row0);
-            if (valid1) {
-                tma_load_3d(sQ + kTileBytes, &map_q, bar_q, 0, head0 + 1, q_row0);
-                tma_load_3d(sQ + kTileBytes + kHalfBytes, &map_q, bar_q, 64, head0 + 1, q_row0);
-            }
-            for (int j = 0; j < n_tiles; ++j) {
-                const int st = j & 1, use = j >> 1;
-                const int row = kv_begin + j * kTileN;
-                const int c1 = p.kv_head_major ? row : kvh, c2 = p.kv_head_major ? kvh : row;
-                if (j >= 2) mbar_wait(k_empty + st, (use - 1) & 1, abort_flag, kp.status);
-                TRACE(j, 7);
-                mbar_expect_tx(k_full + st, kTileBytes);
-                tma_load_3d(sK + st * kTileBytes, &map_k, k_full + st, 0, c1, c2);
-                tma_load_3d(sK + st * kTileBytes + kHalfBytes, &map_k, k_full + st, 64, c1, c2);
-                if (j >= 2) mbar_wait(v_empty + st, (use - 1) & 1, abort_flag, kp.status);
-                mbar_expect_tx(v_full + st, kTileBytes);
-                tma_load_3d(sV + st * kTileBytes, &map_v, v_full + st, 0, c1, c2);
-                tma_load_3d(sV + st * kTileBytes + kHalfBytes, &map_v, v_full + st, 64, c1, c2);
+            int git = 0, qn = 0;
+            for (int k = 0; k < n_rounds; ++k) {
+                const int item = item_of(k);
+                if (item >= n_items) continue;
+                const Item it = decode_item(kp, item);
+                if (it.n_tiles == 0) continue;
+                if (qn > 0) mbar_wait(q_empty, (qn - 1) & 1, abort_flag, kp.status);   // previous item's S MMAs done
+                mbar_expect_tx(q_full, it.valid1 ? 2 * kTileBytes : kTileBytes);
+                tma_load_3d(sQ, &map_q, q_full, 0, it.head0, it.q_row0);
+                tma_load_3d(sQ + kHalfBytes, &map_q, q_full, 64, it.head0, it.q_row0);
+                if (it.valid1) {
+                    tma_load_3d(sQ + kTileBytes, &map_q, q_full, 0, it.head0 + 1, it.q_row0);
+                    tma_load_3d(sQ + kTileBytes + kHalfBytes, &map_q, q_full, 64, it.head0 + 1, it.q_row0);
+                }
+                for (int j = 0; j < it.n_tiles; ++j) {
+                    const int gt = git + j, st = gt & 1, use = gt >> 1;
+                    const int row = it.kv_begin + j * kTileN;
+                    const int c1 = p.kv_head_major ? row : it.kvh, c2 = p.kv_head_major ? it.kvh : row;
+                    if (gt >= 2) mbar_wait(k_empty + st, (use - 1) & 1, abort_flag, kp.status);
+                    TRACE(j, 7);
+                    mbar_expect_tx(k_full + st, kTileBytes);
+                    tma_load_3d(sK + st * kTileBytes, &map_k, k_full + st, 0, c1, c2);
+                    tma_load_3d(sK + st * kTileBytes + kHalfBytes, &map_k, k_full + st, 64, c1, c2);
+                    if (gt >= 2) mbar_wait(v_empty + st, (use - 1) & 1, abort_flag, kp.status);
+                    mbar_expect_tx(v_full + st, kTileBytes);
+                    tma_load_3d(sV + st * kTileBytes, &map_v, v_full + st, 0, c1, c2);
+                    tma_load_3d(sV + st * kTileBytes + kHalfBytes, &map_v, v_full + st, 64, c1, c2);
+                }
+                git += it.n_tiles;
+                ++qn;
             }
             if (*abort_flag) {
                 // give the copies still in flight a bounded chance to land before the CTA retires
-                for (int j = max(0, n_tiles - 2); j < n_tiles; ++j) {
-                    for (uint32_t it = 0; it < 4096 && !mbar_try_wait(k_full + (j & 1), (j >> 1) & 1); ++it) {}
-                    for (uint32_t it = 0; it < 4096 && !mbar_try_wait(v_full + (j & 1), (j >> 1) & 1); ++it) {}
+                for (int gt = max(0, git - 2); gt < git; ++gt) {
+                    for (uint32_t w = 0; w < 4096 && !mbar_try_wait(k_full + (gt & 1), (gt >> 1) & 1); ++w) {}
+                    for (uint32_t w = 0; w < 4096 && !mbar_try_wait(v_full + (gt & 1), (gt >> 1) & 1); ++w) {}
                 }
-                for (uint32_t it = 0; it < 4096 && !mbar_try_wait(bar_q, 0); ++it) {}
+                if (qn > 0)
+                    for (uint32_t w = 0; w < 4096 && !mbar_try_wait(q_full, (qn - 1) & 1); ++w) {}
             }
         }
     } else if (warp == kMmaWarp) {
         // ================= MMA issuer =================
-        // Issue order  S0(0) S1(0) | PV0(0) S0(1) | PV1(0) S1(1) | PV0(1) S0(2) | ...  : while one sub-tile's
-        // softmax runs, the tensor pipe works on the other sub-tile.
-        if (lane == 0 && n_tiles > 0) {
+        // Issue order per item  S0(0) S1(0) | PV0(0) S0(1) | PV1(0) S1(1) | PV0(1) S0(2) | ...  : while one
+        // sub-tile's softmax runs, the tensor pipe works on the other sub-tile.
+        if (lane == 0) {
             const uint32_t aQ = smem_u32(sQ), aK = smem_u32(sK), aV = smem_u32(sV);
-            const int n_sub = valid1 ? 2 : 1;
             auto issue_s = [&](int t, int st) {
 #pragma unroll
                 for (int ks = 0; ks < kD / 16; ++ks) {
@@ -356,158 +404,192 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                             make_desc(aK + st * kTileBytes + off, 16, 1024), kIdescQK, ks > 0);
                 }
             };
-            mbar_wait(bar_q, 0, abort_flag, kp.status);
-            mbar_wait(k_full + 0, 0, abort_flag, kp.status);
-            tc_fence_after();
-            for (int t = 0; t < n_sub; ++t) {
-                issue_s(t, 0);
-                tc_commit(s_full + t);
-            }
-            tc_commit(k_empty + 0);
-            for (int j = 0; j < n_tiles; ++j) {
-                const int st = j & 1, ph = (j >> 1) & 1;
-                const int st1 = (j + 1) & 1, ph1 = ((j + 1) >> 1) & 1;
+            // git / qn count the KV tiles / items of sub-tile 0 (and of the K/V ring); gsub[1] / qsub[1]
+            // count only the items in which the pair's second head exists.
+            int git = 0, qn = 0, git1 = 0, qn1 = 0;
+            for (int k = 0; k < n_rounds; ++k) {
+                const int item = item_of(k);
+                if (item >= n_items) continue;
+                const Item it = decode_item(kp, item);
+                const int n = it.n_tiles;
+                if (n == 0) continue;
+                const int n_sub = it.valid1 ? 2 : 1;
+                mbar_wait(q_full, qn & 1, abort_flag, kp.status);
+                mbar_wait(k_full + (git & 1), (git >> 1) & 1, abort_flag, kp.status);
+                tc_fence_after();
                 for (int t = 0; t < n_sub; ++t) {
-                    mbar_wait(p_full + t, j & 1, abort_flag, kp.status);
-                    if (t == 0) mbar_wait(v_full + st, ph, abort_flag, kp.status);
-                    TRACE(j, 2 + t);
-                    tc_fence_after();
-#pragma unroll
-                    for (int ks = 0; ks < kTileN / 16; ++ks)
-                        umma_ts(tmem_base + kColO + t * 128, tmem_base + kColS + t * 128 + ks * 8,
-                                make_desc(aV + st * kTileBytes + ks * 2048, kHalfBytes, 1024), kIdescPV,
-                                (j > 0 || ks > 0));
-                    tc_commit(o_done + t);
-                    if (t == n_sub - 1) tc_commit(v_empty + st);
-                    if (j + 1 < n_tiles) {
-                        if (t == 0) mbar_wait(k_full + st1, ph1, abort_flag, kp.status);
-                        issue_s(t, st1);
-                        tc_commit(s_full + t);
-                        if (t == n_sub - 1) tc_commit(k_empty + st1);
-                    }
-                    if (t == 1) TRACE(j, 4);
+                    issue_s(t, git & 1);
+                    tc_commit(s_full + t);
                 }
+                tc_commit(k_empty + (git & 1));
+                if (n == 1) tc_commit(q_empty);
+                for (int j = 0; j < n; ++j) {
+                    const int gt = git + j, st = gt & 1, ph = (gt >> 1) & 1;
+                    const int st1 = (gt + 1) & 1, ph1 = ((gt + 1) >> 1) & 1;
+                    for (int t = 0; t < n_sub; ++t) {
+                        const int gsub = (t ? git1 : git) + j, qsub = t ? qn1 : qn;
+                        mbar_wait(p_full + t, gsub & 1, abort_flag, kp.status);
+                        if (t == 0) mbar_wait(v_full + st, ph, abort_flag, kp.status);
+                        if (j == 0 && qsub > 0) mbar_wait(o_free + t, (qsub - 1) & 1, abort_flag, kp.status);
+                        TRACE(j, 2 + t);
+                        tc_fence_after();
+#pragma unroll
+                        for (int ks = 0; ks < kTileN / 16; ++ks)
+                            umma_ts(tmem_base + kColO + t * 128, tmem_base + kColS + t * 128 + ks * 8,
+                                    make_desc(aV + st * kTileBytes + ks * 2048, kHalfBytes, 1024), kIdescPV,
+                                    (j > 0 || ks > 0));
+                        tc_commit(o_done + t);
+                        if (t == n_sub - 1) tc_commit(v_empty + st);
+                        if (j + 1 < n) {
+                            if (t == 0) mbar_wait(k_full + st1, ph1, abort_flag, kp.status);
+                            issue_s(t, st1);
+                            tc_commit(s_full + t);
+                            if (t == n_sub - 1) {
+                                tc_commit(k_empty + st1);
+                                if (j + 2 == n) tc_commit(q_empty);     // last S of this item issued
+                            }
+                        }
+                        if (t == 1) TRACE(j, 4);
+                    }
+                }
+                git += n;
+                ++qn;
+                if (it.valid1) { git1 += n; ++qn1; }
             }
         }
-    } else if (warp < 4 || valid1) {
+    } else {
         // ================= softmax + epilogue: warpgroup = sub-tile, thread = query row =================
         const int t = warp >> 2;                                // sub-tile 0 or 1
         const int r = tid & 127;                                // query row = TMEM lane
-        const int h = head0 + t;
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
         const uint32_t tS = tmem_base + lane_base + kColS + t * 128, tP = tS,
                        tO = tmem_base + lane_base + kColO + t * 128;
         uint64_t *bar_s = s_full + t, *bar_p = p_full + t, *bar_o = o_done + t;
-        const int c_r = prefix_len(r);
         const float sl2 = p.scale * 1.4426950408889634f;
         const uint64_t sl2_2 = pack_f32x2(sl2, sl2);
-        float m_used = 0.f, l = 0.f;
-
-        for (int j = 0; j < n_tiles; ++j) {
-            mbar_wait(bar_s, j & 1, abort_flag, kp.status);
-            if ((tid & 127) == 0) TRACE(j, t ? 5 : 0);
-            tc_fence_after();
-            uint32_t s[128];
-            FEDATTN_TMEM_LD32(tS + 0, (s + 0));
-            FEDATTN_TMEM_LD32(tS + 32, (s + 32));
-            FEDATTN_TMEM_LD32(tS + 64, (s + 64));
-            FEDATTN_TMEM_LD32(tS + 96, (s + 96));
-            tmem_wait_ld();
-            const int lim = c_r - j * kTileN;                  // columns < lim are visible
-            if (lim < kTileN) {
-#pragma unroll
-                for (int c = 0; c < 128; ++c)
-                    if (c >= lim) s[c] = 0xff800000u;           // -inf
-            }
-            // row maximum: 8 independent chains, then a tree
-            float mx[8];
-#pragma unroll
-            for (int i = 0; i < 8; ++i) mx[i] = fmaxf(__uint_as_float(s[2 * i]), __uint_as_float(s[2 * i + 1]));
-#pragma unroll
-            for (int c = 16; c < 128; c += 16)
-#pragma unroll
-                for (int i = 0; i < 8; ++i)
-                    mx[i] = max3(mx[i], __uint_as_float(s[c + 2 * i]), __uint_as_float(s[c + 2 * i + 1]));
-            const float t_max = fmaxf(max3(mx[0], mx[1], mx[2]), fmaxf(max3(mx[3], mx[4], mx[5]), fmaxf(mx[6], mx[7]))) * sl2;
-            if (j == 0) {
-                m_used = (t_max == -INFINITY) ? 0.f : t_max;
-            } else {
-                // The exponent reference moves only when the maximum grew by more than 2^8; then what
-                // this row has accumulated so far (O in TMEM, l) is rescaled to the new reference.
-                const bool need = t_max > m_used + kRescaleThreshold;
-                if (__any_sync(0xffffffffu, need)) {
-                    const float alpha = need ? ex2(m_used - t_max) : 1.f;
-                    mbar_wait(bar_o, (j - 1) & 1, abort_flag, kp.status);   // O holds tiles 0..j-1
-                    tc_fence_after();
-#pragma unroll 1
-                    for (int oc = 0; oc < 4; ++oc) {
-                        uint32_t o[32];
-                        FEDATTN_TMEM_LD32(tO + oc * 32, o);
-                        tmem_wait_ld();
-#pragma unroll
-                        for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
-                        FEDATTN_TMEM_ST32(tO + oc * 32, o);
-                    }
-                    if (need) { l *= alpha; m_used = t_max; }
-                }
-            }
-            const uint64_t negm2 = pack_f32x2(-m_used, -m_used);
-            uint64_t sum2[4] = {0, 0, 0, 0};
-#pragma unroll
-            for (int cc = 0; cc < 4; ++cc) {
-                uint32_t pk[16];
-#pragma unroll
-                for (int c = 0; c < 16; ++c) {
-                    float x0, x1;
-                    unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(s[cc * 32 + 2 * c]),
-                                                      __uint_as_float(s[cc * 32 + 2 * c + 1])), sl2_2, negm2), x0, x1);
-                    const float p0 = ex2(x0), p1 = ex2(x1);
-                    sum2[c & 3] = add_f32x2(sum2[c & 3], pack_f32x2(p0, p1));
-                    pk[c] = pack_bf16(p0, p1);
-                }
-                FEDATTN_TMEM_ST16(tP + cc * 16, pk);
-            }
-            float r0, r1, r2, r3;
-            unpack_f32x2(add_f32x2(add_f32x2(sum2[0], sum2[1]), add_f32x2(sum2[2], sum2[3])), r0, r1);
-            (void)r2; (void)r3;
-            l += r0 + r1;
-            tmem_wait_st();
-            tc_fence_before();
-            if ((tid & 127) == 0) TRACE(j, t ? 6 : 1);
-            mbar_arrive(bar_p);
-        }
-
-        // ---- epilogue: O / l -> bf16 -> global -------------------------------------------------------
-        const bool valid = r < n_valid;
-        __nv_bfloat16 *orow = reinterpret_cast<__nv_bfloat16 *>(p.o) + ((int64_t)(q_row0 + r) * p.hq + h) * kD;
-        if (n_tiles > 0) {
-            mbar_wait(bar_o, (n_tiles - 1) & 1, abort_flag, kp.status);
-            tc_fence_after();
-            const float inv = l > 0.f ? 1.f / l : 0.f;
-#pragma unroll
-            for (int cc = 0; cc < 4; ++cc) {
-                uint32_t o[32];
-                FEDATTN_TMEM_LD32(tO + cc * 32, o);
-                tmem_wait_ld();
+        int git = 0;
+        for (int k = 0; k < n_rounds; ++k) {
+            const int item = item_of(k);
+            if (item >= n_items) continue;
+            const Item it = decode_item(kp, item);
+            if (t == 1 && !it.valid1) continue;                 // git counts only tiles this warpgroup works on
+            const int n_tiles = it.n_tiles;
+            const int h = it.head0 + t;
+            const bool valid = r < it.n_valid;
+            __nv_bfloat16 *orow = reinterpret_cast<__nv_bfloat16 *>(p.o) + ((int64_t)(it.q_row0 + r) * p.hq + h) * kD;
+            float *lse_out = p.lse ? p.lse + (int64_t)(it.q_row0 + r) * p.hq + h : nullptr;
+            if (n_tiles == 0) {                                 // nothing visible to any row of the tile
                 if (valid) {
 #pragma unroll
-                    for (int c = 0; c < 32; c += 8) {
-                        uint4 w;
-                        w.x = pack_bf16(__uint_as_float(o[c + 0]) * inv, __uint_as_float(o[c + 1]) * inv);
-                        w.y = pack_bf16(__uint_as_float(o[c + 2]) * inv, __uint_as_float(o[c + 3]) * inv);
-                        w.z = pack_bf16(__uint_as_float(o[c + 4]) * inv, __uint_as_float(o[c + 5]) * inv);
-                        w.w = pack_bf16(__uint_as_float(o[c + 6]) * inv, __uint_as_float(o[c + 7]) * inv);
-                        *reinterpret_cast<uint4 *>(orow + cc * 32 + c) = w;
+                    for (int c = 0; c < kD; c += 8) *reinterpret_cast<uint4 *>(orow + c) = make_uint4(0, 0, 0, 0);
+                    if (lse_out) *lse_out = -INFINITY;
+                }
+                continue;
+            }
+            const int c_r = prefix_len(p, it, r);
+            float m_used = 0.f, l = 0.f;
+
+            for (int j = 0; j < n_tiles; ++j) {
+                const int gt = git + j;
+                mbar_wait(bar_s, gt & 1, abort_flag, kp.status);
+                if ((tid & 127) == 0) TRACE(j, t ? 5 : 0);
+                tc_fence_after();
+                uint32_t s[128];
+                FEDATTN_TMEM_LD32(tS + 0, (s + 0));
+                FEDATTN_TMEM_LD32(tS + 32, (s + 32));
+                FEDATTN_TMEM_LD32(tS + 64, (s + 64));
+                FEDATTN_TMEM_LD32(tS + 96, (s + 96));
+                tmem_wait_ld();
+                const int lim = c_r - j * kTileN;                  // columns < lim are visible
+                if (lim < kTileN) {
+#pragma unroll
+                    for (int c = 0; c < 128; ++c)
+                        if (c >= lim) s[c] = 0xff800000u;           // -inf
+                }
+                // row maximum: 8 independent chains, then a tree
+                float mx[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) mx[i] = fmaxf(__uint_as_float(s[2 * i]), __uint_as_float(s[2 * i + 1]));
+#pragma unroll
+                for (int c = 16; c < 128; c += 16)
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        mx[i] = max3(mx[i], __uint_as_float(s[c + 2 * i]), __uint_as_float(s[c + 2 * i + 1]));
+                const float t_max =
+                    fmaxf(max3(mx[0], mx[1], mx[2]), fmaxf(max3(mx[3], mx[4], mx[5]), fmaxf(mx[6], mx[7]))) * sl2;
+                if (j == 0) {
+                    m_used = (t_max == -INFINITY) ? 0.f : t_max;
+                } else {
+                    // The exponent reference moves only when the maximum grew by more than 2^8; then what
+                    // this row has accumulated so far (O in TMEM, l) is rescaled to the new reference.
+                    const bool need = t_max > m_used + kRescaleThreshold;
+                    if (__any_sync(0xffffffffu, need)) {
+                        const float alpha = need ? ex2(m_used - t_max) : 1.f;
+                        mbar_wait(bar_o, (gt - 1) & 1, abort_flag, kp.status);   // O holds tiles 0..j-1
+                        tc_fence_after();
+#pragma unroll 1
+                        for (int oc = 0; oc < 4; ++oc) {
+                            uint32_t o[32];
+                            FEDATTN_TMEM_LD32(tO + oc * 32, o);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
+                            FEDATTN_TMEM_ST32(tO + oc * 32, o);
+                        }
+                        if (need) { l *= alpha; m_used = t_max; }
                     }
                 }
-            }
-        } else if (valid) {
+                const uint64_t negm2 = pack_f32x2(-m_used, -m_used);
+                uint64_t sum2[4] = {0, 0, 0, 0};
 #pragma unroll
-            for (int c = 0; c < kD; c += 8) *reinterpret_cast<uint4 *>(orow + c) = make_uint4(0, 0, 0, 0);
+                for (int cc = 0; cc < 4; ++cc) {
+                    uint32_t pk[16];
+#pragma unroll
+                    for (int c = 0; c < 16; ++c) {
+                        float x0, x1;
+                        unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(s[cc * 32 + 2 * c]),
+                                                          __uint_as_float(s[cc * 32 + 2 * c + 1])), sl2_2, negm2), x0, x1);
+                        const float p0 = ex2(x0), p1 = ex2(x1);
+                        sum2[c & 3] = add_f32x2(sum2[c & 3], pack_f32x2(p0, p1));
+                        pk[c] = pack_bf16(p0, p1);
+                    }
+                    FEDATTN_TMEM_ST16(tP + cc * 16, pk);
+                }
+                float r0, r1;
+                unpack_f32x2(add_f32x2(add_f32x2(sum2[0], sum2[1]), add_f32x2(sum2[2], sum2[3])), r0, r1);
+                l += r0 + r1;
+                tmem_wait_st();
+                tc_fence_before();
+                if ((tid & 127) == 0) TRACE(j, t ? 6 : 1);
+                mbar_arrive(bar_p);
+            }
+
+            // ---- epilogue: drain O from TMEM (frees it for the next item), then O / l -> bf16 -> global
+            mbar_wait(bar_o, (git + n_tiles - 1) & 1, abort_flag, kp.status);
+            tc_fence_after();
+            uint32_t o[128];
+            FEDATTN_TMEM_LD32(tO + 0, (o + 0));
+            FEDATTN_TMEM_LD32(tO + 32, (o + 32));
+            FEDATTN_TMEM_LD32(tO + 64, (o + 64));
+            FEDATTN_TMEM_LD32(tO + 96, (o + 96));
+            tmem_wait_ld();
+            tc_fence_before();
+            mbar_arrive(o_free + t);
+            if (valid) {
+                const float inv = l > 0.f ? 1.f / l : 0.f;
+#pragma unroll
+                for (int c = 0; c < 128; c += 8) {
+                    uint4 w;
+                    w.x = pack_bf16(__uint_as_float(o[c + 0]) * inv, __uint_as_float(o[c + 1]) * inv);
+                    w.y = pack_bf16(__uint_as_float(o[c + 2]) * inv, __uint_as_float(o[c + 3]) * inv);
+                    w.z = pack_bf16(__uint_as_float(o[c + 4]) * inv, __uint_as_float(o[c + 5]) * inv);
+                    w.w = pack_bf16(__uint_as_float(o[c + 6]) * inv, __uint_as_float(o[c + 7]) * inv);
+                    *reinterpret_cast<uint4 *>(orow + c) = w;
+                }
+                if (lse_out) *lse_out = l > 0.f ? (m_used + log2f(l)) * 0.6931471805599453f : -INFINITY;
+            }
+            git += n_tiles;
         }
-        if (valid && p.lse)
-            p.lse[(int64_t)(q_row0 + r) * p.hq + h] =
-                l > 0.f ? (m_used + log2f(l)) * 0.6931471805599453f : -INFINITY;
     }
 
     // ---- teardown -----------------------------------------------------------------------------------
@@ -559,13 +641,26 @@ cudaError_t launch_prefill_sm100(const Context *ctx, const PrefillParams &p, cud
     KernelParams kp;
     kp.p = p;
     kp.status = ctx->status;
-    kp.tile_cu[0] = 0;
-    for (int n = 0; n < p.n_seg; ++n)
-        kp.tile_cu[n + 1] = kp.tile_cu[n] + (p.cu[n + 1] - p.cu[n] + kTileM - 1) / kTileM;
+    int64_t n_qtiles = 0;
+    for (int n = 0; n < p.n_seg; ++n) {
+        kp.ord_seg[n] = n;
+        kp.ord_nt[n] = (p.cu[n + 1] - p.cu[n] + kTileM - 1) / kTileM;
+        n_qtiles += kp.ord_nt[n];
+    }
+    for (int a = 1; a < p.n_seg; ++a)          // insertion sort by tile count, descending (stable)
+        for (int b = a; b > 0 && kp.ord_nt[b] > kp.ord_nt[b - 1]; --b) {
+            const int32_t tn = kp.ord_nt[b], ts = kp.ord_seg[b];
+            kp.ord_nt[b] = kp.ord_nt[b - 1]; kp.ord_seg[b] = kp.ord_seg[b - 1];
+            kp.ord_nt[b - 1] = tn; kp.ord_seg[b - 1] = ts;
+        }
+    if (n_qtiles > 0x7fffffffLL) return cudaErrorInvalidValue;
+    kp.n_qtiles = (int32_t)n_qtiles;
     const int g = p.hq / p.hkv;
-    const int64_t blocks = (int64_t)kp.tile_cu[p.n_seg] * p.hkv * ((g + 1) / 2);
-    if (blocks == 0) return cudaSuccess;
-    if (blocks > 0x7fffffffLL) return cudaErrorInvalidValue;
+    const int64_t items = n_qtiles * p.hkv * ((g + 1) / 2);
+    if (items == 0) return cudaSuccess;
+    if (items > 0x7fffffffLL) return cudaErrorInvalidValue;
+    kp.n_items = (int32_t)items;
+    const int64_t blocks = items < ctx->sm_count ? items : ctx->sm_count;     // persistent: one CTA per SM
     CUtensorMap mq, mk, mv;
     if (!encode_map(ctx, &mq, p.q, p.n_q_rows, p.hq, false) ||
         !encode_map(ctx, &mk, p.k, p.total_kv, p.hkv, p.kv_head_major != 0) ||

@@ -43,7 +43,7 @@ def test_cfg1_fp32_local_and_sync(oracle):
 
 
 @pytest.mark.parametrize("dtype,hq,hkv,d", [("f32", 4, 2, 32), ("f32", 2, 2, 128), ("bf16", 4, 2, 64),
-                                            ("bf16", 8, 2, 128), ("bf16", 4, 4, 128)])
+                                            ("bf16", 8, 2, 128), ("bf16", 4, 4, 128), ("bf16", 6, 2, 128)])
 @pytest.mark.parametrize("causal", [True, False])
 def test_ragged_segments_local_and_sync(oracle, dtype, hq, hkv, d, causal):
     """Ragged lengths incl. 1, 0 and non-multiples of the 128-row tile; several tiles per segment."""
