@@ -47,7 +47,7 @@ def library_path() -> str:
 
 def _load():
     if not os.path.exists(_LIB_PATH):
-        raise ImportError("FedAttn CUDA library missing: %s (run `python -m paper_2511_02647_b200.build` "
+        raise ImportError("FedAttn CUDA library missing: %s (run `python paper_2511_02647_b200/build.py` "
                           "or __graft_entry__.build()); there is no fallback path" % _LIB_PATH)
     lib = C.CDLL(_LIB_PATH)
     vp, i32, i64 = C.c_void_p, C.c_int32, C.c_int64
