@@ -19,6 +19,10 @@
 // stops waiting and runs to its normal end (TMEM is always released).
 #include <cuda.h>
 
+#include <stdio.h>
+#include <stdlib.h>
+#include <type_traits>
+
 #include "common.cuh"
 
 namespace fedattn {
@@ -28,13 +32,23 @@ namespace {
 constexpr int kTileM = 128;          // query rows per CTA
 constexpr int kTileN = 128;          // keys per KV tile
 constexpr int kD = 128;              // head dim
-constexpr int kThreads = 320;         // warps 0-3 / 4-7: softmax warpgroups, 8: TMA producer, 9: MMA issuer
-constexpr int kProducerWarp = 8, kMmaWarp = 9;
+#ifndef FEDATTN_SPLIT
+#define FEDATTN_SPLIT 2
+#endif
+constexpr int kSplit = FEDATTN_SPLIT; // softmax warpgroups; each owns kCols key columns of every S tile
+constexpr int kCols = kTileN / kSplit;
+constexpr int kSoftmaxThreads = 128 * kSplit;
+constexpr int kThreads = kSoftmaxThreads + 64;   // then one TMA producer warp and one MMA issuer warp
+constexpr int kProducerWarp = 4 * kSplit, kMmaWarp = 4 * kSplit + 1;
+static_assert(kSplit == 2 || kSplit == 4, "column split");
 constexpr uint32_t kTileBytes = kTileM * kD * 2;      // 32 KB: one Q, K or V tile
 constexpr uint32_t kHalfBytes = kTileBytes / 2;       // one 64-column TMA box
-constexpr uint32_t kSmemBytes = 6 * kTileBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr uint32_t kSmemBytes = 6 * kTileBytes + 1024 /*alignment slack*/ + 256 /*barriers*/ +
+                                4 * kSplit * kTileM * 4 /*row max / row sum exchange*/;
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kColS = 0, kColO = 256;   // S (and P, aliased) of sub-tile t at kColS + 128 t; O at kColO + 128 t
+// P (bf16 pairs) of keys kCols q .. kCols q + kCols - 1 sits at S column kCols q, i.e. inside the S
+// columns that the same softmax warpgroup reads
 constexpr uint32_t kWaitLimit = 1u << 20;
 constexpr float kRescaleThreshold = 8.0f;
 
@@ -49,8 +63,8 @@ struct KernelParams {
 
 #ifdef FEDATTN_TRACE
 // Debug build only: cycle stamps of one CTA's pipeline events, [tile][event].
-__device__ long long g_trace[64 * 8];
-#define TRACE(j, e) do { if (k == 0 && blockIdx.x == gridDim.x / 2 && (j) < 64) g_trace[(j) * 8 + (e)] = clock64(); } while (0)
+__device__ long long g_trace[64 * 16];
+#define TRACE(j, e) do { if (k == 0 && blockIdx.x == gridDim.x / 2 && (j) < 64) g_trace[(j) * 16 + (e)] = clock64(); } while (0)
 #else
 #define TRACE(j, e) do { } while (0)
 #endif
@@ -81,8 +95,18 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
 }
 // Bounded wait.  Returns false (after flagging the status word once) when the limit is reached or
 // another thread of this CTA already gave up.
+__device__ __forceinline__ bool mbar_test_wait(uint64_t *bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\t"
+                 "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+                 "selp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag, int32_t *status)
 {
+    if (mbar_test_wait(bar, parity)) return true;        // phase already over: skip the suspending wait
     for (uint32_t it = 0; it < kWaitLimit; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
@@ -210,6 +234,35 @@ __device__ __forceinline__ float max3(float a, float b, float c)
     return r;
 }
 
+// 2^x for a packed pair on the FMA/ALU pipes (no MUFU): x = n + f with n = round(x), |f| <= 1/2;
+// 2^f by a degree-3 minimax polynomial (relative error 7.5e-5, far below the bf16 rounding of P),
+// 2^n by adding n to the exponent field.  The magic constant 1.5 * 2^23 makes the low mantissa
+// bits of x + magic hold n.  x is clamped at -125 so that the exponent arithmetic cannot wrap:
+// anything smaller contributes 2^-125 instead of an even smaller value.  Needs x <= 100.
+#ifndef FEDATTN_POLY_MASK
+#define FEDATTN_POLY_MASK 0x49     // bit (c & 7) set: column pair c takes the polynomial instead of ex2.approx
+#endif
+__device__ __forceinline__ void exp2_poly_x2(uint64_t x2, float &p0, float &p1)
+{
+    float x0, x1;
+    unpack_f32x2(x2, x0, x1);
+    x0 = fmaxf(x0, -125.f); x1 = fmaxf(x1, -125.f);
+    const uint64_t xc = pack_f32x2(x0, x1);
+    const uint64_t magic = pack_f32x2(12582912.f, 12582912.f), neg_magic = pack_f32x2(-12582912.f, -12582912.f);
+    const uint64_t neg_one = pack_f32x2(-1.f, -1.f);
+    const uint64_t t2 = add_f32x2(xc, magic);
+    const uint64_t f2 = fma_f32x2(add_f32x2(t2, neg_magic), neg_one, xc);
+    uint64_t q2 = pack_f32x2(0.0551716685295105f, 0.0551716685295105f);
+    q2 = fma_f32x2(q2, f2, pack_f32x2(0.2426111251115799f, 0.2426111251115799f));
+    q2 = fma_f32x2(q2, f2, pack_f32x2(0.6932609677314758f, 0.6932609677314758f));
+    q2 = fma_f32x2(q2, f2, pack_f32x2(0.9999280571937561f, 0.9999280571937561f));
+    float q0, q1, t0, t1;
+    unpack_f32x2(q2, q0, q1);
+    unpack_f32x2(t2, t0, t1);
+    p0 = __int_as_float(__float_as_int(q0) + (__float_as_int(t0) << 23));
+    p1 = __int_as_float(__float_as_int(q1) + (__float_as_int(t1) << 23));
+}
+
 // Shared-memory matrix descriptor, 128-byte swizzle, 8-row groups 1024 bytes apart.
 //   K-major operand (Q, K): rows of 64 bf16 = 128 B; a tile is two such [128 x 64] halves.
 //   MN-major operand (V as B, N = head dim): 64 head-dim elements contiguous per key row;
@@ -317,9 +370,12 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + 6 * kTileBytes);
     uint64_t *q_full = bars + 0, *q_empty = bars + 1;
     uint64_t *k_full = bars + 2, *k_empty = bars + 4, *v_full = bars + 6, *v_empty = bars + 8;
-    uint64_t *s_full = bars + 10, *p_full = bars + 12, *o_done = bars + 14, *o_free = bars + 16;
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 18);
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(bars + 19);
+    uint64_t *s_full = bars + 10, *o_done = bars + 12, *o_free = bars + 14;
+    uint64_t *p_full = bars + 16;                        // [sub-tile][column part]
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 24);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(bars + 25);
+    float *x_max = reinterpret_cast<float *>(bars + 32);            // [2 buffers][kSplit column parts][128 rows]
+    float *x_sum = x_max + 2 * kSplit * kTileM;                     // [2 sub-tiles][kSplit column parts][128 rows]
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int n_items = kp.n_items;
@@ -336,7 +392,8 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         mbar_init(q_full, 1); mbar_init(q_empty, 1);
         for (int i = 0; i < 2; ++i) {
             mbar_init(k_full + i, 1); mbar_init(k_empty + i, 1); mbar_init(v_full + i, 1); mbar_init(v_empty + i, 1);
-            mbar_init(s_full + i, 1); mbar_init(p_full + i, 128); mbar_init(o_done + i, 1); mbar_init(o_free + i, 128);
+            mbar_init(s_full + i, 1); mbar_init(o_done + i, 1); mbar_init(o_free + i, kSoftmaxThreads / 32);
+            for (int q = 0; q < kSplit; ++q) mbar_init(p_full + kSplit * i + q, 4);
         }
         *abort_flag = (*reinterpret_cast<volatile int32_t *>(kp.status) == FEDATTN_ERR_TIMEOUT) ? 1 : 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -443,17 +500,22 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                 const int st1 = (gt + 1) & 1, ph1 = ((gt + 1) >> 1) & 1;
                 for (int t = 0; t < n_sub; ++t) {
                     const int gsub = (t ? git1 : git) + j, qsub = t ? qn1 : qn;
-                    mbar_wait(p_full + t, gsub & 1, abort_flag, kp.status);
                     if (t == 0) mbar_wait(v_full + st, ph, abort_flag, kp.status);
                     if (j == 0 && qsub > 0) mbar_wait(o_free + t, (qsub - 1) & 1, abort_flag, kp.status);
-                    if (lane == 0) TRACE(j, 2 + t);
-                    tc_fence_after();
-                    if (leader) {
 #pragma unroll
-                        for (int ks = 0; ks < kTileN / 16; ++ks)
-                            umma_ts(tmem_base + kColO + t * 128, tmem_base + kColS + t * 128 + ks * 8,
-                                    dV + (uint64_t)(st * (kTileBytes >> 4) + ks * (2048 >> 4)), kIdescPV,
-                                    (j > 0 || ks > 0));
+                    for (int q = 0; q < kSplit; ++q) {
+                        mbar_wait(p_full + kSplit * t + q, gsub & 1, abort_flag, kp.status);
+                        if (lane == 0 && q == 0) TRACE(j, 2 + t);
+                        tc_fence_after();
+                        if (leader) {
+#pragma unroll
+                            for (int kk = 0; kk < kCols / 16; ++kk) {
+                                const int ks = q * (kCols / 16) + kk;
+                                umma_ts(tmem_base + kColO + t * 128, tmem_base + kColS + t * 128 + q * kCols + kk * 8,
+                                        dV + (uint64_t)(st * (kTileBytes >> 4) + ks * (2048 >> 4)), kIdescPV,
+                                        (j > 0 || ks > 0));
+                            }
+                        }
                     }
                     commit(o_done + t);
                     if (t == n_sub - 1) commit(v_empty + st);
@@ -474,137 +536,200 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             if (it.valid1) { git1 += n; ++qn1; }
         }
     } else {
-        // ================= softmax + epilogue: warpgroup = sub-tile, thread = query row =================
-        const int t = warp >> 2;                                // sub-tile 0 or 1
+        // ================= softmax + epilogue =================
+        // All softmax warpgroups work on the same S tile: thread = (query row r = TMEM lane, column part hf).
+        // Warpgroup hf owns keys kCols hf .. kCols hf + kCols - 1 of every S tile and the same head-dim
+        // columns of O.  The two sub-tiles (heads) are served alternately, so while the
+        // softmax of one sub-tile runs the tensor pipe works on the other.  Row maxima are exchanged
+        // through shared memory once per tile, row sums once per item.
+        const int hf = warp >> 2;                               // column part 0 .. kSplit - 1
         const int r = tid & 127;                                // query row = TMEM lane
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-        const uint32_t tS = tmem_base + lane_base + kColS + t * 128, tP = tS,
-                       tO = tmem_base + lane_base + kColO + t * 128;
-        uint64_t *bar_s = s_full + t, *bar_p = p_full + t, *bar_o = o_done + t;
         const float sl2 = p.scale * 1.4426950408889634f;
         const uint64_t sl2_2 = pack_f32x2(sl2, sl2);
-        int git = 0;
-        for (int k = 0; k < n_rounds; ++k) {
+        int gsub0 = 0, gsub1 = 0;                               // KV tiles each sub-tile has been through
+        int xb = 0;                                             // exchange buffer parity
+        int k = 0;                                              // round of the static schedule
+        auto wg_sync = [&]() { asm volatile("bar.sync 1, %0;" ::"n"(kSoftmaxThreads) : "memory"); };
+
+        // One visit = the softmax of one S tile of one sub-tile.  kPartial: some row of the tile has masked
+        // columns (they become -inf and every exponential goes through ex2.approx, which maps -inf to 0);
+        // otherwise a fixed subset of the columns takes the polynomial so that the ex2 unit, which is as
+        // slow as the tensor pipe for this tile shape, is not the bottleneck.
+        auto visit = [&](auto partial_tag, int t, int j, int gt, int lim, float &m_used, float &l) {
+            constexpr bool kPartial = decltype(partial_tag)::value;
+            const uint32_t tS = tmem_base + lane_base + kColS + t * 128 + kCols * hf;   // fp32 S, this part
+            const uint32_t tP = tS;                                                      // bf16 P, this part
+            const uint32_t tO = tmem_base + lane_base + kColO + t * 128 + kCols * hf;
+            if (tid == 0 && t == 1) TRACE(j, 13);
+            mbar_wait(s_full + t, gt & 1, abort_flag, kp.status);
+            if (tid == 0) TRACE(j, t ? 5 : 0);
+            tc_fence_after();
+            uint32_t s[kCols];
+#pragma unroll
+            for (int c = 0; c < kCols; c += 32) FEDATTN_TMEM_LD32(tS + c, (s + c));
+            tmem_wait_ld();
+            if (tid == 0 && t == 0) TRACE(j, 8);
+            if (kPartial) {
+#pragma unroll
+                for (int c = 0; c < kCols; ++c)
+                    if (c >= lim) s[c] = 0xff800000u;           // -inf; columns < lim are visible
+            }
+            // partial row maximum: 8 independent chains, then a tree
+            float mx[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) mx[i] = fmaxf(__uint_as_float(s[2 * i]), __uint_as_float(s[2 * i + 1]));
+#pragma unroll
+            for (int c = 16; c < kCols; c += 16)
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+                    mx[i] = max3(mx[i], __uint_as_float(s[c + 2 * i]), __uint_as_float(s[c + 2 * i + 1]));
+            const float pm = fmaxf(max3(mx[0], mx[1], mx[2]), fmaxf(max3(mx[3], mx[4], mx[5]), fmaxf(mx[6], mx[7])));
+            // row maximum over all parts: post this thread's partial maximum, meet the threads that hold the
+            // other parts of the row (one softmax-wide barrier per visit), read theirs
+            x_max[(xb * kSplit + hf) * kTileM + r] = pm;
+            wg_sync();
+            float rm = pm;
+#pragma unroll
+            for (int q = 1; q < kSplit; ++q) rm = fmaxf(rm, x_max[(xb * kSplit + ((hf + q) & (kSplit - 1))) * kTileM + r]);
+            xb ^= 1;
+            const float t_max = rm * sl2;
+            if (tid == 0 && t == 0) TRACE(j, 10);
+            if (j == 0) {
+                m_used = (t_max == -INFINITY) ? 0.f : t_max;
+            } else {
+                // The exponent reference moves only when the maximum grew by more than 2^8; then what
+                // this row has accumulated so far (O in TMEM, l) is rescaled to the new reference.
+                const bool need = t_max > m_used + kRescaleThreshold;
+                if (__any_sync(0xffffffffu, need)) {
+                    const float alpha = need ? ex2(m_used - t_max) : 1.f;
+                    mbar_wait(o_done + t, (gt - 1) & 1, abort_flag, kp.status);   // O holds tiles 0..j-1
+                    tc_fence_after();
+#pragma unroll 1
+                    for (int oc = 0; oc < kCols / 32; ++oc) {
+                        uint32_t o[32];
+                        FEDATTN_TMEM_LD32(tO + oc * 32, o);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
+                        FEDATTN_TMEM_ST32(tO + oc * 32, o);
+                    }
+                    if (need) { l *= alpha; m_used = t_max; }
+                }
+            }
+            const uint64_t negm2 = pack_f32x2(-m_used, -m_used);
+            uint64_t sum2[4] = {0, 0, 0, 0};
+#pragma unroll
+            for (int cc = 0; cc < kCols / 32; ++cc) {
+                uint32_t pk[16];
+#pragma unroll
+                for (int c = 0; c < 16; ++c) {
+                    const uint64_t x2 = fma_f32x2(pack_f32x2(__uint_as_float(s[cc * 32 + 2 * c]),
+                                                             __uint_as_float(s[cc * 32 + 2 * c + 1])), sl2_2, negm2);
+                    float p0, p1;
+                    if (!kPartial && ((FEDATTN_POLY_MASK >> (c & 7)) & 1)) {
+                        exp2_poly_x2(x2, p0, p1);
+                    } else {
+                        float x0, x1;
+                        unpack_f32x2(x2, x0, x1);
+                        p0 = ex2(x0); p1 = ex2(x1);
+                    }
+                    sum2[c & 3] = add_f32x2(sum2[c & 3], pack_f32x2(p0, p1));
+                    pk[c] = pack_bf16(p0, p1);
+                }
+                FEDATTN_TMEM_ST16(tP + cc * 16, pk);
+            }
+            float r0, r1;
+            unpack_f32x2(add_f32x2(add_f32x2(sum2[0], sum2[1]), add_f32x2(sum2[2], sum2[3])), r0, r1);
+            l += r0 + r1;
+            if (tid == 0 && t == 0) TRACE(j, 11);
+            tmem_wait_st();
+            tc_fence_before();
+            if (tid == 0) TRACE(j, t ? 6 : 1);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(p_full + kSplit * t + hf);      // one arrival per warp
+            if (tid == 0 && t == 0) TRACE(j, 12);
+        };
+
+        for (k = 0; k < n_rounds; ++k) {
             const int item = item_of(k);
             if (item >= n_items) continue;
             const Item it = decode_item(kp, item);
-            if (t == 1 && !it.valid1) continue;                 // git counts only tiles this warpgroup works on
             const int n_tiles = it.n_tiles;
-            const int h = it.head0 + t;
+            const int n_sub = it.valid1 ? 2 : 1;
             const bool valid = r < it.n_valid;
-            __nv_bfloat16 *orow = reinterpret_cast<__nv_bfloat16 *>(p.o) + ((int64_t)(it.q_row0 + r) * p.hq + h) * kD;
-            float *lse_out = p.lse ? p.lse + (int64_t)(it.q_row0 + r) * p.hq + h : nullptr;
+            __nv_bfloat16 *orow0 = reinterpret_cast<__nv_bfloat16 *>(p.o) +
+                                   ((int64_t)(it.q_row0 + r) * p.hq + it.head0) * kD + kCols * hf;
+            float *lse0 = p.lse ? p.lse + (int64_t)(it.q_row0 + r) * p.hq + it.head0 : nullptr;
             if (n_tiles == 0) {                                 // nothing visible to any row of the tile
                 if (valid) {
+                    for (int t = 0; t < n_sub; ++t) {
 #pragma unroll
-                    for (int c = 0; c < kD; c += 8) *reinterpret_cast<uint4 *>(orow + c) = make_uint4(0, 0, 0, 0);
-                    if (lse_out) *lse_out = -INFINITY;
+                        for (int c = 0; c < kCols; c += 8) *reinterpret_cast<uint4 *>(orow0 + t * kD + c) = make_uint4(0, 0, 0, 0);
+                        if (lse0 && hf == 0) lse0[t] = -INFINITY;
+                    }
                 }
                 continue;
             }
-            const int c_r = prefix_len(p, it, r);
-            float m_used = 0.f, l = 0.f;
-
-            for (int j = 0; j < n_tiles; ++j) {
-                const int gt = git + j;
-                mbar_wait(bar_s, gt & 1, abort_flag, kp.status);
-                if ((tid & 127) == 0) TRACE(j, t ? 5 : 0);
-                tc_fence_after();
-                uint32_t s[128];
-                FEDATTN_TMEM_LD32(tS + 0, (s + 0));
-                FEDATTN_TMEM_LD32(tS + 32, (s + 32));
-                FEDATTN_TMEM_LD32(tS + 64, (s + 64));
-                FEDATTN_TMEM_LD32(tS + 96, (s + 96));
-                tmem_wait_ld();
-                const int lim = c_r - j * kTileN;                  // columns < lim are visible
-                if (lim < kTileN) {
-#pragma unroll
-                    for (int c = 0; c < 128; ++c)
-                        if (c >= lim) s[c] = 0xff800000u;           // -inf
+            const int c_r = prefix_len(p, it, r) - kCols * hf;     // visible keys, counted from this thread's first column
+            // prefix lengths do not decrease with the row, so KV tiles below row 0's prefix are unmasked for all rows
+            const int n_full = prefix_len(p, it, 0) / kTileN;
+            // state of the sub-tile being visited (a) and of the other one (b); swapped after every visit
+            float m_a = 0.f, l_a = 0.f, m_b = 0.f, l_b = 0.f;
+            const int n_visits = n_tiles * n_sub;
+            for (int v = 0; v < n_visits; ++v) {
+                const int t = n_sub == 2 ? (v & 1) : 0;
+                const int j = n_sub == 2 ? (v >> 1) : v;
+                const int gt = (t ? gsub1 : gsub0) + j;
+                if (j < n_full) visit(std::false_type{}, t, j, gt, kCols, m_a, l_a);
+                else visit(std::true_type{}, t, j, gt, c_r - j * kTileN, m_a, l_a);
+                if (tid == 0 && t == 0) TRACE(j, 9);
+                if (n_sub == 2) {
+                    float x = m_a; m_a = m_b; m_b = x;
+                    x = l_a; l_a = l_b; l_b = x;
                 }
-                // row maximum: 8 independent chains, then a tree
-                float mx[8];
-#pragma unroll
-                for (int i = 0; i < 8; ++i) mx[i] = fmaxf(__uint_as_float(s[2 * i]), __uint_as_float(s[2 * i + 1]));
-#pragma unroll
-                for (int c = 16; c < 128; c += 16)
-#pragma unroll
-                    for (int i = 0; i < 8; ++i)
-                        mx[i] = max3(mx[i], __uint_as_float(s[c + 2 * i]), __uint_as_float(s[c + 2 * i + 1]));
-                const float t_max =
-                    fmaxf(max3(mx[0], mx[1], mx[2]), fmaxf(max3(mx[3], mx[4], mx[5]), fmaxf(mx[6], mx[7]))) * sl2;
-                if (j == 0) {
-                    m_used = (t_max == -INFINITY) ? 0.f : t_max;
-                } else {
-                    // The exponent reference moves only when the maximum grew by more than 2^8; then what
-                    // this row has accumulated so far (O in TMEM, l) is rescaled to the new reference.
-                    const bool need = t_max > m_used + kRescaleThreshold;
-                    if (__any_sync(0xffffffffu, need)) {
-                        const float alpha = need ? ex2(m_used - t_max) : 1.f;
-                        mbar_wait(bar_o, (gt - 1) & 1, abort_flag, kp.status);   // O holds tiles 0..j-1
-                        tc_fence_after();
+            }
+            // after an even number of swaps (a) is sub-tile 0 again
+
+            // ---- epilogue: drain this thread's half of O from TMEM (frees it for the next item), exchange
+            //      the row sums, then O / l -> bf16 -> global
 #pragma unroll 1
-                        for (int oc = 0; oc < 4; ++oc) {
-                            uint32_t o[32];
-                            FEDATTN_TMEM_LD32(tO + oc * 32, o);
-                            tmem_wait_ld();
+            for (int t = 0; t < n_sub; ++t) {
+                const float m_t = t ? m_b : m_a, l_t = t ? l_b : l_a;
+                const uint32_t tO = tmem_base + lane_base + kColO + t * 128 + kCols * hf;
+                mbar_wait(o_done + t, ((t ? gsub1 : gsub0) + n_tiles - 1) & 1, abort_flag, kp.status);
+                tc_fence_after();
+                uint32_t o[kCols];
 #pragma unroll
-                            for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
-                            FEDATTN_TMEM_ST32(tO + oc * 32, o);
-                        }
-                        if (need) { l *= alpha; m_used = t_max; }
-                    }
-                }
-                const uint64_t negm2 = pack_f32x2(-m_used, -m_used);
-                uint64_t sum2[4] = {0, 0, 0, 0};
-#pragma unroll
-                for (int cc = 0; cc < 4; ++cc) {
-                    uint32_t pk[16];
-#pragma unroll
-                    for (int c = 0; c < 16; ++c) {
-                        float x0, x1;
-                        unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(s[cc * 32 + 2 * c]),
-                                                          __uint_as_float(s[cc * 32 + 2 * c + 1])), sl2_2, negm2), x0, x1);
-                        const float p0 = ex2(x0), p1 = ex2(x1);
-                        sum2[c & 3] = add_f32x2(sum2[c & 3], pack_f32x2(p0, p1));
-                        pk[c] = pack_bf16(p0, p1);
-                    }
-                    FEDATTN_TMEM_ST16(tP + cc * 16, pk);
-                }
-                float r0, r1;
-                unpack_f32x2(add_f32x2(add_f32x2(sum2[0], sum2[1]), add_f32x2(sum2[2], sum2[3])), r0, r1);
-                l += r0 + r1;
-                tmem_wait_st();
+                for (int c = 0; c < kCols; c += 32) FEDATTN_TMEM_LD32(tO + c, (o + c));
+                tmem_wait_ld();
                 tc_fence_before();
-                if ((tid & 127) == 0) TRACE(j, t ? 6 : 1);
-                mbar_arrive(bar_p);
-            }
-
-            // ---- epilogue: drain O from TMEM (frees it for the next item), then O / l -> bf16 -> global
-            mbar_wait(bar_o, (git + n_tiles - 1) & 1, abort_flag, kp.status);
-            tc_fence_after();
-            uint32_t o[128];
-            FEDATTN_TMEM_LD32(tO + 0, (o + 0));
-            FEDATTN_TMEM_LD32(tO + 32, (o + 32));
-            FEDATTN_TMEM_LD32(tO + 64, (o + 64));
-            FEDATTN_TMEM_LD32(tO + 96, (o + 96));
-            tmem_wait_ld();
-            tc_fence_before();
-            mbar_arrive(o_free + t);
-            if (valid) {
-                const float inv = l > 0.f ? 1.f / l : 0.f;
+                __syncwarp();
+                if (lane == 0) mbar_arrive(o_free + t);             // one arrival per warp
+                x_sum[(t * kSplit + hf) * kTileM + r] = l_t;
+                wg_sync();
+                float lt = 0.f;                                 // same summation order in every part of the row
 #pragma unroll
-                for (int c = 0; c < 128; c += 8) {
-                    uint4 w;
-                    w.x = pack_bf16(__uint_as_float(o[c + 0]) * inv, __uint_as_float(o[c + 1]) * inv);
-                    w.y = pack_bf16(__uint_as_float(o[c + 2]) * inv, __uint_as_float(o[c + 3]) * inv);
-                    w.z = pack_bf16(__uint_as_float(o[c + 4]) * inv, __uint_as_float(o[c + 5]) * inv);
-                    w.w = pack_bf16(__uint_as_float(o[c + 6]) * inv, __uint_as_float(o[c + 7]) * inv);
-                    *reinterpret_cast<uint4 *>(orow + c) = w;
+                for (int q = 0; q < kSplit; ++q) lt += x_sum[(t * kSplit + q) * kTileM + r];
+                if (valid) {
+                    const float inv = lt > 0.f ? 1.f / lt : 0.f;
+                    __nv_bfloat16 *orow = orow0 + t * kD;
+#pragma unroll
+                    for (int c = 0; c < kCols; c += 8) {
+                        uint4 w;
+                        w.x = pack_bf16(__uint_as_float(o[c + 0]) * inv, __uint_as_float(o[c + 1]) * inv);
+                        w.y = pack_bf16(__uint_as_float(o[c + 2]) * inv, __uint_as_float(o[c + 3]) * inv);
+                        w.z = pack_bf16(__uint_as_float(o[c + 4]) * inv, __uint_as_float(o[c + 5]) * inv);
+                        w.w = pack_bf16(__uint_as_float(o[c + 6]) * inv, __uint_as_float(o[c + 7]) * inv);
+                        *reinterpret_cast<uint4 *>(orow + c) = w;
+                    }
+                    if (lse0 && hf == 0) lse0[t] = lt > 0.f ? (m_t + log2f(lt)) * 0.6931471805599453f : -INFINITY;
                 }
-                if (lse_out) *lse_out = l > 0.f ? (m_used + log2f(l)) * 0.6931471805599453f : -INFINITY;
             }
-            git += n_tiles;
+            gsub0 += n_tiles;
+            if (n_sub == 2) gsub1 += n_tiles;
+            // x_sum of this item is read before the next item's epilogue writes it again: the next item's
+            // first wg_sync (row-max exchange or row-sum exchange) lies in between
         }
     }
 
@@ -685,12 +810,17 @@ cudaError_t launch_prefill_sm100(const Context *ctx, const PrefillParams &p, cud
     static bool attr_set[64] = {};
     if (!attr_set[ctx->device & 63]) {
         cudaError_t e = cudaFuncSetAttribute(prefill_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-        if (e != cudaSuccess) return e;
+        if (e != cudaSuccess) {
+            if (getenv("FEDATTN_DEBUG")) fprintf(stderr, "prefill_sm100_kernel attribute: %s\n", cudaGetErrorString(e));
+            return e;
+        }
         attr_set[ctx->device & 63] = true;
     }
     prefill_sm100_kernel<<<(unsigned)blocks, kThreads, kSmemBytes, s>>>(mq, mk, mv, kp);
     ++*launches;
-    return cudaGetLastError();
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess && getenv("FEDATTN_DEBUG")) fprintf(stderr, "prefill_sm100_kernel launch: %s\n", cudaGetErrorString(e));
+    return e;
 }
 
 }  // namespace fedattn
