@@ -174,7 +174,7 @@ fedattn_status fedattn_decode(fedattn_ctx *ctx, const fedattn_shape *shape, int3
  * must not be entered (inside a serving loop with a frozen memory plan, a plugin that receives
  * its tensors and nothing more, a process whose memory is fully pre-partitioned).  This entry
  * point takes no context and allocates nothing, on the host or on the device: the split-KV
- * partials go to a fixed 2.03 MiB array built into the library image, which every GPU that loads
+ * partials go to a fixed 2.07 MiB array built into the library image, which every GPU that loads
  * the library holds until the process exits.
  *
  * Same arguments, layouts and results as fedattn_decode (bf16, head_dim 128 only; anything else

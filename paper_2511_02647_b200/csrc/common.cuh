@@ -9,8 +9,11 @@
 
 namespace fedattn {
 
-// Workspace layout: [0, kStatusBytes) status words, then the scratch region.
-constexpr size_t kStatusBytes = 256;
+// Workspace layout: [0, 256) status words, [256, kStatusBytes) arrival counters of the split-KV decode
+// (zero between calls: the last arriver resets its counter), then the scratch region.
+constexpr size_t kStatusWords = 256;
+constexpr int kDecodeCounters = 4096;
+constexpr size_t kStatusBytes = kStatusWords + kDecodeCounters * sizeof(int32_t);
 constexpr int kMaxP = FEDATTN_MAX_PARTICIPANTS;
 // Upper bound on spin iterations of any in-kernel wait before it gives up.
 constexpr uint32_t kSpinLimit = 1u << 22;
@@ -104,8 +107,9 @@ struct DecodeParams {
     int64_t cache_stride;
     const int32_t *kv_len;
     int32_t max_kv_len;
-    float *partial;               // scratch
+    float *partial;               // scratch: per-split partial results
     size_t partial_bytes;
+    int32_t *counters;            // kDecodeCounters arrival counters, all zero between calls
 };
 size_t decode_scratch_bytes(int n_part, int hq, int d, int sm_count);
 cudaError_t launch_decode_bf16(const Context *ctx, const DecodeParams &p, cudaStream_t s, int64_t *launches);

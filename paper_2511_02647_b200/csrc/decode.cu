@@ -5,8 +5,13 @@
 // (mma.sync m16n8k16), which keeps the 32 flop/byte of the sync step far below the memory time.
 // K/V tiles of 64 keys stream through a 3-stage cp.async pipeline with a 16-byte-chunk XOR
 // swizzle (conflict-free ldmatrix).  Row max / row sum are reduced with warp shuffles inside
-// each 4-lane quad.  Each CTA handles one (cache, KV head, split) and writes an unnormalised
-// partial (m, l, o); a second kernel merges the splits.
+// each 4-lane quad.  Each CTA handles one (cache, KV head, split) and leaves an unnormalised
+// partial (m, l, o) in its shared memory.  The splits of one (cache, KV head) are launched as
+// thread-block clusters of up to 8 CTAs, which merge their partials through distributed shared
+// memory (each CTA of the cluster takes a share of the rows).  If a (cache, KV head) spans several
+// clusters, the cluster results go to global scratch and the CTA that arrives last for its rows
+// merges them, so a decode step is one launch and no CTA ever spins on another.
+#include <cooperative_groups.h>
 #include <string.h>
 
 #include "common.cuh"
@@ -21,7 +26,10 @@ constexpr int kStages = 3;
 constexpr int kTileBytes = kTileKeys * kD * 2;          // 16 KB (K or V)
 constexpr int kStageBytes = 2 * kTileBytes;             // K + V
 constexpr int kMaxSplits = 64;
-constexpr int kPartialStride = kD + 2;                  // m, l, o[128]
+constexpr int kPartialStride = kD + 4;                  // m, l, 2 pad, o[128]: o is 16-byte aligned
+constexpr int kMaxCluster = 8;                          // CTAs per cluster (portable maximum)
+constexpr int kMaxSlots = 16;                           // clusters per (cache, KV head): partials in global scratch
+constexpr int kCtaPartOffset = 72 * 1024;               // byte offset of the CTA's merged partial in shared memory
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -66,6 +74,84 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 __device__ __forceinline__ uint32_t swz(int row, int chunk) { return (uint32_t)(row * 256 + ((chunk ^ (row & 7)) << 4)); }
 
 }  // namespace
+
+
+// Merges the n cluster results (slots 0 .. n-1, n <= kMaxSlots) of `rows` stacked query rows row0,
+// row0 + row_step, ... of one (cache, KV head), normalises and writes o / lse.  Called by every thread
+// of the CTA; `sm` holds rows * (n + 2) floats.
+template <int kThreads>
+__device__ __forceinline__ void merge_slots(const DecodeParams &p, float *sm, int n, int cache, int kvh, int row0,
+                                            int row_step, int rows)
+{
+    const int tid = threadIdx.x;
+    const int g = p.hq / p.hkv;
+    auto out_row = [&](int srow) -> size_t {
+        const int part = p.sync ? srow / g : cache;
+        const int head = kvh * g + (p.sync ? srow % g : srow);
+        return (size_t)part * p.hq + head;
+    };
+    float *sc = sm, *big_m = sm + rows * n, *big_l = big_m + rows;          // sc[row][slot]
+    float2 *ml = reinterpret_cast<float2 *>(big_l + rows);                 // (m, l)[row][slot]
+    for (int i = tid; i < rows * n; i += kThreads) {
+        const int rr = i / n, k = i - rr * n;
+        ml[i] = __ldcg(reinterpret_cast<const float2 *>(p.partial + (out_row(row0 + rr * row_step) * n + k) * kPartialStride));
+    }
+    __syncthreads();
+    if (tid < rows) {
+        float mm = -INFINITY;
+        for (int k = 0; k < n; ++k) mm = fmaxf(mm, ml[tid * n + k].x);
+        const float ms = mm == -INFINITY ? 0.f : mm;
+        float ll = 0.f;
+        for (int k = 0; k < n; ++k) {
+            const float f = ex2(ml[tid * n + k].x - ms);
+            ll += ml[tid * n + k].y * f;
+            sc[tid * n + k] = f;
+        }
+        big_m[tid] = mm; big_l[tid] = ll;
+    }
+    __syncthreads();
+    for (int i = tid; i < rows * (kD / 4); i += kThreads) {
+        const int rr = i / (kD / 4), c4 = i - rr * (kD / 4);
+        const size_t orow = out_row(row0 + rr * row_step);
+        const float *src = p.partial + orow * n * kPartialStride + 4 + c4 * 4;
+        float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int k0 = 0; k0 < n; k0 += 4) {
+            float4 v[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+                if (k0 + k < n) v[k] = __ldcg(reinterpret_cast<const float4 *>(src + (size_t)(k0 + k) * kPartialStride));
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+                if (k0 + k < n) {
+                    const float f = sc[rr * n + k0 + k];
+                    a.x += v[k].x * f; a.y += v[k].y * f; a.z += v[k].z * f; a.w += v[k].w * f;
+                }
+        }
+        const float ll = big_l[rr], mm = big_m[rr];
+        const float inv = ll > 0.f ? 1.f / ll : 0.f;
+        __nv_bfloat162 lo = __floats2bfloat162_rn(a.x * inv, a.y * inv), hi = __floats2bfloat162_rn(a.z * inv, a.w * inv);
+        uint2 w;
+        w.x = *reinterpret_cast<uint32_t *>(&lo); w.y = *reinterpret_cast<uint32_t *>(&hi);
+        *reinterpret_cast<uint2 *>(reinterpret_cast<__nv_bfloat16 *>(p.o) + orow * kD + c4 * 4) = w;
+        if (c4 == 0 && p.lse) p.lse[orow] = ll > 0.f ? (mm + log2f(ll)) * 0.6931471805599453f : -INFINITY;
+    }
+}
+
+// true in exactly one CTA: the last of `expected` to call this for the counter (which it resets to zero)
+__device__ __forceinline__ bool arrive_last(int32_t *ctr, int expected, int *s_flag)
+{
+    __threadfence();                                            // this CTA's partials before its arrival
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const int prev = atomicAdd(ctr, 1);
+        *s_flag = prev == expected - 1;
+        if (*s_flag) *ctr = 0;                                  // ready for the next call
+    }
+    __syncthreads();
+    const bool last = *s_flag != 0;
+    if (last) __threadfence();                                  // the others' partials after their arrivals
+    return last;
+}
 
 // grid: x = split, y = KV head, z = cache * n_chunks + chunk   (cache = participant for LOCAL, 0 for SYNC)
 // block: 128 * kMTiles threads.  Warp w: M-tile w % kMTiles, key slice w / kMTiles (16 keys of every tile).
@@ -221,12 +307,11 @@ decode_split_kernel(const DecodeParams p, int n_splits, int n_chunks)
         }
     }
     __syncthreads();
-    // thread -> (M-tile, row, 4 consecutive columns... ) : 16 * kMTiles rows x 128 columns
+    // slices -> this CTA's partial (m, l, pad, pad, o[128]) per stacked row, kept in shared memory
+    float *cta_part = reinterpret_cast<float *>(smem + kCtaPartOffset);   // [16 * kMTiles][kPartialStride]
     for (int idx = tid; idx < 16 * kMTiles * kD; idx += 128 * kMTiles) {
         const int c = idx % kD, rr = idx / kD;                 // rr: row within CTA (mt' * 16 + r)
         const int mtp = rr >> 4, r = rr & 15;
-        const int srow = (chunk * kMTiles + mtp) * 16 + r;
-        if (srow >= rows_total) continue;
         float mm = -INFINITY;
 #pragma unroll
         for (int sl = 0; sl < 4; ++sl) mm = fmaxf(mm, red[((size_t)(sl * kMTiles + mtp) * 16 + r) * kPartialStride]);
@@ -239,47 +324,85 @@ decode_split_kernel(const DecodeParams p, int n_splits, int n_chunks)
             ll += w[1] * sc;
             oo += w[2 + c] * sc;
         }
+        float *dst = cta_part + rr * kPartialStride;
+        dst[4 + c] = oo;
+        if (c == 0) { dst[0] = mm; dst[1] = ll; }
+    }
+
+    // ---- cluster merge through distributed shared memory: rank k takes rows k, k + cs, ... ----
+    namespace cg = cooperative_groups;
+    cg::cluster_group cluster = cg::this_cluster();
+    const int cs = (int)cluster.num_blocks(), rank = (int)cluster.block_rank();
+    const int ncl = n_splits / cs, ci = split / cs;            // clusters per (cache, KV head); this cluster
+    const int row0 = chunk * kMTiles * 16, rows = min(kMTiles * 16, rows_total - row0);
+    const int my_rows = rows > rank ? (rows - rank + cs - 1) / cs : 0;
+    auto out_row = [&](int srow) -> size_t {
         const int part = p.sync ? srow / g : cache;
         const int head = kvh * g + (p.sync ? srow % g : srow);
-        const size_t orow = (size_t)part * p.hq + head;
-        if (n_splits == 1) {
-            reinterpret_cast<__nv_bfloat16 *>(p.o)[orow * kD + c] = __float2bfloat16_rn(ll > 0.f ? oo / ll : 0.f);
-            if (c == 0 && p.lse) p.lse[orow] = ll > 0.f ? (mm + log2f(ll)) * 0.6931471805599453f : -INFINITY;
+        return (size_t)part * p.hq + head;
+    };
+    cluster.sync();                                             // every CTA's partial is in place
+    for (int i = tid; i < my_rows * (kD / 4); i += 128 * kMTiles) {
+        const int k = i / (kD / 4), c4 = i - k * (kD / 4);
+        const int rr = rank + k * cs;
+        float2 ml[kMaxCluster];
+        float4 v[kMaxCluster];
+#pragma unroll
+        for (int q = 0; q < kMaxCluster; ++q)
+            if (q < cs) {
+                const float *peer = cluster.map_shared_rank(cta_part, q) + rr * kPartialStride;
+                ml[q] = *reinterpret_cast<const float2 *>(peer);
+                v[q] = *reinterpret_cast<const float4 *>(peer + 4 + c4 * 4);
+            }
+        float mm = -INFINITY;
+#pragma unroll
+        for (int q = 0; q < kMaxCluster; ++q)
+            if (q < cs) mm = fmaxf(mm, ml[q].x);
+        const float ms = mm == -INFINITY ? 0.f : mm;
+        float ll = 0.f;
+        float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int q = 0; q < kMaxCluster; ++q)
+            if (q < cs) {
+                const float f = ex2(ml[q].x - ms);
+                ll += ml[q].y * f;
+                a.x += v[q].x * f; a.y += v[q].y * f; a.z += v[q].z * f; a.w += v[q].w * f;
+            }
+        const size_t orow = out_row(row0 + rr);
+        if (ncl == 1) {
+            const float inv = ll > 0.f ? 1.f / ll : 0.f;
+            __nv_bfloat162 lo = __floats2bfloat162_rn(a.x * inv, a.y * inv), hi = __floats2bfloat162_rn(a.z * inv, a.w * inv);
+            uint2 w;
+            w.x = *reinterpret_cast<uint32_t *>(&lo); w.y = *reinterpret_cast<uint32_t *>(&hi);
+            *reinterpret_cast<uint2 *>(reinterpret_cast<__nv_bfloat16 *>(p.o) + orow * kD + c4 * 4) = w;
+            if (c4 == 0 && p.lse) p.lse[orow] = ll > 0.f ? (mm + log2f(ll)) * 0.6931471805599453f : -INFINITY;
         } else {
-            float *dst = p.partial + (orow * n_splits + split) * kPartialStride;
-            dst[2 + c] = oo;
-            if (c == 0) { dst[0] = mm; dst[1] = ll; }
+            float *dst = p.partial + (orow * ncl + ci) * kPartialStride;
+            *reinterpret_cast<float4 *>(dst + 4 + c4 * 4) = a;
+            if (c4 == 0) { dst[0] = mm; dst[1] = ll; }
         }
     }
-}
+    cluster.sync();                                             // peers are done reading this CTA's partial
+    if (ncl == 1 || my_rows == 0) return;
 
-// grid: one CTA per output row (participant, query head); 128 threads = head dim.
-__global__ void __launch_bounds__(kD)
-decode_combine_kernel(const DecodeParams p, int n_splits)
-{
-    const size_t orow = blockIdx.x;
-    const int c = threadIdx.x;
-    const float *src = p.partial + orow * n_splits * kPartialStride;
-    float mm = -INFINITY;
-    for (int s = 0; s < n_splits; ++s) mm = fmaxf(mm, src[s * kPartialStride]);
-    const float ms = mm == -INFINITY ? 0.f : mm;
-    float ll = 0.f, oo = 0.f;
-    for (int s = 0; s < n_splits; ++s) {
-        const float sc = ex2(src[s * kPartialStride] - ms);
-        ll += src[s * kPartialStride + 1] * sc;
-        oo += src[s * kPartialStride + 2 + c] * sc;
-    }
-    reinterpret_cast<__nv_bfloat16 *>(p.o)[orow * kD + c] = __float2bfloat16_rn(ll > 0.f ? oo / ll : 0.f);
-    if (c == 0 && p.lse) p.lse[orow] = ll > 0.f ? (mm + log2f(ll)) * 0.6931471805599453f : -INFINITY;
+    // ---- several clusters per (cache, KV head): the last to arrive for these rows merges them ----
+    __shared__ int s_flag;
+    const int source = blockIdx.z * gridDim.y + kvh;
+    if (!arrive_last(p.counters + source * kMaxCluster + rank, ncl, &s_flag)) return;
+    merge_slots<128 * kMTiles>(p, red, ncl, cache, kvh, row0 + rank, cs, my_rows);
 }
 
 size_t decode_scratch_bytes(int n_part, int hq, int d, int /*sm_count*/)
 {
     if (d != kD) return 0;
-    return (size_t)n_part * hq * kMaxSplits * kPartialStride * sizeof(float);
+    return (size_t)n_part * hq * kMaxSlots * kPartialStride * sizeof(float);
 }
 
-cudaError_t launch_decode_bf16(const Context *ctx, const DecodeParams &p, cudaStream_t s, int64_t *launches)
+// Grid rule shared by both entry points.  Splits are chosen so that the whole grid is resident at
+// once (two CTAs per SM): a grid slightly larger than that would run a nearly empty second wave.
+// The splits of one (cache, KV head) form clusters of cs = 1, 2, 4 or 8 CTAs along grid.x.
+static cudaError_t launch_decode_split(const DecodeParams &p, int sm_count, int max_slots, cudaStream_t s,
+                                       int64_t *launches)
 {
     const int g = p.hq / p.hkv;
     const int rows_total = p.sync ? p.n_part * g : g;
@@ -287,33 +410,54 @@ cudaError_t launch_decode_bf16(const Context *ctx, const DecodeParams &p, cudaSt
     const int n_chunks = (rows_total + 16 * m_tiles - 1) / (16 * m_tiles);
     const int caches = p.sync ? 1 : p.n_part;
     const int sources = caches * p.hkv * n_chunks;
+    if (sources * kMaxCluster > kDecodeCounters) return cudaErrorInvalidValue;
     const int tiles = (p.max_kv_len + kTileKeys - 1) / kTileKeys;
-    int n_splits = (2 * ctx->sm_count + sources - 1) / sources;
+    int n_splits = 2 * sm_count / sources;                     // rounded down: one wave
     if (n_splits > tiles / 2) n_splits = tiles / 2;            // at least two tiles per split
-    if (n_splits > kMaxSplits) n_splits = kMaxSplits;
     if (n_splits < 1) n_splits = 1;
-    if (n_splits > 1 && (size_t)p.n_part * p.hq * n_splits * kPartialStride * sizeof(float) > p.partial_bytes)
+    int cs = 1;
+    while (cs * 2 <= kMaxCluster && cs * 2 <= n_splits) cs *= 2;
+    int ncl = n_splits / cs;
+    if (ncl > max_slots) ncl = max_slots;
+    if (ncl > kMaxSlots) ncl = kMaxSlots;
+    n_splits = ncl * cs;
+    if (ncl > 1 && (size_t)p.n_part * p.hq * ncl * kPartialStride * sizeof(float) > p.partial_bytes)
         return cudaErrorInvalidValue;
-    const int smem = kStages * kStageBytes;                    // 96 KB (also covers the merge buffer)
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3(n_splits, p.hkv, caches * n_chunks);
+    cfg.blockDim = dim3(128 * m_tiles, 1, 1);
+    cfg.dynamicSmemBytes = kStages * kStageBytes;              // 96 KB (also covers the merge buffers)
+    cfg.stream = s;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = cs; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    cudaError_t e = m_tiles == 1 ? cudaLaunchKernelEx(&cfg, decode_split_kernel<1>, p, n_splits, n_chunks)
+                                 : cudaLaunchKernelEx(&cfg, decode_split_kernel<2>, p, n_splits, n_chunks);
+    if (launches) ++*launches;
+    return e != cudaSuccess ? e : cudaGetLastError();
+}
+
+static cudaError_t set_decode_smem_attr()
+{
+    const int smem = kStages * kStageBytes;
+    cudaError_t e = cudaFuncSetAttribute(decode_split_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(decode_split_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    return e;
+}
+
+cudaError_t launch_decode_bf16(const Context *ctx, const DecodeParams &p, cudaStream_t s, int64_t *launches)
+{
     static bool attr_set[64] = {};
     if (!attr_set[ctx->device & 63]) {
-        cudaError_t e = cudaFuncSetAttribute(decode_split_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-        if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(decode_split_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        cudaError_t e = set_decode_smem_attr();
         if (e != cudaSuccess) return e;
         attr_set[ctx->device & 63] = true;
     }
-    const dim3 grid(n_splits, p.hkv, caches * n_chunks);
-    if (m_tiles == 1)
-        decode_split_kernel<1><<<grid, 128, smem, s>>>(p, n_splits, n_chunks);
-    else
-        decode_split_kernel<2><<<grid, 256, smem, s>>>(p, n_splits, n_chunks);
-    ++*launches;
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess || n_splits == 1) return e;
-    decode_combine_kernel<<<p.n_part * p.hq, kD, 0, s>>>(p, n_splits);
-    ++*launches;
-    return cudaGetLastError();
+    return launch_decode_split(p, ctx->sm_count, kMaxSlots, s, launches);
 }
 
 }  // namespace fedattn
@@ -323,20 +467,23 @@ cudaError_t launch_decode_bf16(const Context *ctx, const DecodeParams &p, cudaSt
 // allocator must not be entered (a latency-critical serving loop, a plugin that is handed its
 // buffers and nothing else), or code that cannot create the workspace-owning context because it
 // is not allowed to call cudaMalloc.  For them the split-KV partials live in a fixed array that is
-// part of the library image: every GPU that loads the library holds these 2.03 MiB until exit.
+// part of the library image: every GPU that loads the library holds these 2.07 MiB until exit.
 namespace fedattn {
 namespace {
 
 constexpr int kStaticMaxRows = 256;     // n_participants * n_q_heads
-constexpr int kStaticMaxSplits = 16;
-constexpr size_t kStaticScratchFloats = (size_t)kStaticMaxRows * kStaticMaxSplits * kPartialStride;
+constexpr int kStaticMaxSlots = 16;       // cluster results per (cache, KV head)
+constexpr size_t kStaticScratchFloats = (size_t)kStaticMaxRows * kStaticMaxSlots * kPartialStride;
 
 static __device__ __align__(256) float g_decode_scratch[kStaticScratchFloats];
+// arrival counters of the split merge; zero at load, and every call leaves them zero again
+static __device__ __align__(256) int32_t g_decode_counters[kDecodeCounters];
 
 // Device address of g_decode_scratch per device.  In host code the array's name is only a handle
 // for the runtime, so the address handed to the kernels comes from cudaGetSymbolAddress, taken
 // once per device with that device current.
 float *g_decode_scratch_ptr[64] = {};
+int32_t *g_decode_counters_ptr[64] = {};
 int g_decode_sm_count[64] = {};
 
 }  // namespace
@@ -370,11 +517,11 @@ extern "C" fedattn_status fedattn_decode_noalloc(const fedattn_shape *shape, int
         int sms = 0;
         if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1)
             return FEDATTN_ERR_CUDA;
-        const int smem = kStages * kStageBytes;
-        if (cudaFuncSetAttribute(decode_split_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess ||
-            cudaFuncSetAttribute(decode_split_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
-            return FEDATTN_ERR_CUDA;
+        if (set_decode_smem_attr() != cudaSuccess) return FEDATTN_ERR_CUDA;
+        int32_t *cptr = nullptr;
+        if (cudaGetSymbolAddress((void **)&cptr, g_decode_counters) != cudaSuccess || !cptr) return FEDATTN_ERR_CUDA;
         g_decode_sm_count[dev] = sms;
+        g_decode_counters_ptr[dev] = cptr;
         g_decode_scratch_ptr[dev] = ptr;
     }
 
@@ -387,30 +534,11 @@ extern "C" fedattn_status fedattn_decode_noalloc(const fedattn_shape *shape, int
     p.cache_stride = cache_stride_participant; p.kv_len = kv_len; p.max_kv_len = max_kv_len;
     p.partial = g_decode_scratch_ptr[dev];
     p.partial_bytes = kStaticScratchFloats * sizeof(float);
+    p.counters = g_decode_counters_ptr[dev];
 
     // same grid rule as the workspace-backed call, with the split count capped to the built-in scratch
-    const int g = p.hq / p.hkv;
-    const int rows_total = p.sync ? p.n_part * g : g;
-    const int m_tiles = rows_total > 16 ? 2 : 1;
-    const int n_chunks = (rows_total + 16 * m_tiles - 1) / (16 * m_tiles);
-    const int caches = p.sync ? 1 : p.n_part;
-    const int sources = caches * p.hkv * n_chunks;
-    const int tiles = (p.max_kv_len + kTileKeys - 1) / kTileKeys;
-    int n_splits = (2 * g_decode_sm_count[dev] + sources - 1) / sources;
-    if (n_splits > tiles / 2) n_splits = tiles / 2;
-    if (n_splits > kStaticMaxSplits) n_splits = kStaticMaxSplits;
-    if (n_splits < 1) n_splits = 1;
-    cudaStream_t s = static_cast<cudaStream_t>(stream);
-    const dim3 grid(n_splits, p.hkv, caches * n_chunks);
-    const int smem = kStages * kStageBytes;
-    if (m_tiles == 1)
-        decode_split_kernel<1><<<grid, 128, smem, s>>>(p, n_splits, n_chunks);
-    else
-        decode_split_kernel<2><<<grid, 256, smem, s>>>(p, n_splits, n_chunks);
-    if (cudaGetLastError() != cudaSuccess) return FEDATTN_ERR_CUDA;
-    if (n_splits > 1) {
-        decode_combine_kernel<<<p.n_part * p.hq, kD, 0, s>>>(p, n_splits);
-        if (cudaGetLastError() != cudaSuccess) return FEDATTN_ERR_CUDA;
-    }
+    if (launch_decode_split(p, g_decode_sm_count[dev], kStaticMaxSlots, static_cast<cudaStream_t>(stream), nullptr) !=
+        cudaSuccess)
+        return FEDATTN_ERR_CUDA;
     return FEDATTN_OK;
 }
