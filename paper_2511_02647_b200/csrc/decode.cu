@@ -27,6 +27,7 @@ constexpr int kTileBytes = kTileKeys * kD * 2;          // 16 KB (K or V)
 constexpr int kStageBytes = 2 * kTileBytes;             // K + V
 constexpr int kMaxSplits = 64;
 constexpr int kPartialStride = kD + 4;                  // m, l, 2 pad, o[128]: o is 16-byte aligned
+constexpr float kRescaleThreshold = 8.0f;               // log2 units
 constexpr int kMaxCluster = 8;                          // CTAs per cluster (portable maximum)
 constexpr int kMaxSlots = 16;                           // clusters per (cache, KV head): partials in global scratch
 constexpr int kCtaPartOffset = 72 * 1024;               // byte offset of the CTA's merged partial in shared memory
@@ -154,19 +155,19 @@ __device__ __forceinline__ bool arrive_last(int32_t *ctr, int expected, int *s_f
 }
 
 // grid: x = split, y = KV head, z = cache * n_chunks + chunk   (cache = participant for LOCAL, 0 for SYNC)
-// block: 128 * kMTiles threads.  Warp w: M-tile w % kMTiles, key slice w / kMTiles (16 keys of every tile).
+// block: 128 threads.  Warp w takes key slice w (16 keys of every 64-key tile) for all kMTiles
+// 16-row M-tiles of the chunk, so each K/V fragment is read from shared memory once.
 template <int kMTiles>
-__global__ void __launch_bounds__(128 * kMTiles, 2)
+__global__ void __launch_bounds__(128, 2)
 decode_split_kernel(const DecodeParams p, int n_splits, int n_chunks)
 {
     extern __shared__ __align__(1024) uint8_t smem[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int mt = warp % kMTiles, slice = warp / kMTiles;
+    const int slice = warp;
     const int split = blockIdx.x, kvh = blockIdx.y;
     const int cache = blockIdx.z / n_chunks, chunk = blockIdx.z - cache * n_chunks;
     const int g = p.hq / p.hkv;
     const int rows_total = p.sync ? p.n_part * g : g;          // query rows sharing this cache + KV head
-    const int row_base = (chunk * kMTiles + mt) * 16;           // first stacked row of this warp's M-tile
 
     const int len = p.sync ? p.kv_len[0] : p.kv_len[cache];
     const int tiles_total = (len + kTileKeys - 1) / kTileKeys;
@@ -189,39 +190,51 @@ decode_split_kernel(const DecodeParams p, int n_splits, int n_chunks)
         return reinterpret_cast<const __nv_bfloat16 *>(p.q) + ((size_t)part * p.hq + head) * kD;
     };
 
-    // Q fragments (A operand, 16 x 128): 8 k-steps x 4 registers
-    uint32_t qf[8][4];
-    {
+    // Q fragments (A operand, 16 x 128 per M-tile): 8 k-steps x 4 registers
+    uint32_t qf[kMTiles][8][4];
+#pragma unroll
+    for (int im = 0; im < kMTiles; ++im) {
+        const int row_base = (chunk * kMTiles + im) * 16;       // first stacked row of this M-tile
         const __nv_bfloat16 *r0 = q_ptr(row_base + (lane >> 2)), *r1 = q_ptr(row_base + (lane >> 2) + 8);
         const int c = (lane & 3) * 2;
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks) {
-            qf[ks][0] = r0 ? *reinterpret_cast<const uint32_t *>(r0 + ks * 16 + c) : 0u;
-            qf[ks][1] = r1 ? *reinterpret_cast<const uint32_t *>(r1 + ks * 16 + c) : 0u;
-            qf[ks][2] = r0 ? *reinterpret_cast<const uint32_t *>(r0 + ks * 16 + c + 8) : 0u;
-            qf[ks][3] = r1 ? *reinterpret_cast<const uint32_t *>(r1 + ks * 16 + c + 8) : 0u;
+            qf[im][ks][0] = r0 ? *reinterpret_cast<const uint32_t *>(r0 + ks * 16 + c) : 0u;
+            qf[im][ks][1] = r1 ? *reinterpret_cast<const uint32_t *>(r1 + ks * 16 + c) : 0u;
+            qf[im][ks][2] = r0 ? *reinterpret_cast<const uint32_t *>(r0 + ks * 16 + c + 8) : 0u;
+            qf[im][ks][3] = r1 ? *reinterpret_cast<const uint32_t *>(r1 + ks * 16 + c + 8) : 0u;
         }
     }
 
+    // K and V tiles: 64 rows x 16 chunks of 16 bytes each.  Thread tid copies chunk (tid & 15) of rows
+    // (tid >> 4) + 8 i, i = 0..7; the row's swizzle term (row & 7) is the same for all i, so the global
+    // and shared offsets are fixed per thread up to a multiple of 8 rows.  Rows past `len` are zero-filled.
+    const int ld_row = tid >> 4, ld_ch = tid & 15;
+    const __nv_bfloat16 *ld_k = Kb + (size_t)ld_row * tok_stride + ld_ch * 8, *ld_v = Vb + (size_t)ld_row * tok_stride + ld_ch * 8;
+    const uint32_t ld_s = smem_u32(smem) + swz(ld_row, ld_ch);
     auto load_tile = [&](int t, int stage) {
-        // K and V tiles: 64 rows x 16 chunks each; rows past `len` are zero-filled
         const int key0 = (tile_lo + t) * kTileKeys;
-        const uint32_t sK = smem_u32(smem) + stage * kStageBytes, sV = sK + kTileBytes;
+        const uint32_t sK = ld_s + stage * kStageBytes, sV = sK + kTileBytes;
+        const size_t base = (size_t)key0 * tok_stride;
+        const int n_ok = len - key0 - ld_row;                  // rows ld_row + 8 i with 8 i < n_ok exist
 #pragma unroll
-        for (int i = tid; i < kTileKeys * 16; i += 128 * kMTiles) {
-            const int row = i >> 4, ch = i & 15;
-            const bool ok = key0 + row < len;
-            const size_t off = (size_t)(ok ? key0 + row : 0) * tok_stride + ch * 8;
-            cp_async16(sK + swz(row, ch), Kb + off, ok);
-            cp_async16(sV + swz(row, ch), Vb + off, ok);
+        for (int i = 0; i < kTileKeys / 8; ++i) {
+            const bool ok = 8 * i < n_ok;
+            const size_t off = ok ? base + (size_t)(8 * i) * tok_stride : 0;
+            cp_async16(sK + i * 8 * 256, ld_k + off, ok);
+            cp_async16(sV + i * 8 * 256, ld_v + off, ok);
         }
     };
 
     const float sl2 = p.scale * 1.4426950408889634f;
-    float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;   // rows lane/4 and lane/4 + 8
-    float acc[16][4];
+    float m0[kMTiles], m1[kMTiles], l0[kMTiles], l1[kMTiles];  // rows lane/4 and lane/4 + 8 of each M-tile
+    float acc[kMTiles][16][4];
 #pragma unroll
-    for (int i = 0; i < 16; ++i) acc[i][0] = acc[i][1] = acc[i][2] = acc[i][3] = 0.f;
+    for (int im = 0; im < kMTiles; ++im) {
+        m0[im] = m1[im] = -INFINITY; l0[im] = l1[im] = 0.f;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) acc[im][i][0] = acc[im][i][1] = acc[im][i][2] = acc[im][i][3] = 0.f;
+    }
 
 #pragma unroll
     for (int s = 0; s < kStages - 1; ++s) {
@@ -236,8 +249,12 @@ decode_split_kernel(const DecodeParams p, int n_splits, int n_chunks)
 
         const uint32_t sK = smem_u32(smem) + (t % kStages) * kStageBytes, sV = sK + kTileBytes;
         const int krow0 = slice * 16;
-        // ---- S = Q K^T for this warp's 16 keys: two n-tiles of 8 keys ----
-        float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
+        // ---- S = Q K^T for this warp's 16 keys: two n-tiles of 8 keys per M-tile ----
+        float s0[kMTiles][4], s1[kMTiles][4];
+#pragma unroll
+        for (int im = 0; im < kMTiles; ++im)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) s0[im][i] = s1[im][i] = 0.f;
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks) {
             // matrices: (keys 0-7, d 0-7) (keys 0-7, d 8-15) (keys 8-15, d 0-7) (keys 8-15, d 8-15)
@@ -245,36 +262,51 @@ decode_split_kernel(const DecodeParams p, int n_splits, int n_chunks)
             const int ch = ks * 2 + ((lane >> 3) & 1);
             uint32_t b[4];
             ldmatrix_x4(b, sK + swz(row, ch));
-            mma_bf16(s0, qf[ks], b[0], b[1]);
-            mma_bf16(s1, qf[ks], b[2], b[3]);
+#pragma unroll
+            for (int im = 0; im < kMTiles; ++im) {
+                mma_bf16(s0[im], qf[im][ks], b[0], b[1]);
+                mma_bf16(s1[im], qf[im][ks], b[2], b[3]);
+            }
         }
         // ---- mask keys past the end, online softmax (rows lane/4 and lane/4+8) ----
         const int key = (tile_lo + t) * kTileKeys + krow0 + (lane & 3) * 2;
-        float v[8] = {s0[0], s0[1], s1[0], s1[1], s0[2], s0[3], s1[2], s1[3]};   // row0: v[0..3], row1: v[4..7]
         const bool ok[4] = {key < len, key + 1 < len, key + 8 < len, key + 9 < len};
+        uint32_t pf[kMTiles][4];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            v[i] = ok[i] ? v[i] * sl2 : -INFINITY;
-            v[i + 4] = ok[i] ? v[i + 4] * sl2 : -INFINITY;
+        for (int im = 0; im < kMTiles; ++im) {
+            float v[8] = {s0[im][0], s0[im][1], s1[im][0], s1[im][1], s0[im][2], s0[im][3], s1[im][2], s1[im][3]};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                v[i] = ok[i] ? v[i] * sl2 : -INFINITY;
+                v[i + 4] = ok[i] ? v[i + 4] * sl2 : -INFINITY;
+            }
+            float mx0 = fmaxf(fmaxf(v[0], v[1]), fmaxf(v[2], v[3])), mx1 = fmaxf(fmaxf(v[4], v[5]), fmaxf(v[6], v[7]));
+            mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1)); mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
+            mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1)); mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
+            // The exponent reference of a row moves only when its maximum grew by more than 2^8 (or is
+            // still unset); the accumulators are rescaled only then.  The final normalisation uses the
+            // same reference, so the result is exact up to rounding.
+            const bool g0 = mx0 > m0[im] + kRescaleThreshold, g1 = mx1 > m1[im] + kRescaleThreshold;
+            if (__any_sync(0xffffffffu, g0 || g1)) {
+                const float mn0 = g0 ? mx0 : m0[im], mn1 = g1 ? mx1 : m1[im];
+                const float a0 = g0 ? ex2(m0[im] - mn0) : 1.f, a1 = g1 ? ex2(m1[im] - mn1) : 1.f;
+                m0[im] = mn0; m1[im] = mn1;
+                l0[im] *= a0; l1[im] *= a1;
+#pragma unroll
+                for (int i = 0; i < 16; ++i) { acc[im][i][0] *= a0; acc[im][i][1] *= a0; acc[im][i][2] *= a1; acc[im][i][3] *= a1; }
+            }
+            const float ms0 = m0[im] == -INFINITY ? 0.f : m0[im], ms1 = m1[im] == -INFINITY ? 0.f : m1[im];
+            float ps0 = 0.f, ps1 = 0.f;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                v[i] = ex2(v[i] - ms0); ps0 += v[i];
+                v[i + 4] = ex2(v[i + 4] - ms1); ps1 += v[i + 4];
+            }
+            l0[im] += ps0; l1[im] += ps1;
+            // P as A operand (16 rows x 16 keys)
+            pf[im][0] = pack_bf16(v[0], v[1]); pf[im][1] = pack_bf16(v[4], v[5]);
+            pf[im][2] = pack_bf16(v[2], v[3]); pf[im][3] = pack_bf16(v[6], v[7]);
         }
-        float mx0 = fmaxf(fmaxf(v[0], v[1]), fmaxf(v[2], v[3])), mx1 = fmaxf(fmaxf(v[4], v[5]), fmaxf(v[6], v[7]));
-        mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1)); mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
-        mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1)); mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
-        const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);
-        const float ms0 = mn0 == -INFINITY ? 0.f : mn0, ms1 = mn1 == -INFINITY ? 0.f : mn1;
-        const float a0 = ex2(m0 - ms0), a1 = ex2(m1 - ms1);
-        m0 = mn0; m1 = mn1;
-        float ps0 = 0.f, ps1 = 0.f;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            v[i] = ex2(v[i] - ms0); ps0 += v[i];
-            v[i + 4] = ex2(v[i + 4] - ms1); ps1 += v[i + 4];
-        }
-        l0 = l0 * a0 + ps0; l1 = l1 * a1 + ps1;
-#pragma unroll
-        for (int i = 0; i < 16; ++i) { acc[i][0] *= a0; acc[i][1] *= a0; acc[i][2] *= a1; acc[i][3] *= a1; }
-        // P as A operand (16 rows x 16 keys)
-        uint32_t pf[4] = {pack_bf16(v[0], v[1]), pack_bf16(v[4], v[5]), pack_bf16(v[2], v[3]), pack_bf16(v[6], v[7])};
         // ---- O += P V ----
 #pragma unroll
         for (int nd = 0; nd < 8; ++nd) {
@@ -283,33 +315,38 @@ decode_split_kernel(const DecodeParams p, int n_splits, int n_chunks)
             const int ch = nd * 2 + (lane >> 4);
             uint32_t b[4];
             ldmatrix_x4_trans(b, sV + swz(row, ch));
-            mma_bf16(acc[2 * nd], pf, b[0], b[1]);
-            mma_bf16(acc[2 * nd + 1], pf, b[2], b[3]);
+#pragma unroll
+            for (int im = 0; im < kMTiles; ++im) {
+                mma_bf16(acc[im][2 * nd], pf[im], b[0], b[1]);
+                mma_bf16(acc[im][2 * nd + 1], pf[im], b[2], b[3]);
+            }
         }
     }
     cp_async_wait<0>();
     __syncthreads();
 
     // ---- merge the four key slices of each M-tile through shared memory ----
-    float *red = reinterpret_cast<float *>(smem);              // [warp][16 rows][kPartialStride]
-    {
+    float *red = reinterpret_cast<float *>(smem);              // [slice][M-tile][16 rows][kPartialStride]
+#pragma unroll
+    for (int im = 0; im < kMTiles; ++im) {
         // quad-reduce l (each lane of a quad summed different keys)
-        l0 += __shfl_xor_sync(0xffffffffu, l0, 1); l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
-        l1 += __shfl_xor_sync(0xffffffffu, l1, 1); l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
-        float *w0 = red + ((size_t)warp * 16 + (lane >> 2)) * kPartialStride;
+        float la = l0[im], lb = l1[im];
+        la += __shfl_xor_sync(0xffffffffu, la, 1); la += __shfl_xor_sync(0xffffffffu, la, 2);
+        lb += __shfl_xor_sync(0xffffffffu, lb, 1); lb += __shfl_xor_sync(0xffffffffu, lb, 2);
+        float *w0 = red + ((size_t)(slice * kMTiles + im) * 16 + (lane >> 2)) * kPartialStride;
         float *w1 = w0 + 8 * kPartialStride;
-        if ((lane & 3) == 0) { w0[0] = m0; w0[1] = l0; w1[0] = m1; w1[1] = l1; }
+        if ((lane & 3) == 0) { w0[0] = m0[im]; w0[1] = la; w1[0] = m1[im]; w1[1] = lb; }
 #pragma unroll
         for (int i = 0; i < 16; ++i) {
             const int c = i * 8 + (lane & 3) * 2;
-            w0[2 + c] = acc[i][0]; w0[2 + c + 1] = acc[i][1];
-            w1[2 + c] = acc[i][2]; w1[2 + c + 1] = acc[i][3];
+            w0[2 + c] = acc[im][i][0]; w0[2 + c + 1] = acc[im][i][1];
+            w1[2 + c] = acc[im][i][2]; w1[2 + c + 1] = acc[im][i][3];
         }
     }
     __syncthreads();
     // slices -> this CTA's partial (m, l, pad, pad, o[128]) per stacked row, kept in shared memory
     float *cta_part = reinterpret_cast<float *>(smem + kCtaPartOffset);   // [16 * kMTiles][kPartialStride]
-    for (int idx = tid; idx < 16 * kMTiles * kD; idx += 128 * kMTiles) {
+    for (int idx = tid; idx < 16 * kMTiles * kD; idx += 128) {
         const int c = idx % kD, rr = idx / kD;                 // rr: row within CTA (mt' * 16 + r)
         const int mtp = rr >> 4, r = rr & 15;
         float mm = -INFINITY;
@@ -342,7 +379,7 @@ decode_split_kernel(const DecodeParams p, int n_splits, int n_chunks)
         return (size_t)part * p.hq + head;
     };
     cluster.sync();                                             // every CTA's partial is in place
-    for (int i = tid; i < my_rows * (kD / 4); i += 128 * kMTiles) {
+    for (int i = tid; i < my_rows * (kD / 4); i += 128) {
         const int k = i / (kD / 4), c4 = i - k * (kD / 4);
         const int rr = rank + k * cs;
         float2 ml[kMaxCluster];
@@ -389,7 +426,7 @@ decode_split_kernel(const DecodeParams p, int n_splits, int n_chunks)
     __shared__ int s_flag;
     const int source = blockIdx.z * gridDim.y + kvh;
     if (!arrive_last(p.counters + source * kMaxCluster + rank, ncl, &s_flag)) return;
-    merge_slots<128 * kMTiles>(p, red, ncl, cache, kvh, row0 + rank, cs, my_rows);
+    merge_slots<128>(p, red, ncl, cache, kvh, row0 + rank, cs, my_rows);
 }
 
 size_t decode_scratch_bytes(int n_part, int hq, int d, int /*sm_count*/)
@@ -426,7 +463,7 @@ static cudaError_t launch_decode_split(const DecodeParams &p, int sm_count, int 
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof(cfg));
     cfg.gridDim = dim3(n_splits, p.hkv, caches * n_chunks);
-    cfg.blockDim = dim3(128 * m_tiles, 1, 1);
+    cfg.blockDim = dim3(128, 1, 1);
     cfg.dynamicSmemBytes = kStages * kStageBytes;              // 96 KB (also covers the merge buffers)
     cfg.stream = s;
     cudaLaunchAttribute attr;
