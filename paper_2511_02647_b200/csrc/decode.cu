@@ -25,7 +25,6 @@ constexpr int kTileKeys = 64;
 constexpr int kStages = 3;
 constexpr int kTileBytes = kTileKeys * kD * 2;          // 16 KB (K or V)
 constexpr int kStageBytes = 2 * kTileBytes;             // K + V
-constexpr int kMaxSplits = 64;
 constexpr int kPartialStride = kD + 4;                  // m, l, 2 pad, o[128]: o is 16-byte aligned
 constexpr float kRescaleThreshold = 8.0f;               // log2 units
 constexpr int kMaxCluster = 8;                          // CTAs per cluster (portable maximum)
@@ -79,56 +78,47 @@ __device__ __forceinline__ uint32_t swz(int row, int chunk) { return (uint32_t)(
 
 // Merges the n cluster results (slots 0 .. n-1, n <= kMaxSlots) of `rows` stacked query rows row0,
 // row0 + row_step, ... of one (cache, KV head), normalises and writes o / lse.  Called by every thread
-// of the CTA; `sm` holds rows * (n + 2) floats.
+// of the CTA.  Each thread owns 4 output columns of a row and reads every slot's (m, l) itself, so all
+// loads are issued at once and there is no barrier.
 template <int kThreads>
-__device__ __forceinline__ void merge_slots(const DecodeParams &p, float *sm, int n, int cache, int kvh, int row0,
-                                            int row_step, int rows)
+__device__ __forceinline__ void merge_slots(const DecodeParams &p, int n, int cache, int kvh, int row0, int row_step,
+                                            int rows)
 {
-    const int tid = threadIdx.x;
     const int g = p.hq / p.hkv;
-    auto out_row = [&](int srow) -> size_t {
+    for (int i = threadIdx.x; i < rows * (kD / 4); i += kThreads) {
+        const int rr = i / (kD / 4), c4 = i - rr * (kD / 4);
+        const int srow = row0 + rr * row_step;
         const int part = p.sync ? srow / g : cache;
         const int head = kvh * g + (p.sync ? srow % g : srow);
-        return (size_t)part * p.hq + head;
-    };
-    float *sc = sm, *big_m = sm + rows * n, *big_l = big_m + rows;          // sc[row][slot]
-    float2 *ml = reinterpret_cast<float2 *>(big_l + rows);                 // (m, l)[row][slot]
-    for (int i = tid; i < rows * n; i += kThreads) {
-        const int rr = i / n, k = i - rr * n;
-        ml[i] = __ldcg(reinterpret_cast<const float2 *>(p.partial + (out_row(row0 + rr * row_step) * n + k) * kPartialStride));
-    }
-    __syncthreads();
-    if (tid < rows) {
-        float mm = -INFINITY;
-        for (int k = 0; k < n; ++k) mm = fmaxf(mm, ml[tid * n + k].x);
-        const float ms = mm == -INFINITY ? 0.f : mm;
-        float ll = 0.f;
-        for (int k = 0; k < n; ++k) {
-            const float f = ex2(ml[tid * n + k].x - ms);
-            ll += ml[tid * n + k].y * f;
-            sc[tid * n + k] = f;
-        }
-        big_m[tid] = mm; big_l[tid] = ll;
-    }
-    __syncthreads();
-    for (int i = tid; i < rows * (kD / 4); i += kThreads) {
-        const int rr = i / (kD / 4), c4 = i - rr * (kD / 4);
-        const size_t orow = out_row(row0 + rr * row_step);
-        const float *src = p.partial + orow * n * kPartialStride + 4 + c4 * 4;
+        const size_t orow = (size_t)part * p.hq + head;
+        const float *src = p.partial + orow * n * kPartialStride;
+        float mm = -INFINITY, ll = 0.f;
         float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
         for (int k0 = 0; k0 < n; k0 += 4) {
+            float2 ml[4];
             float4 v[4];
 #pragma unroll
             for (int k = 0; k < 4; ++k)
-                if (k0 + k < n) v[k] = __ldcg(reinterpret_cast<const float4 *>(src + (size_t)(k0 + k) * kPartialStride));
+                if (k0 + k < n) {
+                    ml[k] = __ldcg(reinterpret_cast<const float2 *>(src + (size_t)(k0 + k) * kPartialStride));
+                    v[k] = __ldcg(reinterpret_cast<const float4 *>(src + (size_t)(k0 + k) * kPartialStride + 4 + c4 * 4));
+                }
+            float mn = mm;
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+                if (k0 + k < n) mn = fmaxf(mn, ml[k].x);
+            const float ms = mn == -INFINITY ? 0.f : mn;
+            const float f0 = ex2(mm - ms);                      // 0 on the first chunk (mm = -inf)
+            ll *= f0; a.x *= f0; a.y *= f0; a.z *= f0; a.w *= f0;
 #pragma unroll
             for (int k = 0; k < 4; ++k)
                 if (k0 + k < n) {
-                    const float f = sc[rr * n + k0 + k];
+                    const float f = ex2(ml[k].x - ms);
+                    ll += ml[k].y * f;
                     a.x += v[k].x * f; a.y += v[k].y * f; a.z += v[k].z * f; a.w += v[k].w * f;
                 }
+            mm = mn;
         }
-        const float ll = big_l[rr], mm = big_m[rr];
         const float inv = ll > 0.f ? 1.f / ll : 0.f;
         __nv_bfloat162 lo = __floats2bfloat162_rn(a.x * inv, a.y * inv), hi = __floats2bfloat162_rn(a.z * inv, a.w * inv);
         uint2 w;
@@ -154,6 +144,14 @@ __device__ __forceinline__ bool arrive_last(int32_t *ctr, int expected, int *s_f
     return last;
 }
 
+#ifdef FEDATTN_DTRACE
+// Debug build only: cycle stamps of the phases of every CTA's thread 0, [cta][event].
+__device__ long long g_dtrace[1024 * 8];
+#define DTRACE(e) do { if (threadIdx.x == 0) { const int b_ = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z); if (b_ < 1024) g_dtrace[b_ * 8 + (e)] = clock64(); } } while (0)
+#else
+#define DTRACE(e) do { } while (0)
+#endif
+
 // grid: x = split, y = KV head, z = cache * n_chunks + chunk   (cache = participant for LOCAL, 0 for SYNC)
 // block: 128 threads.  Warp w takes key slice w (16 keys of every 64-key tile) for all kMTiles
 // 16-row M-tiles of the chunk, so each K/V fragment is read from shared memory once.
@@ -164,6 +162,7 @@ decode_split_kernel(const DecodeParams p, int n_splits, int n_chunks)
     extern __shared__ __align__(1024) uint8_t smem[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int slice = warp;
+    DTRACE(0);
     const int split = blockIdx.x, kvh = blockIdx.y;
     const int cache = blockIdx.z / n_chunks, chunk = blockIdx.z - cache * n_chunks;
     const int g = p.hq / p.hkv;
@@ -189,22 +188,6 @@ decode_split_kernel(const DecodeParams p, int n_splits, int n_chunks)
         const int head = kvh * g + (p.sync ? srow % g : srow);
         return reinterpret_cast<const __nv_bfloat16 *>(p.q) + ((size_t)part * p.hq + head) * kD;
     };
-
-    // Q fragments (A operand, 16 x 128 per M-tile): 8 k-steps x 4 registers
-    uint32_t qf[kMTiles][8][4];
-#pragma unroll
-    for (int im = 0; im < kMTiles; ++im) {
-        const int row_base = (chunk * kMTiles + im) * 16;       // first stacked row of this M-tile
-        const __nv_bfloat16 *r0 = q_ptr(row_base + (lane >> 2)), *r1 = q_ptr(row_base + (lane >> 2) + 8);
-        const int c = (lane & 3) * 2;
-#pragma unroll
-        for (int ks = 0; ks < 8; ++ks) {
-            qf[im][ks][0] = r0 ? *reinterpret_cast<const uint32_t *>(r0 + ks * 16 + c) : 0u;
-            qf[im][ks][1] = r1 ? *reinterpret_cast<const uint32_t *>(r1 + ks * 16 + c) : 0u;
-            qf[im][ks][2] = r0 ? *reinterpret_cast<const uint32_t *>(r0 + ks * 16 + c + 8) : 0u;
-            qf[im][ks][3] = r1 ? *reinterpret_cast<const uint32_t *>(r1 + ks * 16 + c + 8) : 0u;
-        }
-    }
 
     // K and V tiles: 64 rows x 16 chunks of 16 bytes each.  Thread tid copies chunk (tid & 15) of rows
     // (tid >> 4) + 8 i, i = 0..7; the row's swizzle term (row & 7) is the same for all i, so the global
@@ -236,14 +219,44 @@ decode_split_kernel(const DecodeParams p, int n_splits, int n_chunks)
         for (int i = 0; i < 16; ++i) acc[im][i][0] = acc[im][i][1] = acc[im][i][2] = acc[im][i][3] = 0.f;
     }
 
+    // Q rows of this chunk -> shared memory (in the third stage's buffer, which the first tile loads do
+    // not touch), same swizzle as the K/V tiles; rows past rows_total are zero
+    {
+        const uint32_t sQ = smem_u32(smem) + (kStages - 1) * kStageBytes;
+#pragma unroll
+        for (int i = tid; i < 16 * kMTiles * 16; i += 128) {
+            const int row = i >> 4, ch = i & 15;
+            const __nv_bfloat16 *src = q_ptr(chunk * kMTiles * 16 + row);
+            cp_async16(sQ + swz(row, ch), src ? src + ch * 8 : reinterpret_cast<const __nv_bfloat16 *>(p.q), src != nullptr);
+        }
+        cp_async_commit();
+    }
 #pragma unroll
     for (int s = 0; s < kStages - 1; ++s) {
         if (s < n_tiles) load_tile(s, s);
         cp_async_commit();
     }
+    // Q fragments (A operand, 16 x 128 per M-tile): 8 k-steps x 4 registers
+    uint32_t qf[kMTiles][8][4];
+    cp_async_wait<kStages - 1>();                               // the Q group; the tile groups may still be in flight
+    __syncthreads();
+    {
+        const uint32_t sQ = smem_u32(smem) + (kStages - 1) * kStageBytes;
+#pragma unroll
+        for (int im = 0; im < kMTiles; ++im)
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) {
+                // matrices: (rows 0-7, d 0-7) (rows 8-15, d 0-7) (rows 0-7, d 8-15) (rows 8-15, d 8-15)
+                const int row = im * 16 + (lane & 7) + (((lane >> 3) & 1) << 3);
+                const int ch = ks * 2 + (lane >> 4);
+                ldmatrix_x4(qf[im][ks], sQ + swz(row, ch));
+            }
+    }
+    DTRACE(1);
     for (int t = 0; t < n_tiles; ++t) {
         cp_async_wait<kStages - 2>();
         __syncthreads();
+        if (t == 0) DTRACE(2);
         if (t + kStages - 1 < n_tiles) load_tile(t + kStages - 1, (t + kStages - 1) % kStages);
         cp_async_commit();
 
@@ -324,46 +337,62 @@ decode_split_kernel(const DecodeParams p, int n_splits, int n_chunks)
     }
     cp_async_wait<0>();
     __syncthreads();
+    DTRACE(3);
 
-    // ---- merge the four key slices of each M-tile through shared memory ----
-    float *red = reinterpret_cast<float *>(smem);              // [slice][M-tile][16 rows][kPartialStride]
+    // ---- merge the four key slices (warps) into this CTA's partial, kept in shared memory ----
+    // 1. every warp posts the exponent references of its rows; 2. every thread rescales its own
+    // accumulators to the common reference of its rows (in registers) and posts them; 3. the slices
+    // are summed with 16-byte reads.
+    float *red = reinterpret_cast<float *>(smem);               // [slice][16 kMTiles rows][kPartialStride]
+    float *sm_m = reinterpret_cast<float *>(smem + 68 * 1024);  // [slice][16 kMTiles rows]
+    float *sm_l = sm_m + 4 * 16 * kMTiles;
+    float *cta_part = reinterpret_cast<float *>(smem + kCtaPartOffset);   // [16 kMTiles rows][kPartialStride]
+    constexpr int kRows = 16 * kMTiles;
+    if ((lane & 3) == 0) {
+#pragma unroll
+        for (int im = 0; im < kMTiles; ++im) {
+            sm_m[slice * kRows + im * 16 + (lane >> 2)] = m0[im];
+            sm_m[slice * kRows + im * 16 + (lane >> 2) + 8] = m1[im];
+        }
+    }
+    __syncthreads();
 #pragma unroll
     for (int im = 0; im < kMTiles; ++im) {
+        const int ra = im * 16 + (lane >> 2), rb = ra + 8;
+        float ma = -INFINITY, mb = -INFINITY;
+#pragma unroll
+        for (int sl = 0; sl < 4; ++sl) { ma = fmaxf(ma, sm_m[sl * kRows + ra]); mb = fmaxf(mb, sm_m[sl * kRows + rb]); }
+        const float fa = ex2(m0[im] - (ma == -INFINITY ? 0.f : ma)), fb = ex2(m1[im] - (mb == -INFINITY ? 0.f : mb));
         // quad-reduce l (each lane of a quad summed different keys)
         float la = l0[im], lb = l1[im];
         la += __shfl_xor_sync(0xffffffffu, la, 1); la += __shfl_xor_sync(0xffffffffu, la, 2);
         lb += __shfl_xor_sync(0xffffffffu, lb, 1); lb += __shfl_xor_sync(0xffffffffu, lb, 2);
-        float *w0 = red + ((size_t)(slice * kMTiles + im) * 16 + (lane >> 2)) * kPartialStride;
+        if ((lane & 3) == 0) { sm_l[slice * kRows + ra] = la * fa; sm_l[slice * kRows + rb] = lb * fb; }
+        float *w0 = red + ((size_t)slice * kRows + ra) * kPartialStride + 4 + (lane & 3) * 2;
         float *w1 = w0 + 8 * kPartialStride;
-        if ((lane & 3) == 0) { w0[0] = m0[im]; w0[1] = la; w1[0] = m1[im]; w1[1] = lb; }
 #pragma unroll
         for (int i = 0; i < 16; ++i) {
-            const int c = i * 8 + (lane & 3) * 2;
-            w0[2 + c] = acc[im][i][0]; w0[2 + c + 1] = acc[im][i][1];
-            w1[2 + c] = acc[im][i][2]; w1[2 + c + 1] = acc[im][i][3];
+            *reinterpret_cast<float2 *>(w0 + i * 8) = make_float2(acc[im][i][0] * fa, acc[im][i][1] * fa);
+            *reinterpret_cast<float2 *>(w1 + i * 8) = make_float2(acc[im][i][2] * fb, acc[im][i][3] * fb);
         }
     }
     __syncthreads();
-    // slices -> this CTA's partial (m, l, pad, pad, o[128]) per stacked row, kept in shared memory
-    float *cta_part = reinterpret_cast<float *>(smem + kCtaPartOffset);   // [16 * kMTiles][kPartialStride]
-    for (int idx = tid; idx < 16 * kMTiles * kD; idx += 128) {
-        const int c = idx % kD, rr = idx / kD;                 // rr: row within CTA (mt' * 16 + r)
-        const int mtp = rr >> 4, r = rr & 15;
-        float mm = -INFINITY;
+    for (int i = tid; i < kRows * (kD / 4); i += 128) {
+        const int rr = i / (kD / 4), c4 = i - rr * (kD / 4);
+        float4 a = *reinterpret_cast<const float4 *>(red + (size_t)rr * kPartialStride + 4 + c4 * 4);
 #pragma unroll
-        for (int sl = 0; sl < 4; ++sl) mm = fmaxf(mm, red[((size_t)(sl * kMTiles + mtp) * 16 + r) * kPartialStride]);
-        const float ms = mm == -INFINITY ? 0.f : mm;
-        float ll = 0.f, oo = 0.f;
-#pragma unroll
-        for (int sl = 0; sl < 4; ++sl) {
-            const float *w = red + ((size_t)(sl * kMTiles + mtp) * 16 + r) * kPartialStride;
-            const float sc = ex2(w[0] - ms);
-            ll += w[1] * sc;
-            oo += w[2 + c] * sc;
+        for (int sl = 1; sl < 4; ++sl) {
+            const float4 v = *reinterpret_cast<const float4 *>(red + ((size_t)sl * kRows + rr) * kPartialStride + 4 + c4 * 4);
+            a.x += v.x; a.y += v.y; a.z += v.z; a.w += v.w;
         }
         float *dst = cta_part + rr * kPartialStride;
-        dst[4 + c] = oo;
-        if (c == 0) { dst[0] = mm; dst[1] = ll; }
+        *reinterpret_cast<float4 *>(dst + 4 + c4 * 4) = a;
+        if (c4 == 0) {
+            float mm = -INFINITY, ll = 0.f;
+#pragma unroll
+            for (int sl = 0; sl < 4; ++sl) { mm = fmaxf(mm, sm_m[sl * kRows + rr]); ll += sm_l[sl * kRows + rr]; }
+            dst[0] = mm; dst[1] = ll;
+        }
     }
 
     // ---- cluster merge through distributed shared memory: rank k takes rows k, k + cs, ... ----
@@ -378,6 +407,7 @@ decode_split_kernel(const DecodeParams p, int n_splits, int n_chunks)
         const int head = kvh * g + (p.sync ? srow % g : srow);
         return (size_t)part * p.hq + head;
     };
+    DTRACE(4);
     cluster.sync();                                             // every CTA's partial is in place
     for (int i = tid; i < my_rows * (kD / 4); i += 128) {
         const int k = i / (kD / 4), c4 = i - k * (kD / 4);
@@ -420,14 +450,25 @@ decode_split_kernel(const DecodeParams p, int n_splits, int n_chunks)
         }
     }
     cluster.sync();                                             // peers are done reading this CTA's partial
+    DTRACE(5);
     if (ncl == 1 || my_rows == 0) return;
 
     // ---- several clusters per (cache, KV head): the last to arrive for these rows merges them ----
     __shared__ int s_flag;
     const int source = blockIdx.z * gridDim.y + kvh;
-    if (!arrive_last(p.counters + source * kMaxCluster + rank, ncl, &s_flag)) return;
-    merge_slots<128>(p, red, ncl, cache, kvh, row0 + rank, cs, my_rows);
+    const bool last = arrive_last(p.counters + source * kMaxCluster + rank, ncl, &s_flag);
+    DTRACE(6);
+    if (!last) return;
+    merge_slots<128>(p, ncl, cache, kvh, row0 + rank, cs, my_rows);
+    DTRACE(7);
 }
+
+#ifdef FEDATTN_DTRACE
+extern "C" int fedattn_debug_read_dtrace(long long *host, int n)
+{
+    return (int)cudaMemcpyFromSymbol(host, g_dtrace, sizeof(long long) * n);
+}
+#endif
 
 size_t decode_scratch_bytes(int n_part, int hq, int d, int /*sm_count*/)
 {
