@@ -83,6 +83,9 @@ cudaError_t launch_concat(const PartsParams &pp, int hkv, int d, int elt_bytes, 
 // One thread per (token, KV head): s = sum_c x_c^2 accumulated in fp64 in increasing c.  Each
 // square of a bf16/fp32 value is exact in fp64, so only the summation order matters and it is
 // fixed here.  Output index: Hkv * off[n] + h * L_n + j.
+// s + x^2 for the two bf16 values packed in w, low half first; each square is exact in fp64.
+// (Squaring in fp32 and widening the result by integer bit moves avoids the slow fp32->fp64
+// conversion but was measured slower: the extra integer and range-check instructions cost more.)
 __device__ __forceinline__ double sq_acc_bf16x2(double s, uint32_t w)
 {
     const double lo = (double)__uint_as_float(w << 16);
@@ -92,163 +95,307 @@ __device__ __forceinline__ double sq_acc_bf16x2(double s, uint32_t w)
     return s;
 }
 
+// A warp takes chunks of 32 consecutive (token, head) rows.  The rows of a chunk are contiguous in
+// memory (within a participant), so the warp copies them with coalesced 16-byte cp.async into its
+// own shared-memory buffer, each row padded by 16 bytes; lane r then walks row r with conflict-free
+// 16-byte reads.  (Reading the rows straight from global memory, one thread per 256-byte row, is
+// limited by the load unit: every warp-wide load touches 32 different sectors.)  Chunks are dealt
+// round-robin over all warps of a persistent grid, so every SM gets the same share and the warps
+// of an SM are in different phases: one warp's loads overlap another's fp64 chain.
+constexpr int kScoreWarps = 4;            // warps per CTA
+
 template <int kDtype>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(32 * kScoreWarps)
 knorm_score_kernel(const PartsParams pp, int hkv, int d, double *scores)
 {
-    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    extern __shared__ __align__(16) uint8_t score_smem[];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int row_bytes = d * (kDtype == FEDATTN_BF16 ? 2 : 4), stride = row_bytes + 16, vpr = row_bytes / 16;
+    uint8_t *buf = score_smem + warp * 32 * stride;
+    const uint32_t sbase = (uint32_t)__cvta_generic_to_shared(buf);
     const int64_t total = (int64_t)pp.off[pp.n] * hkv;
-    if (t >= total) return;
-    const int32_t row = (int32_t)(t / hkv);
-    const int h = (int)(t % hkv);
-    const int n = find_segment(pp.off, pp.n, row);
-    const int32_t j = row - pp.off[n];
-    const int32_t len = pp.off[n + 1] - pp.off[n];
-    double s = 0.0;
-    if (kDtype == FEDATTN_BF16) {
-        const uint4 *src = reinterpret_cast<const uint4 *>(
-            reinterpret_cast<const __nv_bfloat16 *>(pp.k[n]) + ((int64_t)j * hkv + h) * d);
-        for (int c = 0; c < d / 8; ++c) {
-            const uint4 w = __ldg(src + c);
-            s = sq_acc_bf16x2(s, w.x);
-            s = sq_acc_bf16x2(s, w.y);
-            s = sq_acc_bf16x2(s, w.z);
-            s = sq_acc_bf16x2(s, w.w);
+    const int64_t n_chunks = (total + 31) / 32;
+    const int64_t n_warps = (int64_t)gridDim.x * kScoreWarps;
+    for (int64_t c = blockIdx.x + (int64_t)gridDim.x * warp; c < n_chunks; c += n_warps) {
+        const int64_t g = c * 32 + lane;                              // this lane's row
+        int n = 0, h = 0;
+        int32_t j = 0, len = 0;
+        const uint8_t *my_src = nullptr;
+        if (g < total) {
+            const int32_t row = (int32_t)(g / hkv);
+            h = (int)(g % hkv);
+            n = find_segment(pp.off, pp.n, row);
+            j = row - pp.off[n];
+            len = pp.off[n + 1] - pp.off[n];
+            my_src = reinterpret_cast<const uint8_t *>(pp.k[n]) + ((int64_t)j * hkv + h) * row_bytes;
         }
-    } else {
-        const float4 *src = reinterpret_cast<const float4 *>(
-            reinterpret_cast<const float *>(pp.k[n]) + ((int64_t)j * hkv + h) * d);
-        for (int c = 0; c < d / 4; ++c) {
-            const float4 w = __ldg(src + c);
-            s = __dadd_rn(s, __dmul_rn((double)w.x, (double)w.x));
-            s = __dadd_rn(s, __dmul_rn((double)w.y, (double)w.y));
-            s = __dadd_rn(s, __dmul_rn((double)w.z, (double)w.z));
-            s = __dadd_rn(s, __dmul_rn((double)w.w, (double)w.w));
+        __syncwarp();                                                 // the previous chunk's reads are done
+        for (int q = lane; q < 32 * vpr; q += 32) {
+            const int r = q / vpr, ch = q - r * vpr;
+            const uint8_t *src = reinterpret_cast<const uint8_t *>(__shfl_sync(0xffffffffu, (unsigned long long)my_src, r));
+            if (src)
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(sbase + r * stride + ch * 16), "l"(src + ch * 16) : "memory");
         }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+        __syncwarp();
+        if (g >= total) continue;
+        double s = 0.0;
+        const uint4 *mine = reinterpret_cast<const uint4 *>(buf + lane * stride);
+        if (kDtype == FEDATTN_BF16) {
+            for (int v = 0; v < vpr; ++v) {
+                const uint4 w = mine[v];
+                s = sq_acc_bf16x2(s, w.x);
+                s = sq_acc_bf16x2(s, w.y);
+                s = sq_acc_bf16x2(s, w.z);
+                s = sq_acc_bf16x2(s, w.w);
+            }
+        } else {
+            for (int v = 0; v < vpr; ++v) {
+                const uint4 u = mine[v];
+                const float x0 = __uint_as_float(u.x), x1 = __uint_as_float(u.y), x2 = __uint_as_float(u.z), x3 = __uint_as_float(u.w);
+                s = __dadd_rn(s, __dmul_rn((double)x0, (double)x0));
+                s = __dadd_rn(s, __dmul_rn((double)x1, (double)x1));
+                s = __dadd_rn(s, __dmul_rn((double)x2, (double)x2));
+                s = __dadd_rn(s, __dmul_rn((double)x3, (double)x3));
+            }
+        }
+        scores[(int64_t)hkv * pp.off[n] + (int64_t)h * len + j] = s;
     }
-    scores[(int64_t)hkv * pp.off[n] + (int64_t)h * len + j] = s;
 }
 
-cudaError_t launch_knorm_scores(const PartsParams &pp, int hkv, int d, int dtype, double *scores,
+cudaError_t launch_knorm_scores(const PartsParams &pp, int hkv, int d, int dtype, double *scores, int sm_count,
                                 cudaStream_t s, int64_t *launches)
 {
     const int64_t total = (int64_t)pp.off[pp.n] * hkv;
     if (total == 0) return cudaSuccess;
-    const unsigned blocks = (unsigned)((total + 255) / 256);
+    const int smem = kScoreWarps * 32 * (d * (dtype == FEDATTN_BF16 ? 2 : 4) + 16);
+    static bool attr_set = false;
+    if (!attr_set) {                                            // 128 rows x 528 bytes for fp32, head_dim 128
+        cudaError_t e = cudaFuncSetAttribute(knorm_score_kernel<FEDATTN_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             kScoreWarps * 32 * (FEDATTN_MAX_HEAD_DIM * 4 + 16));
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    const int64_t chunks = (total + 31) / 32;
+    int64_t blocks = (int64_t)sm_count * (200 * 1024 / smem);   // as many CTAs as fit, by shared memory
+    if (blocks > (chunks + kScoreWarps - 1) / kScoreWarps) blocks = (chunks + kScoreWarps - 1) / kScoreWarps;
     if (dtype == FEDATTN_BF16)
-        knorm_score_kernel<FEDATTN_BF16><<<blocks, 256, 0, s>>>(pp, hkv, d, scores);
+        knorm_score_kernel<FEDATTN_BF16><<<(unsigned)blocks, 32 * kScoreWarps, smem, s>>>(pp, hkv, d, scores);
     else
-        knorm_score_kernel<FEDATTN_F32><<<blocks, 256, 0, s>>>(pp, hkv, d, scores);
+        knorm_score_kernel<FEDATTN_F32><<<(unsigned)blocks, 32 * kScoreWarps, smem, s>>>(pp, hkv, d, scores);
     ++*launches;
     return cudaGetLastError();
 }
 
-// ---- top-k selection ---------------------------------------------------------------------------
-// One CTA per (KV head, participant).  Scores are non-negative doubles, so their bit patterns
-// order like unsigned integers.  An 8-bit-per-pass radix select finds the k-th largest score
-// tau and how many rows equal to tau are still needed; an ordered compaction then emits, in
-// ascending index order, every row with score > tau plus the lowest-index rows with score == tau.
+// ---- top-k selection + gather ---------------------------------------------------------------------
+// grid (KV head, participant, slice).  Scores are non-negative doubles, so their bit patterns order
+// like unsigned integers.  Every CTA of a (head, participant) runs the same selection: an
+// 8-bit-per-pass radix select finds the k-th largest score tau and how many rows equal to tau are
+// still needed; one ordered compaction then gives every kept row its output position (rows with
+// score > tau, plus the lowest-index rows with score == tau, in ascending index order).  CTA
+// `slice` then copies its share of the kept K/V rows into the head-major output and writes their
+// indices and global positions.  Redoing the cheap selection per slice spreads the copy over the
+// whole GPU without a second launch.
 constexpr int kSelThreads = 256;
 constexpr int kSelMaxLen = 4096;
 
-__device__ __forceinline__ int block_excl_scan_flag(bool flag, int *warp_tot, int &block_total)
-{
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const unsigned bal = __ballot_sync(0xffffffffu, flag);
-    const int in_warp = __popc(bal & ((1u << lane) - 1u));
-    if (lane == 0) warp_tot[warp] = __popc(bal);
-    __syncthreads();
-    int base = 0, tot = 0;
-#pragma unroll
-    for (int w = 0; w < kSelThreads / 32; ++w) {
-        const int c = warp_tot[w];
-        if (w < warp) base += c;
-        tot += c;
-    }
-    __syncthreads();
-    block_total = tot;
-    return base + in_warp;
-}
-
 __global__ void __launch_bounds__(kSelThreads)
-topk_select_kernel(const PartsParams pp, int hkv, const double *scores, int32_t *sel_idx)
+topk_select_gather_kernel(const PartsParams pp, int hkv, int vpr /* 16-byte vectors per (row, head) */,
+                          const double *scores, uint4 *k_agg, uint4 *v_agg, int32_t *kv_pos, int32_t *cu_kv,
+                          int32_t *sel_idx_out)
 {
     __shared__ unsigned long long keys[kSelMaxLen];
     __shared__ int hist[256];
     __shared__ int warp_tot[kSelThreads / 32];
-    __shared__ int sh_bin, sh_krem;
+    __shared__ int sh_bin, sh_krem, sh_count;
+    __shared__ unsigned long long sh_tau;
+    __shared__ unsigned long long warp_or[kSelThreads / 32], warp_and[kSelThreads / 32];
+    __shared__ uint16_t my_rows[kSelMaxLen];                  // kept indices of this CTA's slice (< 4096)
 
-    const int h = blockIdx.x, n = blockIdx.y;
+    const int h = blockIdx.x, n = blockIdx.y, slice = blockIdx.z, n_slices = gridDim.z;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (h == 0 && n == 0 && slice == 0 && cu_kv && tid <= pp.n) cu_kv[tid] = pp.cu_kv[tid];
     const int len = pp.off[n + 1] - pp.off[n];
     const int k = pp.cu_kv[n + 1] - pp.cu_kv[n];
     if (k == 0 || len == 0) return;
     const int64_t T = pp.cu_kv[pp.n];
     const double *sc = scores + (int64_t)hkv * pp.off[n] + (int64_t)h * len;
-    for (int j = threadIdx.x; j < len; j += kSelThreads)
-        keys[j] = (unsigned long long)__double_as_longlong(sc[j]);
+    // Bits that all keys share need no pass: (OR of all keys) ^ (AND of all keys) has a 1 exactly where
+    // two keys differ.
+    unsigned long long k_or = 0, k_and = ~0ULL;
+    for (int j = tid; j < len; j += kSelThreads) {
+        const unsigned long long key = (unsigned long long)__double_as_longlong(__ldcg(sc + j));
+        keys[j] = key;
+        k_or |= key; k_and &= key;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        k_or |= __shfl_xor_sync(0xffffffffu, k_or, o);
+        k_and &= __shfl_xor_sync(0xffffffffu, k_and, o);
+    }
+    if (lane == 0) { warp_or[warp] = k_or; warp_and[warp] = k_and; }
+    __syncthreads();
+    k_or = 0; k_and = ~0ULL;
+#pragma unroll
+    for (int w = 0; w < kSelThreads / 32; ++w) { k_or |= warp_or[w]; k_and &= warp_and[w]; }
+    const unsigned long long diff = k_or ^ k_and, key0 = k_and;     // key0: the shared bits
+
+    unsigned long long tau = key0;           // k-th largest score; k_rem rows equal to tau are kept
+    int k_rem = k;
+    if (diff != 0) {
+        // first pass: the 8 bits that end at the highest differing bit, over all keys; the keys that fall
+        // into the chosen bin are listed (my_rows doubles as the list) and later passes walk only the list
+        int shift = max(63 - __clzll((long long)diff) - 7, 0);
+        const unsigned long long above = shift + 8 >= 64 ? 0ULL : ~((1ULL << (shift + 8)) - 1ULL);
+        unsigned long long prefix = key0 & above, mask = above;
+        int n_cand = len;
+        bool listed = false;
+        for (;;) {
+            const int nb = listed ? min(8, shift) : 8;
+            if (listed) shift -= nb;
+            hist[tid] = 0;
+            if (tid == 0) sh_count = 0;
+            __syncthreads();
+            for (int i = tid; i < n_cand; i += kSelThreads) {
+                const unsigned long long key = keys[listed ? my_rows[i] : i];
+                if ((key & mask) == prefix) atomicAdd(&hist[(int)((key >> shift) & ((1u << nb) - 1u))], 1);
+            }
+            __syncthreads();
+            // suffix sums over bins: S[b] = sum_{b' >= b} hist[b']
+            const int mine = hist[tid];
+            int incl = mine;   // inclusive suffix within warp: sum over lanes >= lane
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int up = __shfl_down_sync(0xffffffffu, incl, o);
+                if (lane + o < 32) incl += up;
+            }
+            if (lane == 0) warp_tot[warp] = incl;
+            __syncthreads();
+            int above_w = 0;
+#pragma unroll
+            for (int w = 0; w < kSelThreads / 32; ++w)
+                if (w > warp) above_w += warp_tot[w];
+            const int S_b = incl + above_w;     // count of candidates with these bits >= tid
+            const int S_next = S_b - mine;      // count with these bits > tid
+            if (S_b >= k_rem && S_next < k_rem) {
+                sh_bin = tid;
+                sh_krem = k_rem - S_next;
+            }
+            __syncthreads();
+            prefix |= (unsigned long long)sh_bin << shift;
+            mask |= (unsigned long long)((1u << nb) - 1u) << shift;
+            k_rem = sh_krem;
+            if (shift == 0) break;
+            if (!listed) {
+                // list the keys of the chosen bin (order is irrelevant): one counter bump per warp
+                for (int j0 = 0; j0 < len; j0 += kSelThreads) {
+                    const int j = j0 + tid;
+                    const bool in = j < len && (keys[j] & mask) == prefix;
+                    const unsigned bal = __ballot_sync(0xffffffffu, in);
+                    int base = 0;
+                    if (lane == 0 && bal) base = atomicAdd(&sh_count, __popc(bal));
+                    base = __shfl_sync(0xffffffffu, base, 0);
+                    if (in) my_rows[base + __popc(bal & ((1u << lane) - 1u))] = (uint16_t)j;
+                }
+                __syncthreads();
+                n_cand = sh_count;
+                listed = true;
+                if (n_cand <= kSelThreads) {
+                    // Short list: thread i ranks candidate i against all others (broadcast reads, no more
+                    // passes).  tau is the value v with #(> v) < k_rem <= #(>= v).
+                    if (tid < n_cand) {
+                        const unsigned long long mine_key = keys[my_rows[tid]];
+                        int gt = 0, ge = 0;
+                        for (int i = 0; i < n_cand; ++i) {
+                            const unsigned long long other = keys[my_rows[i]];
+                            gt += other > mine_key;
+                            ge += other >= mine_key;
+                        }
+                        if (gt < k_rem && k_rem <= ge) { sh_tau = mine_key; sh_krem = k_rem - gt; }   // equal keys agree
+                    }
+                    __syncthreads();
+                    prefix = sh_tau;
+                    k_rem = sh_krem;
+                    break;
+                }
+            }
+        }
+        tau = prefix;
+    }
+    __syncthreads();                                          // the list in my_rows is dead from here on
+
+    // ordered compaction: thread tid owns indices [tid * per, (tid + 1) * per)
+    const int per = (len + kSelThreads - 1) / kSelThreads;
+    const int j_lo = min(tid * per, len), j_hi = min(j_lo + per, len);
+    int n_gt = 0, n_eq = 0;
+    for (int j = j_lo; j < j_hi; ++j) {
+        const unsigned long long key = keys[j];
+        n_gt += key > tau;
+        n_eq += key == tau;
+    }
+    // exclusive block scan of (n_gt, n_eq), packed 16 + 16 bits (both <= 4096)
+    unsigned packed = ((unsigned)n_gt << 16) | (unsigned)n_eq, incl = packed;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const unsigned up = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += up;
+    }
+    __syncthreads();                                          // warp_tot is free again
+    if (lane == 31) warp_tot[warp] = (int)incl;
+    __syncthreads();
+    unsigned base = 0;
+#pragma unroll
+    for (int w = 0; w < kSelThreads / 32; ++w)
+        if (w < warp) base += (unsigned)warp_tot[w];
+    const unsigned excl = base + incl - packed;
+    int gt_before = (int)(excl >> 16), eq_before = (int)(excl & 0xffffu);
+    // this CTA's share of the k outputs
+    const int per_slice = (k + n_slices - 1) / n_slices;
+    const int o_lo = min(slice * per_slice, k), o_hi = min(o_lo + per_slice, k);
+    for (int j = j_lo; j < j_hi; ++j) {
+        const unsigned long long key = keys[j];
+        const bool gt = key > tau, eq = key == tau;
+        if (gt || (eq && eq_before < k_rem)) {
+            const int pos = gt_before + min(eq_before, k_rem);
+            if (pos >= o_lo && pos < o_hi) my_rows[pos - o_lo] = (uint16_t)j;
+        }
+        gt_before += gt;
+        eq_before += eq;
+    }
     __syncthreads();
 
-    unsigned long long prefix = 0, mask = 0;
-    int k_rem = k;
-    for (int shift = 56; shift >= 0; shift -= 8) {
-        hist[threadIdx.x] = 0;
-        __syncthreads();
-        for (int j = threadIdx.x; j < len; j += kSelThreads) {
-            const unsigned long long key = keys[j];
-            if ((key & mask) == prefix) atomicAdd(&hist[(int)((key >> shift) & 0xff)], 1);
-        }
-        __syncthreads();
-        // suffix sums over bins: S[b] = sum_{b' >= b} hist[b']
-        const int b = threadIdx.x;
-        const int mine = hist[b];
-        const int lane = b & 31, warp = b >> 5;
-        int incl = mine;   // inclusive suffix within warp: sum over lanes >= lane
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const int up = __shfl_down_sync(0xffffffffu, incl, o);
-            if (lane + o < 32) incl += up;
-        }
-        if (lane == 0) warp_tot[warp] = incl;
-        __syncthreads();
-        int above = 0;
-#pragma unroll
-        for (int w = 0; w < kSelThreads / 32; ++w)
-            if (w > warp) above += warp_tot[w];
-        const int S_b = incl + above;       // count of candidates with byte >= b
-        const int S_next = S_b - mine;      // count with byte > b
-        if (S_b >= k_rem && S_next < k_rem) {
-            sh_bin = b;
-            sh_krem = k_rem - S_next;
-        }
-        __syncthreads();
-        prefix |= (unsigned long long)sh_bin << shift;
-        mask |= 0xffULL << shift;
-        k_rem = sh_krem;
-        __syncthreads();
+    // gather this slice: rows my_rows[0 .. o_hi - o_lo) of participant n, head h
+    const int n_out = o_hi - o_lo;
+    const int64_t out_row0 = (int64_t)h * T + pp.cu_kv[n] + o_lo;
+    const uint4 *ksrc = reinterpret_cast<const uint4 *>(pp.k[n]), *vsrc = reinterpret_cast<const uint4 *>(pp.v[n]);
+    for (int i = tid; i < n_out * vpr; i += kSelThreads) {
+        const int r = i / vpr, vi = i - r * vpr;
+        const int64_t src = ((int64_t)my_rows[r] * hkv + h) * vpr + vi;
+        const int64_t dst = (out_row0 + r) * vpr + vi;
+        const uint4 kk = ld_stream(ksrc + src), vv = ld_stream(vsrc + src);
+        k_agg[dst] = kk;
+        v_agg[dst] = vv;
     }
-    const unsigned long long tau = prefix;   // k-th largest score; k_rem rows equal to tau are kept
-
-    int eq_base = 0, out_base = 0;
-    int32_t *dst = sel_idx + (int64_t)h * T + pp.cu_kv[n];
-    for (int j0 = 0; j0 < len; j0 += kSelThreads) {
-        const int j = j0 + threadIdx.x;
-        const unsigned long long key = j < len ? keys[j] : 0ULL;
-        const bool is_eq = j < len && key == tau;
-        int eq_tot, sel_tot;
-        const int eq_rank = eq_base + block_excl_scan_flag(is_eq, warp_tot, eq_tot);
-        const bool sel = j < len && (key > tau || (is_eq && eq_rank < k_rem));
-        const int pos = out_base + block_excl_scan_flag(sel, warp_tot, sel_tot);
-        if (sel) dst[pos] = j;
-        eq_base += eq_tot;
-        out_base += sel_tot;
+    for (int r = tid; r < n_out; r += kSelThreads) {
+        if (kv_pos) kv_pos[out_row0 + r] = pp.off[n] + my_rows[r];
+        if (sel_idx_out) sel_idx_out[out_row0 + r] = my_rows[r];
     }
 }
 
-cudaError_t launch_topk_select(const PartsParams &pp, int hkv, const double *scores, int32_t *sel_idx,
-                               cudaStream_t s, int64_t *launches)
+cudaError_t launch_topk_select_gather(const PartsParams &pp, int hkv, int d, int elt_bytes, const double *scores,
+                                      void *k_agg, void *v_agg, int32_t *kv_pos, int32_t *cu_kv,
+                                      int32_t *sel_idx_out, int sm_count, cudaStream_t s, int64_t *launches)
 {
-    if (pp.cu_kv[pp.n] == 0) return cudaSuccess;
-    topk_select_kernel<<<dim3(hkv, pp.n), kSelThreads, 0, s>>>(pp, hkv, scores, sel_idx);
+    if (pp.cu_kv[pp.n] == 0) {
+        if (!cu_kv) return cudaSuccess;
+    }
+    const int pairs = hkv * pp.n;
+    int slices = (4 * sm_count + pairs - 1) / pairs;          // about four CTAs per SM in total
+    if (slices < 1) slices = 1;
+    if (slices > 64) slices = 64;
+    topk_select_gather_kernel<<<dim3(hkv, pp.n, slices), kSelThreads, 0, s>>>(
+        pp, hkv, d * elt_bytes / 16, scores, (uint4 *)k_agg, (uint4 *)v_agg, kv_pos, cu_kv, sel_idx_out);
     ++*launches;
     return cudaGetLastError();
 }

@@ -225,19 +225,16 @@ fedattn_status fedattn_aggregate_kv(fedattn_ctx *ctx, const fedattn_shape *shape
         err = launch_concat(pp, hkv, d, eb, k_agg, v_agg, kv_pos, cu_kv, s, ctx->c.sm_count, &ctx->c.launches);
         return err == cudaSuccess ? FEDATTN_OK : FEDATTN_ERR_CUDA;
     }
-    const int32_t *sel = sel_idx_in;
     if (mode == FEDATTN_AGG_TOPK_KNORM) {
         if (ctx->c.scratch_bytes < topk_scratch_bytes(hkv, L)) return FEDATTN_ERR_WORKSPACE;
         double *scores = reinterpret_cast<double *>(ctx->c.scratch);
-        int32_t *sel_buf = sel_idx_out
-                               ? sel_idx_out
-                               : reinterpret_cast<int32_t *>(ctx->c.scratch +
-                                                             align_up((size_t)hkv * L * sizeof(double), 256));
-        err = launch_knorm_scores(pp, hkv, d, shape->dtype, scores, s, &ctx->c.launches);
-        if (err == cudaSuccess) err = launch_topk_select(pp, hkv, scores, sel_buf, s, &ctx->c.launches);
-        if (err != cudaSuccess) return FEDATTN_ERR_CUDA;
-        sel = sel_buf;
+        err = launch_knorm_scores(pp, hkv, d, shape->dtype, scores, ctx->c.sm_count, s, &ctx->c.launches);
+        if (err == cudaSuccess)
+            err = launch_topk_select_gather(pp, hkv, d, eb, scores, k_agg, v_agg, kv_pos, cu_kv, sel_idx_out,
+                                            ctx->c.sm_count, s, &ctx->c.launches);
+        return err == cudaSuccess ? FEDATTN_OK : FEDATTN_ERR_CUDA;
     }
+    const int32_t *sel = sel_idx_in;
     err = launch_gather(pp, hkv, d, eb, sel, k_agg, v_agg, kv_pos, cu_kv, sel_idx_out, ctx->c.status, s,
                         &ctx->c.launches);
     return err == cudaSuccess ? FEDATTN_OK : FEDATTN_ERR_CUDA;
