@@ -18,6 +18,15 @@ flop per query head, divided by the step time, inputs resident in HBM).  `e2e` i
 through the same calls with pinned HOST inputs and outputs (copies inside the timed region).
 `roofline` covers the dominant kernel (the tcgen05 prefill kernel); `calls` gives every call's
 own time and rate.  `--impl reference` times the fp64 CPU oracle on a bounded row sample.
+
+`--workload` selects one of the other seeded configurations, each printing one line of the same
+form with its own metric:
+    cfg3   32-block schedules over 8 heterogeneous segments, sync every H-th block, H in
+           {1,2,4,8,32}: time per H (value: prefill TFLOP/s of the H=1 schedule)
+    cfg4   sparse aggregation (16 x 1024, top 256 keys per KV head) + sync over the selected KV
+           (value: aggregation GB/s, HBM roofline)
+    cfg5   decode, 8 caches x 4096 tokens, a step = 3 local + 1 sync call (H=4)
+           (value: decode GB/s, HBM roofline)
 With --gpus N > 1 every rank runs an independent replica (the path has no exchange step on one
 device; participants are simulated per GPU) and the value is the sum over ranks.
 """
@@ -46,6 +55,9 @@ SPARSE_RATIO_NUM, SPARSE_RATIO_DEN = 1, 4
 # dram__bytes_read.sum + dram__bytes_write.sum per prefill launch of the sync call at this
 # workload, from the ncu capture summarised under profiles/ (None until captured)
 PREFILL_SYNC_DRAM_BYTES = None
+# the same for one decode call (cfg5) and for one sparse aggregation (cfg4: both launches)
+DECODE_DRAM_BYTES = None
+TOPK_DRAM_BYTES = None
 
 
 def env_rank():
@@ -345,6 +357,268 @@ def run_ours(args):
 
 
 # ------------------------------------------------------------------------------------------------
+# the other configurations (one process, one GPU; same timing rules)
+# ------------------------------------------------------------------------------------------------
+def _setup(local_rank=0):
+    import torch
+    import paper_2511_02647_b200 as fa
+    torch.cuda.set_device(local_rank)
+    return torch, fa, torch.device("cuda", local_rank)
+
+
+def _timed(torch, stream, fn, iters, warmup, sampler=None):
+    """Runs fn(i) warmup + iters times; returns ms per iteration (CUDA events on the launching stream)."""
+    for i in range(warmup):
+        fn(i)
+    torch.cuda.synchronize()
+    e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for i in range(iters):
+        fn(i)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / iters
+
+
+def _line(args, metric, unit, value, ms_per_step, dtype, config, clocks, e2e, launches, roofline, calls, extra=None):
+    out = {"metric": metric, "value": round(value, 3), "unit": unit, "n_gpus": 1, "steps": args.steps,
+           "warmup": max(args.warmup, 3), "ms_per_step": round(ms_per_step, 5), "higher_is_better": True,
+           "scaling": "weak", "vs_baseline": None, "dtype": dtype, "data": "synthetic", "config": config,
+           "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "calls": calls}
+    if extra:
+        out.update(extra)
+    print(json.dumps(out), flush=True)
+
+
+def run_cfg5(args):
+    """Decode: N=8 caches x 4096 tokens; a step = 3 local calls + 1 sync call (sync every H=4)."""
+    torch, fa, dev = _setup()
+    w = fi.cfg5()
+    N, Hq, Hkv, d, L = w.n_participants, w.n_q_heads, w.n_kv_heads, w.head_dim, w.total_tokens
+    seqlens = list(w.seqlens)
+    cu = [0] + list(np.cumsum(seqlens))
+    shape = fa.Shape(N, Hq, Hkv, d, fa.BF16)
+    ctx = fa.Context(shape, L, L)
+    bf = torch.bfloat16
+    n_sets = max(2, args.sets)
+    stream = torch.cuda.current_stream()
+    caches = []
+    for s_ in range(n_sets):
+        _, k, v = w.qkv(block=s_)
+        tk, tv = (torch.from_numpy(x).to(bf).to(dev) for x in (k, v))
+        kg, vg = torch.empty_like(tk), torch.empty_like(tv)
+        kp = [tk[cu[n]:cu[n + 1]] for n in range(N)]; vp = [tv[cu[n]:cu[n + 1]] for n in range(N)]
+        fa.fedattn_aggregate_kv(ctx, shape, fa.AGG_CONCAT, kp, vp, seqlens, None, None, kg, vg, None, None, None)
+        caches.append((tk, tv, kg, vg))
+    hq = [torch.from_numpy(w.decode_q(i)).to(bf).pin_memory() for i in range(8)]
+    qs = [x.to(dev) for x in hq]
+    o = torch.empty_like(qs[0])
+    ho = torch.empty((N, Hq, d), dtype=bf).pin_memory()
+    len_local = torch.tensor(seqlens, dtype=torch.int32, device=dev)
+    len_sync = torch.tensor([L], dtype=torch.int32, device=dev)
+    stride = seqlens[0] * Hkv * d
+
+    def call(i, sync):
+        c = caches[i % n_sets]
+        if sync:
+            fa.fedattn_decode(ctx, shape, fa.DECODE_SYNC, qs[i % 8], c[2], c[3], 0, len_sync, L, o)
+        else:
+            fa.fedattn_decode(ctx, shape, fa.DECODE_LOCAL, qs[i % 8], c[0], c[1], stride, len_local, max(seqlens), o)
+
+    def step(i):                                         # decode steps 4i+1 .. 4i+4: the 4th is a sync step
+        for j in range(4):
+            call(4 * i + j, fi.is_sync_block(j + 1, 4))
+
+    K, W = args.steps, max(args.warmup, 3)
+    sampler = ClockSampler(0); sampler.start(); time.sleep(0.25)
+    ms_local = _timed(torch, stream, lambda i: call(i, False), 4 * K, W)
+    ms_sync = _timed(torch, stream, lambda i: call(i, True), 4 * K, W)
+    l0 = ctx.launch_count()
+    ms_step = _timed(torch, stream, step, K, W)
+    launches = (ctx.launch_count() - l0) * K // (K + W)
+    time.sleep(0.25); clocks = sampler.stop()
+    assert ctx.poll() == 0
+
+    def e2e_step(i):
+        qs[i % 8].copy_(hq[i % 8], non_blocking=True)
+        step(i)
+        ho.copy_(o, non_blocking=True)
+    ms_e2e = _timed(torch, stream, e2e_step, max(3, min(K, 10)), 1)
+
+    kv_bytes = 2 * L * Hkv * d * 2 + 2 * N * Hq * d * 2        # per call: every K/V row once + q + o
+    pk = peaks()
+    gbs = lambda ms: kv_bytes / (ms * 1e-3) / 1e9
+    value = 4 * kv_bytes / (ms_step * 1e-3) / 1e9
+    calls = {"decode_local": {"ms": round(ms_local, 5), "gbs": round(gbs(ms_local), 1), "frac_hbm": round(gbs(ms_local) / pk["hbm"], 4)},
+             "decode_sync": {"ms": round(ms_sync, 5), "gbs": round(gbs(ms_sync), 1), "frac_hbm": round(gbs(ms_sync) / pk["hbm"], 4)}}
+    roof = {"bound": "hbm", "kernel": "decode_split_kernel (one launch per decode call)", "achieved": round(value, 1),
+            "peak": pk["hbm"], "unit": "GB/s", "frac": round(value / pk["hbm"], 4), "peak_kind": "copy, " + pk["kind"],
+            "traffic": DECODE_DRAM_BYTES}
+    _line(args, "fedattn_decode_gbs", "GB/s", value, ms_step, "bf16",
+          {"workload": w.name, "participants": N, "cache_tokens": seqlens[0], "q_heads": Hq, "kv_heads": Hkv, "head_dim": d,
+           "step": "3 x decode_local + 1 x decode_sync (sync every 4th decode step)",
+           "l2": "%d rotating cache sets of %d MB (K+V, > 126 MB L2 each)" % (n_sets, 2 * L * Hkv * d * 2 // 2 ** 20),
+           "parallelism": "single"},
+          clocks, {"value": round(4 * kv_bytes / (ms_e2e * 1e-3) / 1e9, 1), "unit": "GB/s",
+                   "h2d_bytes_per_step": hq[0].numel() * 2, "d2h_bytes_per_step": ho.numel() * 2, "ms_per_step": round(ms_e2e, 4)},
+          launches, roof, calls)
+
+
+def run_cfg4(args):
+    """Sparse aggregation (top 256 of 1024 keys per participant and KV head) + sync over the selected KV."""
+    torch, fa, dev = _setup()
+    w = fi.cfg4()
+    N, Hq, Hkv, d, L = w.n_participants, w.n_q_heads, w.n_kv_heads, w.head_dim, w.total_tokens
+    seqlens = list(w.seqlens)
+    cu = [0] + list(np.cumsum(seqlens))
+    ksel = [w.k_sel] * N
+    T = sum(ksel)
+    shape = fa.Shape(N, Hq, Hkv, d, fa.BF16)
+    ctx = fa.Context(shape, L, L)
+    bf = torch.bfloat16
+    n_sets = max(3, args.sets)
+    stream = torch.cuda.current_stream()
+    host, sets = [], []
+    for s_ in range(n_sets):
+        q, k, v = w.qkv(block=s_)
+        hs = [torch.from_numpy(x).to(bf).pin_memory() for x in (q, k, v)]
+        host.append(hs)
+        tq, tk, tv = (x.to(dev) for x in hs)
+        sets.append(dict(q=tq, k=tk, v=tv, kp=[tk[cu[n]:cu[n + 1]] for n in range(N)], vp=[tv[cu[n]:cu[n + 1]] for n in range(N)],
+                         k_sp=torch.empty((Hkv, T, d), dtype=bf, device=dev), v_sp=torch.empty((Hkv, T, d), dtype=bf, device=dev),
+                         pos=torch.empty((Hkv, T), dtype=torch.int32, device=dev), sel=torch.empty((Hkv, T), dtype=torch.int32, device=dev),
+                         o=torch.empty_like(tq)))
+    ho = torch.empty((L, Hq, d), dtype=bf).pin_memory()
+
+    def agg(i):
+        b = sets[i % n_sets]
+        fa.fedattn_aggregate_kv(ctx, shape, fa.AGG_TOPK_KNORM, b["kp"], b["vp"], seqlens, ksel, None, b["k_sp"], b["v_sp"],
+                                b["pos"], None, b["sel"])
+
+    def sync(i):
+        b = sets[i % n_sets]
+        fa.fedattn_sync(ctx, shape, b["q"], None, b["k_sp"], b["v_sp"], b["pos"], T, True, b["o"])
+
+    def step(i):
+        agg(i); sync(i)
+
+    K, W = args.steps, max(args.warmup, 3)
+    step(0)
+    pos = sets[0]["pos"].to(torch.int64)
+    rows = torch.arange(L, device=dev, dtype=torch.int64)
+    pairs = sum(int(torch.searchsorted(pos[h].contiguous(), rows, right=True).sum().item()) for h in range(Hkv))
+    f_sync = 4.0 * d * (Hq // Hkv) * pairs
+    sampler = ClockSampler(0); sampler.start(); time.sleep(0.25)
+    ms_agg = _timed(torch, stream, agg, K, W)
+    ms_sync = _timed(torch, stream, sync, K, W)
+    l0 = ctx.launch_count()
+    ms_step = _timed(torch, stream, step, K, W)
+    launches = (ctx.launch_count() - l0) * K // (K + W)
+    time.sleep(0.25); clocks = sampler.stop()
+    assert ctx.poll() == 0
+
+    def e2e_step(i):
+        b, hs = sets[i % n_sets], host[i % n_sets]
+        b["q"].copy_(hs[0], non_blocking=True); b["k"].copy_(hs[1], non_blocking=True); b["v"].copy_(hs[2], non_blocking=True)
+        step(i)
+        ho.copy_(b["o"], non_blocking=True)
+    ms_e2e = _timed(torch, stream, e2e_step, max(3, min(K, 10)), 1)
+
+    kv_bytes = 2 * L * Hkv * d * 2
+    agg_bytes = kv_bytes // 2 + (kv_bytes // 2) * T // L + kv_bytes * T // L     # K once + selected V + selected K,V written
+    pk = peaks()
+    gbs = agg_bytes / (ms_agg * 1e-3) / 1e9
+    tf = f_sync / (ms_sync * 1e-3) / 1e12
+    roof = {"bound": "hbm", "kernel": "knorm_score_kernel + topk_select_gather_kernel (the two launches of one sparse aggregation)",
+            "achieved": round(gbs, 1), "peak": pk["hbm"], "unit": "GB/s", "frac": round(gbs / pk["hbm"], 4),
+            "peak_kind": "copy, " + pk["kind"], "traffic": TOPK_DRAM_BYTES}
+    calls = {"aggregate_topk": {"ms": round(ms_agg, 5), "gbs": round(gbs, 1), "frac_hbm": round(gbs / pk["hbm"], 4)},
+             "sync_sparse": {"ms": round(ms_sync, 5), "tflops": round(tf, 2), "frac_tensor": round(tf / pk["tensor"], 4)}}
+    _line(args, "fedattn_aggregate_gbs", "GB/s", gbs, ms_step, "bf16",
+          {"workload": w.name, "participants": N, "tokens_per_participant": seqlens[0], "q_heads": Hq, "kv_heads": Hkv,
+           "head_dim": d, "keep_per_kv_head": w.k_sel, "step": "aggregate_topk + sync over the selected KV",
+           "l2": "%d rotating input/output sets (> 126 MB L2 in total)" % n_sets, "parallelism": "single"},
+          clocks, {"value": round(agg_bytes / (ms_e2e * 1e-3) / 1e9, 1), "unit": "GB/s",
+                   "h2d_bytes_per_step": sum(x.numel() * 2 for x in host[0]), "d2h_bytes_per_step": ho.numel() * 2,
+                   "ms_per_step": round(ms_e2e, 4)},
+          launches, roof, calls)
+
+
+def run_cfg3(args):
+    """32-block schedules over 8 heterogeneous segments: block m is a sync block iff m mod H == 0."""
+    torch, fa, dev = _setup()
+    w = fi.cfg3()
+    N, Hq, Hkv, d, L = w.n_participants, w.n_q_heads, w.n_kv_heads, w.head_dim, w.total_tokens
+    seqlens = list(w.seqlens)
+    cu = [0] + list(np.cumsum(seqlens))
+    shape = fa.Shape(N, Hq, Hkv, d, fa.BF16)
+    ctx = fa.Context(shape, L, L)
+    bf = torch.bfloat16
+    n_sets = max(3, args.sets)
+    stream = torch.cuda.current_stream()
+    host, sets = [], []
+    for s_ in range(n_sets):
+        q, k, v = w.qkv(block=s_)
+        hs = [torch.from_numpy(x).to(bf).pin_memory() for x in (q, k, v)]
+        host.append(hs)
+        tq, tk, tv = (x.to(dev) for x in hs)
+        sets.append(dict(q=tq, k=tk, v=tv, kp=[tk[cu[n]:cu[n + 1]] for n in range(N)], vp=[tv[cu[n]:cu[n + 1]] for n in range(N)],
+                         kg=torch.empty_like(tk), vg=torch.empty_like(tv), o=torch.empty_like(tq)))
+    ho = torch.empty((L, Hq, d), dtype=bf).pin_memory()
+    M = w.n_blocks
+
+    def block(m, H):
+        b = sets[m % n_sets]
+        if fi.is_sync_block(m, H):
+            fa.fedattn_aggregate_kv(ctx, shape, fa.AGG_CONCAT, b["kp"], b["vp"], seqlens, None, None, b["kg"], b["vg"], None, None, None)
+            fa.fedattn_sync(ctx, shape, b["q"], None, b["kg"], b["vg"], None, L, False, b["o"])
+        else:
+            fa.fedattn_local(ctx, shape, b["q"], b["k"], b["v"], cu, b["o"])
+
+    f_local = 4.0 * d * Hq * sum(n * (n + 1) // 2 for n in seqlens)
+    f_sync = 4.0 * d * Hq * (L * (L + 1) // 2)
+    K, W = max(1, args.steps // 4), 1
+    sampler = ClockSampler(0); sampler.start(); time.sleep(0.25)
+    per_h = {}
+    for blk in range(1, 4):
+        block(blk, 1); block(blk, M + 1)                     # warm-up of both paths
+    l0 = ctx.launch_count()
+    for H in (1, 2, 4, 8, 32):
+        ms = _timed(torch, stream, lambda i, H=H: [block(m, H) for m in range(1, M + 1)], K, W)
+        n_sync = sum(1 for m in range(1, M + 1) if fi.is_sync_block(m, H))
+        fl = n_sync * f_sync + (M - n_sync) * f_local
+        per_h[str(H)] = {"ms": round(ms, 4), "sync_blocks": n_sync, "ms_per_block": round(ms / M, 4),
+                         "tflops": round(fl / (ms * 1e-3) / 1e12, 2)}
+    launches = (ctx.launch_count() - l0) * K // (K + W)
+    time.sleep(0.25); clocks = sampler.stop()
+    assert ctx.poll() == 0
+
+    def e2e_step(i):                                           # one sync block through host buffers
+        b, hs = sets[i % n_sets], host[i % n_sets]
+        b["q"].copy_(hs[0], non_blocking=True); b["k"].copy_(hs[1], non_blocking=True); b["v"].copy_(hs[2], non_blocking=True)
+        block(1, 1)
+        ho.copy_(b["o"], non_blocking=True)
+    ms_e2e = _timed(torch, stream, e2e_step, 3, 1)
+
+    pk = peaks()
+    value = per_h["1"]["tflops"]
+    roof = {"bound": "tensor", "kernel": "prefill_sm100_kernel (32 sync blocks of the H=1 schedule)", "achieved": value,
+            "peak": pk["tensor"], "unit": "TFLOP/s", "frac": round(value / pk["tensor"], 4),
+            "peak_kind": "burst bf16, " + pk["kind"],
+            "frac_of_sustained": round(value / pk["tensor_sustained"], 4) if pk["tensor_sustained"] else None, "traffic": None}
+    _line(args, METRIC, UNIT, value, per_h["1"]["ms"], "bf16",
+          {"workload": w.name, "participants": N, "segment_lengths": seqlens, "q_heads": Hq, "kv_heads": Hkv, "head_dim": d,
+           "blocks": M, "step": "the H=1 schedule: 32 x (concat + sync); `schedules` lists every H",
+           "l2": "%d rotating seeded blocks of inputs stand in for the 32 fresh ones (> 126 MB L2 each)" % n_sets,
+           "parallelism": "single"},
+          clocks, {"value": round(f_sync / (ms_e2e * 1e-3) / 1e12, 2), "unit": UNIT,
+                   "h2d_bytes_per_step": sum(x.numel() * 2 for x in host[0]), "d2h_bytes_per_step": ho.numel() * 2,
+                   "ms_per_step": round(ms_e2e, 4)},
+          launches, roof, {"local_block_tflop": round(f_local / 1e12, 4), "sync_block_tflop": round(f_sync / 1e12, 4)},
+          extra={"schedules": per_h})
+
+
+# ------------------------------------------------------------------------------------------------
 # CPU oracle legs
 # ------------------------------------------------------------------------------------------------
 def oracle_sample(w, q, k, v, n_rows, seed):
@@ -413,13 +687,16 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--workload", default="cfg2", choices=["cfg2", "cfg3", "cfg4", "cfg5"])
     ap.add_argument("--sets", type=int, default=N_SETS,
                     help="rotating input sets (1 keeps device memory small for a profiler capture)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
-    else:
+    elif args.workload == "cfg2":
         run_ours(args)
+    else:
+        {"cfg3": run_cfg3, "cfg4": run_cfg4, "cfg5": run_cfg5}[args.workload](args)
 
 
 if __name__ == "__main__":
