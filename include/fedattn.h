@@ -181,10 +181,12 @@ fedattn_status fedattn_decode(fedattn_ctx *ctx, const fedattn_shape *shape, int3
  * returns FEDATTN_ERR_UNSUPPORTED).  The built-in scratch covers n_participants * n_q_heads <= 256
  * output rows; a larger shape is rejected with FEDATTN_ERR_WORKSPACE and nothing is launched.
  * It runs on the CURRENT device.  The first call on each device resolves the array's device
- * address and sets kernel attributes; make that first call outside any stream capture.  Nothing
- * in the scratch needs to start at zero (every slot that is read is written earlier in the same
- * call), and its contents after a call are unspecified.  All calls on one device share the one
- * array: two calls that may overlap on the GPU (different streams, no ordering) race on it. */
+ * address and sets kernel attributes; make that first call outside any stream capture.  The
+ * partial slots need not start at zero (every slot that is read is written earlier in the same
+ * call) and their contents after a call are unspecified.  The few arrival counters beside them
+ * must be zero when a call starts: they are zero when the library is loaded and every completed
+ * call leaves them at zero.  All calls on one device share these arrays: two calls that may
+ * overlap on the GPU (different streams, no ordering) race on them. */
 fedattn_status fedattn_decode_noalloc(const fedattn_shape *shape, int32_t mode,
                                       const void *q, const void *k_cache, const void *v_cache,
                                       int64_t cache_stride_participant, const int32_t *kv_len,

@@ -2,21 +2,28 @@
 // online softmax in fp32.  Serves fedattn_local (per-participant causal attention over packed
 // segments) and fedattn_sync (queries over the aggregated KV, causal on global positions).
 //
-// One CTA owns one 128-row query tile of one query head and walks the key/value tiles that its
-// rows may see; tiles the segment descriptors or the causal mask rule out are never loaded.
-// Two CTAs are resident per SM (96 KB shared memory and 256 TMEM columns each), so one CTA's
-// softmax overlaps the other's MMAs.
+// Persistent kernel, one CTA per SM.  A work item is one 128-row query tile of a PAIR of query heads
+// that share a KV head (two "sub-tiles"); the CTA walks the key/value tiles the rows may see, and
+// tiles that the segment descriptors or the causal mask rule out are never loaded.  Items are sorted
+// by cost and dealt to the CTAs in snake order.
 //
-// Per KV tile j:   S = Q K_j^T            (tcgen05.mma, A/B from shared memory, D in TMEM)
-//                  P = exp2(S*c - m)      (128 softmax threads, one query row each, TMEM->regs)
-//                  O += P V_j             (tcgen05.mma, A = P from TMEM, B = V from shared memory)
-// O stays in TMEM for the whole tile walk and is rescaled only when a row's running maximum
-// grows by more than 2^8 (the final normalisation uses the same reference maximum, so the
-// result is exact up to rounding).
+// Per KV tile j and sub-tile t:
+//     S_t = Q_t K_j^T          (tcgen05.mma, A/B from shared memory, D in TMEM)
+//     P_t = exp2(S_t*c - m)    (softmax threads, TMEM -> registers -> TMEM, P aliases S)
+//     O_t += P_t V_j           (tcgen05.mma, A = P from TMEM, B = V from shared memory)
+// The tensor pipe alternates between the sub-tiles (PV_0 S_0 | PV_1 S_1 | ...), the softmax threads
+// serve them alternately as well, so while the softmax of one sub-tile runs the tensor pipe works
+// for the other.  O stays in TMEM for the whole tile walk and is rescaled only when a row's running
+// maximum grows by more than 2^8 (the final normalisation uses the same reference, so the result
+// is exact up to rounding).
 //
-// Warp roles: warps 0-3 softmax/epilogue (TMEM lane = query row), warp 4 TMA producer (+ TMEM
-// allocation), warp 5 MMA issuer.  Every wait is bounded; on expiry the CTA sets the status word,
-// stops waiting and runs to its normal end (TMEM is always released).
+// Warp roles: warps 0-7 softmax/epilogue.  Both warpgroups work on the same S tile, split by
+// columns: thread = (query row = TMEM lane, column half); the halves of a row exchange their
+// maxima through shared memory once per tile.  Warp 8 TMA producer (+ TMEM allocation), warp 9
+// MMA issuer (the whole warp walks the loop, one elected lane issues).  3/8 of the exponentials
+// of unmasked tiles are evaluated by a polynomial on the FMA pipe, because for this tile shape the
+// ex2 unit is exactly as slow as the tensor pipe.  Every wait is bounded; on expiry the CTA sets
+// the status word, stops waiting and runs to its normal end (TMEM is always released).
 #include <cuda.h>
 
 #include <stdio.h>
