@@ -2,6 +2,9 @@
 // selection, and the indexed gather that builds the head-major sparse KV.  All are pure data
 // movement or integer/compare work except the score, which is an fp64 chain in fixed order so
 // that the selected set is bit-identical to a sequential fp64 evaluation.
+#include <cooperative_groups.h>
+#include <string.h>
+
 #include "common.cuh"
 
 namespace fedattn {
@@ -95,116 +98,35 @@ __device__ __forceinline__ double sq_acc_bf16x2(double s, uint32_t w)
     return s;
 }
 
-// A warp takes chunks of 32 consecutive (token, head) rows.  The rows of a chunk are contiguous in
-// memory (within a participant), so the warp copies them with coalesced 16-byte cp.async into its
-// own shared-memory buffer, each row padded by 16 bytes; lane r then walks row r with conflict-free
-// 16-byte reads.  (Reading the rows straight from global memory, one thread per 256-byte row, is
-// limited by the load unit: every warp-wide load touches 32 different sectors.)  Chunks are dealt
-// round-robin over all warps of a persistent grid, so every SM gets the same share and the warps
-// of an SM are in different phases: one warp's loads overlap another's fp64 chain.
-constexpr int kScoreWarps = 4;            // warps per CTA
-
-template <int kDtype>
-__global__ void __launch_bounds__(32 * kScoreWarps)
-knorm_score_kernel(const PartsParams pp, int hkv, int d, double *scores)
-{
-    extern __shared__ __align__(16) uint8_t score_smem[];
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int row_bytes = d * (kDtype == FEDATTN_BF16 ? 2 : 4), stride = row_bytes + 16, vpr = row_bytes / 16;
-    uint8_t *buf = score_smem + warp * 32 * stride;
-    const uint32_t sbase = (uint32_t)__cvta_generic_to_shared(buf);
-    const int64_t total = (int64_t)pp.off[pp.n] * hkv;
-    const int64_t n_chunks = (total + 31) / 32;
-    const int64_t n_warps = (int64_t)gridDim.x * kScoreWarps;
-    for (int64_t c = blockIdx.x + (int64_t)gridDim.x * warp; c < n_chunks; c += n_warps) {
-        const int64_t g = c * 32 + lane;                              // this lane's row
-        int n = 0, h = 0;
-        int32_t j = 0, len = 0;
-        const uint8_t *my_src = nullptr;
-        if (g < total) {
-            const int32_t row = (int32_t)(g / hkv);
-            h = (int)(g % hkv);
-            n = find_segment(pp.off, pp.n, row);
-            j = row - pp.off[n];
-            len = pp.off[n + 1] - pp.off[n];
-            my_src = reinterpret_cast<const uint8_t *>(pp.k[n]) + ((int64_t)j * hkv + h) * row_bytes;
-        }
-        __syncwarp();                                                 // the previous chunk's reads are done
-        for (int q = lane; q < 32 * vpr; q += 32) {
-            const int r = q / vpr, ch = q - r * vpr;
-            const uint8_t *src = reinterpret_cast<const uint8_t *>(__shfl_sync(0xffffffffu, (unsigned long long)my_src, r));
-            if (src)
-                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(sbase + r * stride + ch * 16), "l"(src + ch * 16) : "memory");
-        }
-        asm volatile("cp.async.commit_group;" ::: "memory");
-        asm volatile("cp.async.wait_group 0;" ::: "memory");
-        __syncwarp();
-        if (g >= total) continue;
-        double s = 0.0;
-        const uint4 *mine = reinterpret_cast<const uint4 *>(buf + lane * stride);
-        if (kDtype == FEDATTN_BF16) {
-            for (int v = 0; v < vpr; ++v) {
-                const uint4 w = mine[v];
-                s = sq_acc_bf16x2(s, w.x);
-                s = sq_acc_bf16x2(s, w.y);
-                s = sq_acc_bf16x2(s, w.z);
-                s = sq_acc_bf16x2(s, w.w);
-            }
-        } else {
-            for (int v = 0; v < vpr; ++v) {
-                const uint4 u = mine[v];
-                const float x0 = __uint_as_float(u.x), x1 = __uint_as_float(u.y), x2 = __uint_as_float(u.z), x3 = __uint_as_float(u.w);
-                s = __dadd_rn(s, __dmul_rn((double)x0, (double)x0));
-                s = __dadd_rn(s, __dmul_rn((double)x1, (double)x1));
-                s = __dadd_rn(s, __dmul_rn((double)x2, (double)x2));
-                s = __dadd_rn(s, __dmul_rn((double)x3, (double)x3));
-            }
-        }
-        scores[(int64_t)hkv * pp.off[n] + (int64_t)h * len + j] = s;
-    }
-}
-
-cudaError_t launch_knorm_scores(const PartsParams &pp, int hkv, int d, int dtype, double *scores, int sm_count,
-                                cudaStream_t s, int64_t *launches)
-{
-    const int64_t total = (int64_t)pp.off[pp.n] * hkv;
-    if (total == 0) return cudaSuccess;
-    const int smem = kScoreWarps * 32 * (d * (dtype == FEDATTN_BF16 ? 2 : 4) + 16);
-    static bool attr_set = false;
-    if (!attr_set) {                                            // 128 rows x 528 bytes for fp32, head_dim 128
-        cudaError_t e = cudaFuncSetAttribute(knorm_score_kernel<FEDATTN_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             kScoreWarps * 32 * (FEDATTN_MAX_HEAD_DIM * 4 + 16));
-        if (e != cudaSuccess) return e;
-        attr_set = true;
-    }
-    const int64_t chunks = (total + 31) / 32;
-    int64_t blocks = (int64_t)sm_count * (200 * 1024 / smem);   // as many CTAs as fit, by shared memory
-    if (blocks > (chunks + kScoreWarps - 1) / kScoreWarps) blocks = (chunks + kScoreWarps - 1) / kScoreWarps;
-    if (dtype == FEDATTN_BF16)
-        knorm_score_kernel<FEDATTN_BF16><<<(unsigned)blocks, 32 * kScoreWarps, smem, s>>>(pp, hkv, d, scores);
-    else
-        knorm_score_kernel<FEDATTN_F32><<<(unsigned)blocks, 32 * kScoreWarps, smem, s>>>(pp, hkv, d, scores);
-    ++*launches;
-    return cudaGetLastError();
-}
-
-// ---- top-k selection + gather ---------------------------------------------------------------------
-// grid (KV head, participant, slice).  Scores are non-negative doubles, so their bit patterns order
-// like unsigned integers.  Every CTA of a (head, participant) runs the same selection: an
-// 8-bit-per-pass radix select finds the k-th largest score tau and how many rows equal to tau are
-// still needed; one ordered compaction then gives every kept row its output position (rows with
-// score > tau, plus the lowest-index rows with score == tau, in ascending index order).  CTA
-// `slice` then copies its share of the kept K/V rows into the head-major output and writes their
-// indices and global positions.  Redoing the cheap selection per slice spreads the copy over the
-// whole GPU without a second launch.
+// ---- top-k scores + selection + gather, one launch ----------------------------------------------
+// grid (KV head, participant, slice); the slices of one (head, participant) form a thread-block
+// cluster.
+//  1. Scores.  Slice r takes a contiguous share of the participant's tokens.  It copies their K rows
+//     of this head (row_bytes each, strided by the token pitch) into shared memory with 16-byte
+//     cp.async, each row padded by 16 bytes, and thread i walks row i: s = sum_c x_c^2 accumulated in
+//     fp64 in increasing c.  Each square of a bf16/fp32 value is exact in fp64, so only the order
+//     matters and it is fixed.  Scores are non-negative doubles, so their bit patterns order like
+//     unsigned integers; they are kept as such keys in shared memory.
+//  2. Every slice collects the other slices' keys through distributed shared memory.
+//  3. Selection, repeated by every slice: an 8-bit-per-pass radix select, started at the highest bit
+//     in which two keys differ, finds the k-th largest score tau and how many rows equal to tau are
+//     still needed; the keys of the first chosen bin are listed and, when the list is short, ranked
+//     by counting instead of further passes.  One ordered compaction then gives every kept row its
+//     output position (rows with score > tau, plus the lowest-index rows with score == tau, in
+//     ascending index order).
+//  4. Slice r copies its share of the kept K/V rows into the head-major output and writes their
+//     indices and global positions.
 constexpr int kSelThreads = 256;
 constexpr int kSelMaxLen = 4096;
+constexpr int kStageRows = 128;            // K rows staged per pass and buffer
+constexpr int kMaxSlices = 8;              // portable cluster size
 
+template <int kDtype>
 __global__ void __launch_bounds__(kSelThreads)
-topk_select_gather_kernel(const PartsParams pp, int hkv, int vpr /* 16-byte vectors per (row, head) */,
-                          const double *scores, uint4 *k_agg, uint4 *v_agg, int32_t *kv_pos, int32_t *cu_kv,
-                          int32_t *sel_idx_out)
+topk_fused_kernel(const PartsParams pp, int hkv, int vpr /* 16-byte vectors per (row, head) */,
+                  uint4 *k_agg, uint4 *v_agg, int32_t *kv_pos, int32_t *cu_kv, int32_t *sel_idx_out)
 {
+    extern __shared__ __align__(16) uint8_t stage[];           // [2][kStageRows][row_bytes + 16]
     __shared__ unsigned long long keys[kSelMaxLen];
     __shared__ int hist[256];
     __shared__ int warp_tot[kSelThreads / 32];
@@ -213,20 +135,88 @@ topk_select_gather_kernel(const PartsParams pp, int hkv, int vpr /* 16-byte vect
     __shared__ unsigned long long warp_or[kSelThreads / 32], warp_and[kSelThreads / 32];
     __shared__ uint16_t my_rows[kSelMaxLen];                  // kept indices of this CTA's slice (< 4096)
 
+    namespace cg = cooperative_groups;
+    cg::cluster_group cluster = cg::this_cluster();
     const int h = blockIdx.x, n = blockIdx.y, slice = blockIdx.z, n_slices = gridDim.z;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     if (h == 0 && n == 0 && slice == 0 && cu_kv && tid <= pp.n) cu_kv[tid] = pp.cu_kv[tid];
     const int len = pp.off[n + 1] - pp.off[n];
     const int k = pp.cu_kv[n + 1] - pp.cu_kv[n];
-    if (k == 0 || len == 0) return;
+    if (k == 0 || len == 0) return;                           // the same for every slice of the cluster
     const int64_t T = pp.cu_kv[pp.n];
-    const double *sc = scores + (int64_t)hkv * pp.off[n] + (int64_t)h * len;
+
+    // ---- 1. scores of this slice's tokens ----
+    {
+        const int row_bytes = vpr * 16, stride = row_bytes + 16;
+        const int per = (len + n_slices - 1) / n_slices;
+        const int r0 = min(slice * per, len), r1 = min(r0 + per, len);
+        const uint8_t *src = reinterpret_cast<const uint8_t *>(pp.k[n]) + (size_t)h * row_bytes;
+        const size_t pitch = (size_t)hkv * row_bytes;          // bytes between consecutive tokens
+        const uint32_t sbase = (uint32_t)__cvta_generic_to_shared(stage);
+        // two buffers of kStageRows rows: the copy of the next pass is in flight during the chains of this one
+        auto copy_pass = [&](int c0, int buf) {
+            const int rows = min(kStageRows, r1 - c0);
+            for (int q = tid; q < rows * vpr; q += kSelThreads) {
+                const int r = q / vpr, ch = q - r * vpr;
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(sbase + (buf * kStageRows + r) * stride + ch * 16),
+                             "l"(src + (size_t)(c0 + r) * pitch + ch * 16) : "memory");
+            }
+            asm volatile("cp.async.commit_group;" ::: "memory");
+        };
+        if (r0 < r1) copy_pass(r0, 0);
+        int buf = 0;
+        for (int c0 = r0; c0 < r1; c0 += kStageRows, buf ^= 1) {
+            const int rows = min(kStageRows, r1 - c0);
+            if (c0 + kStageRows < r1) {
+                copy_pass(c0 + kStageRows, buf ^ 1);           // that buffer's chains ended before the last barrier
+                asm volatile("cp.async.wait_group 1;" ::: "memory");
+            } else {
+                asm volatile("cp.async.wait_group 0;" ::: "memory");
+            }
+            __syncthreads();
+            if (tid < rows) {
+                const uint4 *mine = reinterpret_cast<const uint4 *>(stage + (size_t)(buf * kStageRows + tid) * stride);
+                double sc = 0.0;
+                if (kDtype == FEDATTN_BF16) {
+                    for (int v = 0; v < vpr; ++v) {
+                        const uint4 w = mine[v];
+                        sc = sq_acc_bf16x2(sc, w.x);
+                        sc = sq_acc_bf16x2(sc, w.y);
+                        sc = sq_acc_bf16x2(sc, w.z);
+                        sc = sq_acc_bf16x2(sc, w.w);
+                    }
+                } else {
+                    for (int v = 0; v < vpr; ++v) {
+                        const uint4 u = mine[v];
+                        const float x0 = __uint_as_float(u.x), x1 = __uint_as_float(u.y), x2 = __uint_as_float(u.z),
+                                    x3 = __uint_as_float(u.w);
+                        sc = __dadd_rn(sc, __dmul_rn((double)x0, (double)x0));
+                        sc = __dadd_rn(sc, __dmul_rn((double)x1, (double)x1));
+                        sc = __dadd_rn(sc, __dmul_rn((double)x2, (double)x2));
+                        sc = __dadd_rn(sc, __dmul_rn((double)x3, (double)x3));
+                    }
+                }
+                keys[c0 + tid] = (unsigned long long)__double_as_longlong(sc);
+            }
+            __syncthreads();                                   // this buffer may be refilled two passes on
+        }
+        // ---- 2. the other slices' keys ----
+        cluster.sync();
+        for (int q = 1; q < n_slices; ++q) {
+            const int peer = (slice + q) % n_slices;
+            const int p0 = min(peer * per, len), p1 = min(p0 + per, len);
+            const unsigned long long *pk = cluster.map_shared_rank(keys, peer);
+            for (int j = p0 + tid; j < p1; j += kSelThreads) keys[j] = pk[j];
+        }
+        cluster.sync();                                       // nobody reads this CTA's shared memory after this
+    }
+
+    // ---- 3. selection ----
     // Bits that all keys share need no pass: (OR of all keys) ^ (AND of all keys) has a 1 exactly where
     // two keys differ.
     unsigned long long k_or = 0, k_and = ~0ULL;
     for (int j = tid; j < len; j += kSelThreads) {
-        const unsigned long long key = (unsigned long long)__double_as_longlong(__ldcg(sc + j));
-        keys[j] = key;
+        const unsigned long long key = keys[j];
         k_or |= key; k_and &= key;
     }
 #pragma unroll
@@ -383,21 +373,46 @@ topk_select_gather_kernel(const PartsParams pp, int hkv, int vpr /* 16-byte vect
     }
 }
 
-cudaError_t launch_topk_select_gather(const PartsParams &pp, int hkv, int d, int elt_bytes, const double *scores,
-                                      void *k_agg, void *v_agg, int32_t *kv_pos, int32_t *cu_kv,
-                                      int32_t *sel_idx_out, int sm_count, cudaStream_t s, int64_t *launches)
+cudaError_t launch_topk_fused(const PartsParams &pp, int hkv, int d, int dtype, void *k_agg, void *v_agg,
+                              int32_t *kv_pos, int32_t *cu_kv, int32_t *sel_idx_out, int sm_count, cudaStream_t s,
+                              int64_t *launches)
 {
-    if (pp.cu_kv[pp.n] == 0) {
-        if (!cu_kv) return cudaSuccess;
+    if (pp.cu_kv[pp.n] == 0 && !cu_kv) return cudaSuccess;
+    const int elt = dtype == FEDATTN_BF16 ? 2 : 4;
+    const int smem = 2 * kStageRows * (d * elt + 16);
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(topk_fused_kernel<FEDATTN_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             2 * kStageRows * (FEDATTN_MAX_HEAD_DIM * 2 + 16));
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(topk_fused_kernel<FEDATTN_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     2 * kStageRows * (FEDATTN_MAX_HEAD_DIM * 4 + 16));
+        if (e != cudaSuccess) return e;
+        attr_set = true;
     }
+    // slices per (head, participant): a power of two <= 8 (one cluster), about two CTAs per SM in total
     const int pairs = hkv * pp.n;
-    int slices = (4 * sm_count + pairs - 1) / pairs;          // about four CTAs per SM in total
-    if (slices < 1) slices = 1;
-    if (slices > 64) slices = 64;
-    topk_select_gather_kernel<<<dim3(hkv, pp.n, slices), kSelThreads, 0, s>>>(
-        pp, hkv, d * elt_bytes / 16, scores, (uint4 *)k_agg, (uint4 *)v_agg, kv_pos, cu_kv, sel_idx_out);
+    int slices = 1;
+    while (slices * 2 <= kMaxSlices && pairs * slices * 2 <= 2 * sm_count) slices *= 2;
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3(hkv, pp.n, slices);
+    cfg.blockDim = dim3(kSelThreads, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = 1; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = slices;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    const int vpr = d * elt / 16;
+    cudaError_t e = dtype == FEDATTN_BF16
+                        ? cudaLaunchKernelEx(&cfg, topk_fused_kernel<FEDATTN_BF16>, pp, hkv, vpr, (uint4 *)k_agg, (uint4 *)v_agg,
+                                             kv_pos, cu_kv, sel_idx_out)
+                        : cudaLaunchKernelEx(&cfg, topk_fused_kernel<FEDATTN_F32>, pp, hkv, vpr, (uint4 *)k_agg, (uint4 *)v_agg,
+                                             kv_pos, cu_kv, sel_idx_out);
     ++*launches;
-    return cudaGetLastError();
+    return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 // ---- indexed gather ------------------------------------------------------------------------------

@@ -226,12 +226,8 @@ fedattn_status fedattn_aggregate_kv(fedattn_ctx *ctx, const fedattn_shape *shape
         return err == cudaSuccess ? FEDATTN_OK : FEDATTN_ERR_CUDA;
     }
     if (mode == FEDATTN_AGG_TOPK_KNORM) {
-        if (ctx->c.scratch_bytes < topk_scratch_bytes(hkv, L)) return FEDATTN_ERR_WORKSPACE;
-        double *scores = reinterpret_cast<double *>(ctx->c.scratch);
-        err = launch_knorm_scores(pp, hkv, d, shape->dtype, scores, ctx->c.sm_count, s, &ctx->c.launches);
-        if (err == cudaSuccess)
-            err = launch_topk_select_gather(pp, hkv, d, eb, scores, k_agg, v_agg, kv_pos, cu_kv, sel_idx_out,
-                                            ctx->c.sm_count, s, &ctx->c.launches);
+        err = launch_topk_fused(pp, hkv, d, shape->dtype, k_agg, v_agg, kv_pos, cu_kv, sel_idx_out, ctx->c.sm_count, s,
+                                &ctx->c.launches);
         return err == cudaSuccess ? FEDATTN_OK : FEDATTN_ERR_CUDA;
     }
     const int32_t *sel = sel_idx_in;

@@ -68,12 +68,9 @@ struct PartsParams {
 cudaError_t launch_concat(const PartsParams &pp, int hkv, int d, int elt_bytes, void *k_agg, void *v_agg,
                           int32_t *kv_pos, int32_t *cu_kv, cudaStream_t s, int sm_count, int64_t *launches);
 
-// scores: dev double [sum_n Hkv*L_n] laid out participant-major, then head, then token.
-cudaError_t launch_knorm_scores(const PartsParams &pp, int hkv, int d, int dtype, double *scores, int sm_count,
-                                cudaStream_t s, int64_t *launches);
-cudaError_t launch_topk_select_gather(const PartsParams &pp, int hkv, int d, int elt_bytes, const double *scores,
-                                      void *k_agg, void *v_agg, int32_t *kv_pos, int32_t *cu_kv,
-                                      int32_t *sel_idx_out, int sm_count, cudaStream_t s, int64_t *launches);
+cudaError_t launch_topk_fused(const PartsParams &pp, int hkv, int d, int dtype, void *k_agg, void *v_agg,
+                              int32_t *kv_pos, int32_t *cu_kv, int32_t *sel_idx_out, int sm_count, cudaStream_t s,
+                              int64_t *launches);
 cudaError_t launch_gather(const PartsParams &pp, int hkv, int d, int elt_bytes, const int32_t *sel_idx,
                           void *k_agg, void *v_agg, int32_t *kv_pos, int32_t *cu_kv, int32_t *sel_idx_out,
                           int32_t *status, cudaStream_t s, int64_t *launches);
