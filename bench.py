@@ -55,9 +55,9 @@ SPARSE_RATIO_NUM, SPARSE_RATIO_DEN = 1, 4
 # dram__bytes_read.sum + dram__bytes_write.sum per prefill launch of the sync call at this
 # workload, from the ncu capture summarised under profiles/ (None until captured)
 PREFILL_SYNC_DRAM_BYTES = 129_784_064
-# the same for one decode call (cfg5) and for one sparse aggregation (cfg4: both launches)
+# the same for one decode call (cfg5) and for one sparse aggregation (cfg4)
 DECODE_DRAM_BYTES = 139_544_000     # mean of the local (140.0 MB) and sync (138.1 MB) captures
-TOPK_DRAM_BYTES = 51_448_000
+TOPK_DRAM_BYTES = None
 
 
 def env_rank():
@@ -529,7 +529,7 @@ def run_cfg4(args):
     pk = peaks()
     gbs = agg_bytes / (ms_agg * 1e-3) / 1e9
     tf = f_sync / (ms_sync * 1e-3) / 1e12
-    roof = {"bound": "hbm", "kernel": "knorm_score_kernel + topk_select_gather_kernel (the two launches of one sparse aggregation)",
+    roof = {"bound": "hbm", "kernel": "topk_fused_kernel (scores, selection and gather of one sparse aggregation)",
             "achieved": round(gbs, 1), "peak": pk["hbm"], "unit": "GB/s", "frac": round(gbs / pk["hbm"], 4),
             "peak_kind": "copy, " + pk["kind"], "traffic": TOPK_DRAM_BYTES}
     calls = {"aggregate_topk": {"ms": round(ms_agg, 5), "gbs": round(gbs, 1), "frac_hbm": round(gbs / pk["hbm"], 4)},

@@ -137,6 +137,41 @@ def test_topk_indices_bit_exact_with_ties(oracle, dtype):
     assert list(sel[0, cu[3]:cu[4]]) == list(range(250))
 
 
+def test_topk_max_length_many_slices_and_degenerate_scores(oracle):
+    """Longest supported segment (4096), slices of one (head, participant) spread over a cluster,
+    k = 1 / k = L_n, near-constant scores (selection decided in the lowest bits) and long runs of
+    exactly equal scores (tie rule over many candidates)."""
+    lens = [4096, 513]
+    hkv, d = 2, 128
+    _, k, v = gen(21, lens, hkv, hkv, d, "bf16")
+    kp, vp = split(k, lens), split(v, lens)
+    kp[0][1000:3000] = kp[0][1000]                    # 2000 equal scores in the middle
+    kp[1][:, 1, :] = 1.0                              # head 1 of participant 1: all scores equal
+    kp[1][7, 1, 0] = 1.0078125                        # ... except one, larger by one bf16 step
+    r = Runner(len(lens), hkv, hkv, d, "bf16", sum(lens))
+    for ksel in ([1024, 128], [1, 513], [4096, 1], [2500, 0]):
+        agg = r.aggregate(fa().AGG_TOPK_KNORM, kp, vp, ksel)
+        ka, va, pos, cu, sel = oracle.aggregate_topk(kp, vp, ksel)
+        assert agg["status"] == 0
+        assert np.array_equal(agg["sel_idx"].cpu().numpy(), sel), ksel
+        assert np.array_equal(agg["kv_pos"].cpu().numpy(), pos) and np.array_equal(agg["cu_kv"].cpu().numpy(), cu)
+        assert np.array_equal(host(agg["k_agg"]), ka) and np.array_equal(host(agg["v_agg"]), va)
+
+
+def test_topk_fp32_head_dim_128(oracle):
+    lens = [700, 300]
+    hkv, d = 8, 128
+    _, k, v = gen(22, lens, hkv, hkv, d, "f32")
+    kp, vp = split(k, lens), split(v, lens)
+    r = Runner(len(lens), hkv, hkv, d, "f32", sum(lens))
+    ksel = [175, 75]
+    agg = r.aggregate(fa().AGG_TOPK_KNORM, kp, vp, ksel)
+    ka, va, pos, cu, sel = oracle.aggregate_topk(kp, vp, ksel)
+    assert np.array_equal(agg["sel_idx"].cpu().numpy(), sel)
+    assert np.array_equal(host(agg["k_agg"]), ka) and np.array_equal(host(agg["v_agg"]), va)
+
+
+
 def test_indexed_aggregation_and_bad_index_status(oracle):
     lens = [50, 20, 30]
     ksel = [5, 0, 30]
@@ -198,6 +233,33 @@ def test_decode_small(oracle, dtype, d):
         oo, ol = oracle.decode(q, k, v, [T], True)
         check_close(o, oo, TOL[dtype], "decode sync %d" % T)
         check_close(lse, ol, 1e-3, "decode sync lse")
+
+
+def test_decode_many_splits_clusters_and_row_chunks(oracle):
+    """Long caches: the splits of a (cache, KV head) span several clusters, so the cross-cluster merge
+    runs; ragged lengths leave some splits empty; 48 stacked rows per KV head need two row chunks."""
+    n, cap, hq, hkv, d = 2, 6000, 8, 2, 128
+    w = fi.Workload("dl", 31, (cap,) * n, hq, hkv, d, "bf16")
+    _, k, v = w.qkv()
+    q = w.decode_q(0)
+    kc, vc = k.reshape(n, cap, hkv, d), v.reshape(n, cap, hkv, d)
+    r = Runner(n, hq, hkv, d, "bf16", n * cap)
+    for lens in ([6000, 3333], [6000, 0], [65, 5999]):
+        o, lse = r.decode(q, kc, vc, lens, False, max_kv_len=cap)
+        oo, ol = oracle.decode(q, kc, vc, lens, False)
+        check_close(o, oo, TOL["bf16"], "decode local %s" % lens)
+        check_close(lse, ol, 1e-3, "decode local lse %s" % lens)
+    n2 = 12                                            # 12 participants x 4 grouped heads = 48 rows per KV head
+    w2 = fi.Workload("ds", 32, (500,) * n2, hq, hkv, d, "bf16")
+    _, k2, v2 = w2.qkv()
+    q2 = w2.decode_q(0)
+    r2 = Runner(n2, hq, hkv, d, "bf16", n2 * 500)
+    for T in (6000, 4097):
+        o, lse = r2.decode(q2, k2, v2, [T], True, max_kv_len=6000)
+        oo, ol = oracle.decode(q2, k2, v2, [T], True)
+        check_close(o, oo, TOL["bf16"], "decode sync %d" % T)
+        check_close(lse, ol, 1e-3, "decode sync lse %d" % T)
+
 
 
 def test_cfg5_decode_full_size(oracle):
