@@ -557,7 +557,10 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         int gsub0 = 0, gsub1 = 0;                               // KV tiles each sub-tile has been through
         int xb = 0;                                             // exchange buffer parity
         int k = 0;                                              // round of the static schedule
-        auto wg_sync = [&]() { asm volatile("bar.sync 1, %0;" ::"n"(kSoftmaxThreads) : "memory"); };
+        // the threads that share query rows are the warps w, w + 4, ...: one named barrier per row quarter
+        const int bar_id = 1 + (warp & 3);
+        auto wg_sync = [&]() { asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "n"(32 * kSplit) : "memory"); };
+        const bool o_aligned32 = (reinterpret_cast<uintptr_t>(p.o) & 31) == 0;
 
         // One visit = the softmax of one S tile of one sub-tile.  kPartial: some row of the tile has masked
         // columns (they become -inf and every exponential goes through ex2.approx, which maps -inf to 0);
@@ -721,14 +724,20 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                 if (valid) {
                     const float inv = lt > 0.f ? 1.f / lt : 0.f;
                     __nv_bfloat16 *orow = orow0 + t * kD;
+                    // a thread's 32 bytes are one full sector: 256-bit stores halve the store transactions
 #pragma unroll
-                    for (int c = 0; c < kCols; c += 8) {
-                        uint4 w;
-                        w.x = pack_bf16(__uint_as_float(o[c + 0]) * inv, __uint_as_float(o[c + 1]) * inv);
-                        w.y = pack_bf16(__uint_as_float(o[c + 2]) * inv, __uint_as_float(o[c + 3]) * inv);
-                        w.z = pack_bf16(__uint_as_float(o[c + 4]) * inv, __uint_as_float(o[c + 5]) * inv);
-                        w.w = pack_bf16(__uint_as_float(o[c + 6]) * inv, __uint_as_float(o[c + 7]) * inv);
-                        *reinterpret_cast<uint4 *>(orow + c) = w;
+                    for (int c = 0; c < kCols; c += 16) {
+                        uint32_t w[8];
+#pragma unroll
+                        for (int i = 0; i < 8; ++i)
+                            w[i] = pack_bf16(__uint_as_float(o[c + 2 * i]) * inv, __uint_as_float(o[c + 2 * i + 1]) * inv);
+                        if (o_aligned32) {
+                            asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(orow + c), "r"(w[0]), "r"(w[1]),
+                                         "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7]) : "memory");
+                        } else {
+                            *reinterpret_cast<uint4 *>(orow + c) = make_uint4(w[0], w[1], w[2], w[3]);
+                            *reinterpret_cast<uint4 *>(orow + c + 8) = make_uint4(w[4], w[5], w[6], w[7]);
+                        }
                     }
                     if (lse0 && hf == 0) lse0[t] = lt > 0.f ? (m_t + log2f(lt)) * 0.6931471805599453f : -INFINITY;
                 }
