@@ -39,10 +39,10 @@ namespace {
 constexpr int kTileM = 128;          // query rows per CTA
 constexpr int kTileN = 128;          // keys per KV tile
 constexpr int kD = 128;              // head dim
-#ifndef FEDATTN_SPLIT
-#define FEDATTN_SPLIT 2
-#endif
-constexpr int kSplit = FEDATTN_SPLIT; // softmax warpgroups; each owns kCols key columns of every S tile
+// softmax warpgroups; each owns kCols key columns of every S tile.  (Four warpgroups of 32 columns
+// were measured 20 % slower than two of 64: the exponentials are throughput-bound either way and
+// the exchange costs more.)
+constexpr int kSplit = 2;
 constexpr int kCols = kTileN / kSplit;
 constexpr int kSoftmaxThreads = 128 * kSplit;
 constexpr int kThreads = kSoftmaxThreads + 64;   // then one TMA producer warp and one MMA issuer warp
@@ -70,8 +70,8 @@ struct KernelParams {
 
 #ifdef FEDATTN_TRACE
 // Debug build only: cycle stamps of one CTA's pipeline events, [tile][event].
-__device__ long long g_trace[64 * 16];
-#define TRACE(j, e) do { if (k == 0 && blockIdx.x == gridDim.x / 2 && (j) < 64) g_trace[(j) * 16 + (e)] = clock64(); } while (0)
+__device__ long long g_trace[64 * 8];
+#define TRACE(j, e) do { if (k == 0 && blockIdx.x == gridDim.x / 2 && (j) < 64) g_trace[(j) * 8 + (e)] = clock64(); } while (0)
 #else
 #define TRACE(j, e) do { } while (0)
 #endif
@@ -246,9 +246,9 @@ __device__ __forceinline__ float max3(float a, float b, float c)
 // 2^n by adding n to the exponent field.  The magic constant 1.5 * 2^23 makes the low mantissa
 // bits of x + magic hold n.  x is clamped at -125 so that the exponent arithmetic cannot wrap:
 // anything smaller contributes 2^-125 instead of an even smaller value.  Needs x <= 100.
-#ifndef FEDATTN_POLY_MASK
-#define FEDATTN_POLY_MASK 0x49     // bit (c & 7) set: column pair c takes the polynomial instead of ex2.approx
-#endif
+// bit (c & 7) set: column pair c takes the polynomial instead of ex2.approx.  3 of 8 pairs: measured
+// best of 0, 2, 3, 4, 5 of 8 (the polynomial loads the ALU pipe as much as ex2 loads its own unit).
+constexpr uint32_t kPolyMask = 0x49;
 __device__ __forceinline__ void exp2_poly_x2(uint64_t x2, float &p0, float &p1)
 {
     float x0, x1;
@@ -571,7 +571,6 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             const uint32_t tS = tmem_base + lane_base + kColS + t * 128 + kCols * hf;   // fp32 S, this part
             const uint32_t tP = tS;                                                      // bf16 P, this part
             const uint32_t tO = tmem_base + lane_base + kColO + t * 128 + kCols * hf;
-            if (tid == 0 && t == 1) TRACE(j, 13);
             mbar_wait(s_full + t, gt & 1, abort_flag, kp.status);
             if (tid == 0) TRACE(j, t ? 5 : 0);
             tc_fence_after();
@@ -579,7 +578,6 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
 #pragma unroll
             for (int c = 0; c < kCols; c += 32) FEDATTN_TMEM_LD32(tS + c, (s + c));
             tmem_wait_ld();
-            if (tid == 0 && t == 0) TRACE(j, 8);
             if (kPartial) {
 #pragma unroll
                 for (int c = 0; c < kCols; ++c)
@@ -604,7 +602,6 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             for (int q = 1; q < kSplit; ++q) rm = fmaxf(rm, x_max[(xb * kSplit + ((hf + q) & (kSplit - 1))) * kTileM + r]);
             xb ^= 1;
             const float t_max = rm * sl2;
-            if (tid == 0 && t == 0) TRACE(j, 10);
             if (j == 0) {
                 m_used = (t_max == -INFINITY) ? 0.f : t_max;
             } else {
@@ -637,7 +634,7 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                     const uint64_t x2 = fma_f32x2(pack_f32x2(__uint_as_float(s[cc * 32 + 2 * c]),
                                                              __uint_as_float(s[cc * 32 + 2 * c + 1])), sl2_2, negm2);
                     float p0, p1;
-                    if (!kPartial && ((FEDATTN_POLY_MASK >> (c & 7)) & 1)) {
+                    if (!kPartial && ((kPolyMask >> (c & 7)) & 1)) {
                         exp2_poly_x2(x2, p0, p1);
                     } else {
                         float x0, x1;
@@ -652,13 +649,11 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             float r0, r1;
             unpack_f32x2(add_f32x2(add_f32x2(sum2[0], sum2[1]), add_f32x2(sum2[2], sum2[3])), r0, r1);
             l += r0 + r1;
-            if (tid == 0 && t == 0) TRACE(j, 11);
             tmem_wait_st();
             tc_fence_before();
             if (tid == 0) TRACE(j, t ? 6 : 1);
             __syncwarp();
             if (lane == 0) mbar_arrive(p_full + kSplit * t + hf);      // one arrival per warp
-            if (tid == 0 && t == 0) TRACE(j, 12);
         };
 
         for (k = 0; k < n_rounds; ++k) {
@@ -693,7 +688,6 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                 const int gt = (t ? gsub1 : gsub0) + j;
                 if (j < n_full) visit(std::false_type{}, t, j, gt, kCols, m_a, l_a);
                 else visit(std::true_type{}, t, j, gt, c_r - j * kTileN, m_a, l_a);
-                if (tid == 0 && t == 0) TRACE(j, 9);
                 if (n_sub == 2) {
                     float x = m_a; m_a = m_b; m_b = x;
                     x = l_a; l_a = l_b; l_b = x;
