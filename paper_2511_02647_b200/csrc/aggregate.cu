@@ -359,13 +359,30 @@ topk_fused_kernel(const PartsParams pp, int hkv, int vpr /* 16-byte vectors per 
     const int n_out = o_hi - o_lo;
     const int64_t out_row0 = (int64_t)h * T + pp.cu_kv[n] + o_lo;
     const uint4 *ksrc = reinterpret_cast<const uint4 *>(pp.k[n]), *vsrc = reinterpret_cast<const uint4 *>(pp.v[n]);
-    for (int i = tid; i < n_out * vpr; i += kSelThreads) {
-        const int r = i / vpr, vi = i - r * vpr;
-        const int64_t src = ((int64_t)my_rows[r] * hkv + h) * vpr + vi;
-        const int64_t dst = (out_row0 + r) * vpr + vi;
-        const uint4 kk = ld_stream(ksrc + src), vv = ld_stream(vsrc + src);
-        k_agg[dst] = kk;
-        v_agg[dst] = vv;
+    // four vectors of K and of V in flight per thread before the first store
+    constexpr int kGatherUnroll = 4;
+    for (int i0 = tid; i0 < n_out * vpr; i0 += kSelThreads * kGatherUnroll) {
+        uint4 kk[kGatherUnroll], vv[kGatherUnroll];
+#pragma unroll
+        for (int u = 0; u < kGatherUnroll; ++u) {
+            const int i = i0 + u * kSelThreads;
+            if (i < n_out * vpr) {
+                const int r = i / vpr, vi = i - r * vpr;
+                const int64_t src = ((int64_t)my_rows[r] * hkv + h) * vpr + vi;
+                kk[u] = ld_stream(ksrc + src);
+                vv[u] = ld_stream(vsrc + src);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < kGatherUnroll; ++u) {
+            const int i = i0 + u * kSelThreads;
+            if (i < n_out * vpr) {
+                const int r = i / vpr, vi = i - r * vpr;
+                const int64_t dst = (out_row0 + r) * vpr + vi;
+                k_agg[dst] = kk[u];
+                v_agg[dst] = vv[u];
+            }
+        }
     }
     for (int r = tid; r < n_out; r += kSelThreads) {
         if (kv_pos) kv_pos[out_row0 + r] = pp.off[n] + my_rows[r];
