@@ -181,6 +181,28 @@ def sync(q, k_agg, v_agg, kv_pos=None, q_pos=None, kv_head_major: bool = False,
     return o, lse
 
 
+def sync_exchange(q, k, v, seqlens, k_agg, v_agg, kv_pos, cu_kv, scale: float = 0.0,
+                  rows: Optional[Sequence[int]] = None):
+    """Sync block with sparse KV exchange: every participant attends its own complete (causal)
+    segment plus the exchanged, sparsified keys of the other participants that are not later than
+    the query.  q [L,Hq,d]; k, v [L,Hkv,d] local; k_agg, v_agg [Hkv,T,d] head-major aggregate with
+    kv_pos [Hkv,T] and participant ranges cu_kv [N+1]."""
+    q, k, v, k_agg, v_agg = _f64(q), _f64(k), _f64(v), _f64(k_agg), _f64(v_agg)
+    L, hq, d = q.shape
+    hkv, T, _ = k_agg.shape
+    off = offsets(seqlens)
+    kvp, cu = _i32(kv_pos), _i32(cu_kv)
+    assert kvp.shape == (hkv, T) and len(cu) == len(off)
+    r = None if rows is None else np.ascontiguousarray(rows, dtype=np.int64)
+    n_rows = L if r is None else len(r)
+    o = np.zeros((n_rows, hq, d)); lse = np.zeros((n_rows, hq))
+    _load().fedattn_oracle_sync_exchange(_p(q), _p(k), _p(v), _p(off), C.c_int32(len(off) - 1),
+                                         _p(k_agg), _p(v_agg), _p(kvp), _p(cu), C.c_int64(T),
+                                         C.c_int32(hq), C.c_int32(hkv), C.c_int32(d),
+                                         C.c_double(_scale(scale, d)), _p(r), C.c_int64(n_rows), _p(o), _p(lse))
+    return o, lse
+
+
 def decode(q, k_cache, v_cache, kv_len, sync_mode: bool, scale: float = 0.0):
     """Decode step.  LOCAL: caches [N,cap,Hkv,d], kv_len [N].  SYNC: cache [T,Hkv,d], kv_len [1].
     q [N,Hq,d].  Returns (o [N,Hq,d], lse [N,Hq])."""

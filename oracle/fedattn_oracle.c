@@ -292,6 +292,92 @@ void fedattn_oracle_sync(const double *q, int64_t n_q, const int32_t *q_pos,
 }
 
 /*
+ * Sync block with sparse KV exchange as the paper's experiment describes it (Sec. VI, the
+ * discussion of the sparsity-ratio figure: "sparse KV exchange preserves self-attention on
+ * complete local tokens within each participant while sparsifying remote KVs"): row i of
+ * participant n attends
+ *     A = its own keys  { j : off_n <= j <= i }                       (complete, causal), and
+ *     B = the exchanged keys of the OTHER participants that are not later than i,
+ *         { t outside [cu_kv[n], cu_kv[n+1]) : kv_pos[kvh][t] <= i }  (sparsified, causal on the
+ *         global position),
+ * with one softmax over A u B.  k, v: packed local tensors [L, Hkv, d]; k_agg, v_agg: head-major
+ * aggregate [Hkv, T, d] with kv_pos [Hkv, T] and participant ranges cu_kv [N+1].
+ * rows / o / lse as in fedattn_oracle_local.
+ */
+void fedattn_oracle_sync_exchange(const double *q, const double *k, const double *v,
+                                  const int32_t *off, int32_t n_participants,
+                                  const double *k_agg, const double *v_agg, const int32_t *kv_pos,
+                                  const int32_t *cu_kv, int64_t total_kv,
+                                  int32_t hq, int32_t hkv, int32_t d, double scale,
+                                  const int64_t *rows, int64_t n_rows, double *o, double *lse)
+{
+    const int32_t g = hq / hkv;
+    const int64_t L = off[n_participants];
+#pragma omp parallel
+    {
+        const size_t cap = (size_t)(L + total_kv > 0 ? L + total_kv : 1);
+        double *logits = (double *)malloc(sizeof(double) * cap);
+        const double **vrow = (const double **)malloc(sizeof(double *) * cap);
+#pragma omp for schedule(dynamic, 1) collapse(2)
+        for (int64_t r = 0; r < n_rows; ++r) {
+            for (int32_t h = 0; h < hq; ++h) {
+                const int64_t i = rows ? rows[r] : r;
+                int32_t n = 0;
+                while (!(off[n] <= i && i < off[n + 1]))
+                    ++n;
+                const int32_t kvh = h / g;
+                const double *qr = q + (i * hq + h) * d;
+                double *orow = o + (r * hq + h) * d;
+                int64_t na = 0;
+                double mx = -INFINITY;
+                for (int64_t j = off[n]; j <= i; ++j) {            /* set A */
+                    const double *kr = k + (j * hkv + kvh) * d;
+                    double s = 0.0;
+                    for (int32_t c = 0; c < d; ++c)
+                        s += qr[c] * kr[c];
+                    logits[na] = s * scale;
+                    vrow[na] = v + (j * hkv + kvh) * d;
+                    if (logits[na] > mx)
+                        mx = logits[na];
+                    ++na;
+                }
+                for (int64_t t = 0; t < total_kv; ++t) {           /* set B */
+                    if (t >= cu_kv[n] && t < cu_kv[n + 1])
+                        continue;
+                    if (kv_pos[(int64_t)kvh * total_kv + t] > i)
+                        continue;
+                    const double *kr = k_agg + ((int64_t)kvh * total_kv + t) * d;
+                    double s = 0.0;
+                    for (int32_t c = 0; c < d; ++c)
+                        s += qr[c] * kr[c];
+                    logits[na] = s * scale;
+                    vrow[na] = v_agg + ((int64_t)kvh * total_kv + t) * d;
+                    if (logits[na] > mx)
+                        mx = logits[na];
+                    ++na;
+                }
+                for (int32_t c = 0; c < d; ++c)
+                    orow[c] = 0.0;
+                double denom = 0.0;
+                for (int64_t a = 0; a < na; ++a) {
+                    logits[a] = exp(logits[a] - mx);
+                    denom += logits[a];
+                }
+                for (int64_t a = 0; a < na; ++a) {
+                    const double p = logits[a] / denom;
+                    for (int32_t c = 0; c < d; ++c)
+                        orow[c] += p * vrow[a][c];
+                }
+                if (lse)
+                    lse[r * hq + h] = mx + log(denom);            /* A is never empty: the row itself */
+            }
+        }
+        free(logits);
+        free(vrow);
+    }
+}
+
+/*
  * Decode step (Sec. IV-C): one new query token per participant, later than every cached
  * row, so the whole cache is allowed.
  *   sync == 0: participant n reads its own cache k_cache + n * cache_stride_participant,

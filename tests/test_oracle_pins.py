@@ -298,6 +298,99 @@ def test_sparse_sync_special_cases_and_bruteforce(oracle):
     assert np.array_equal(fin, np.isfinite(lse)) and np.abs(lse[fin] - bl[fin]).max() < 1e-12
 
 
+# ----------------------------------------------------------------------------------------------
+# sync block with sparse KV exchange (own segment complete, remote keys sparsified)
+# ----------------------------------------------------------------------------------------------
+def lse_merge(o_a, lse_a, o_b, lse_b):
+    """Attention over a disjoint union of key sets from the two partial results (closed form)."""
+    m = np.maximum(lse_a, lse_b)
+    m = np.where(np.isfinite(m), m, 0.0)
+    wa, wb = np.exp(lse_a - m), np.exp(lse_b - m)
+    z = wa + wb
+    o = (o_a * wa[..., None] + o_b * wb[..., None]) / np.where(z > 0, z, 1.0)[..., None]
+    return o, m + np.log(z)
+
+
+def test_sync_exchange_special_cases(oracle):
+    lens = [4, 3, 5]
+    L, Hq, Hkv, d = sum(lens), 4, 2, 4
+    q, k, v = randn(L, Hq, d), randn(L, Hkv, d), randn(L, Hkv, d)
+    cuts = np.cumsum(lens)[:-1]
+    ks, vs = np.split(k, cuts), np.split(v, cuts)
+    # every remote key exchanged => the dense sync block (= centralised attention)
+    ka, va, pos, cu, _ = oracle.aggregate_topk(ks, vs, lens)
+    o, lse = oracle.sync_exchange(q, k, v, lens, ka, va, pos, cu)
+    dense, dense_lse = oracle.sync(q, k, v)
+    assert np.abs(o - dense).max() < 1e-13 and np.abs(lse - dense_lse).max() < 1e-13
+    # nothing exchanged => the local block
+    ka, va, pos, cu, _ = oracle.aggregate_topk(ks, vs, [0, 0, 0])
+    o, lse = oracle.sync_exchange(q, k, v, lens, ka, va, pos, cu)
+    loc, loc_lse = oracle.local(q, k, v, lens)
+    assert np.abs(o - loc).max() < 1e-13 and np.abs(lse - loc_lse).max() < 1e-13
+    # a participant's own exchanged rows must not be counted twice: with only participant 1 sending,
+    # participant 1's own rows are unchanged and participant 0 (earlier) sees nothing new
+    ka, va, pos, cu, _ = oracle.aggregate_topk(ks, vs, [0, 3, 0])
+    o, lse = oracle.sync_exchange(q, k, v, lens, ka, va, pos, cu)
+    assert np.abs(o[:7] - loc[:7]).max() < 1e-13 and np.abs(lse[:7] - loc_lse[:7]).max() < 1e-13
+    assert np.abs(o[7:] - loc[7:]).max() > 1e-3
+
+
+def test_sync_exchange_bruteforce_and_equal_keys(oracle):
+    lens = [3, 4, 2, 4]
+    L, Hq, Hkv, d = sum(lens), 4, 2, 3
+    q, k, v = randn(L, Hq, d), randn(L, Hkv, d), randn(L, Hkv, d)
+    off = np.concatenate([[0], np.cumsum(lens)])
+    ks, vs = np.split(k, off[1:-1]), np.split(v, off[1:-1])
+    ksel = [2, 1, 0, 3]
+    ka, va, pos, cu, sel = oracle.aggregate_topk(ks, vs, ksel)
+    o, lse = oracle.sync_exchange(q, k, v, lens, ka, va, pos, cu)
+    g = Hq // Hkv
+    T = ka.shape[1]
+    seg = np.searchsorted(off, np.arange(L), side="right") - 1
+
+    # brute force over a tagged union: ("l", j) local rows, ("a", t) exchanged rows
+    def allowed(i, h):
+        n, kvh = seg[i], h // g
+        own = [("l", j) for j in range(off[n], i + 1)]
+        remote = [("a", t) for t in range(T) if not (cu[n] <= t < cu[n + 1]) and pos[kvh, t] <= i]
+        return own + remote, kvh
+
+    K = lambda key, kh: k[key[1], kh] if key[0] == "l" else ka[kh, key[1]]
+    V = lambda key, kh: v[key[1], kh] if key[0] == "l" else va[kh, key[1]]
+    bo, bl = brute_attention(q, K, V, allowed, 1 / math.sqrt(d))
+    assert np.abs(o - bo).max() < 1e-12 and np.abs(lse - bl).max() < 1e-12
+    # all keys equal => uniform weights: o = mean of V over the allowed set, lse = logit + ln |allowed|
+    k_eq = np.broadcast_to(randn(1, Hkv, d), (L, Hkv, d)).copy()
+    ka2, va2, pos2, cu2 = oracle.aggregate_indexed(np.split(k_eq, off[1:-1]), vs, ksel, sel)
+    o, lse = oracle.sync_exchange(q, k_eq, v, lens, ka2, va2, pos2, cu2)
+    for i in (0, 2, 3, 6, 8, 9, 12):
+        for h in range(Hq):
+            keys, kvh = allowed(i, h)
+            mean_v = np.mean([V(key, kvh) for key in keys], axis=0)
+            logit = float(q[i, h] @ k_eq[0, kvh]) / math.sqrt(d)
+            assert np.abs(o[i, h] - mean_v).max() < 1e-12
+            assert abs(lse[i, h] - (logit + math.log(len(keys)))) < 1e-12
+
+
+def test_sync_exchange_is_local_merged_with_remote_only_sync(oracle):
+    """The decomposition the CUDA path uses: attention over own keys (local block) and over the
+    exchanged keys of earlier participants (a sync call whose query position is the last position
+    before the participant's segment), merged through their log-sum-exps."""
+    lens = [5, 2, 6, 3]
+    L, Hq, Hkv, d = sum(lens), 4, 2, 4
+    q, k, v = randn(L, Hq, d), randn(L, Hkv, d), randn(L, Hkv, d)
+    off = np.concatenate([[0], np.cumsum(lens)])
+    ks, vs = np.split(k, off[1:-1]), np.split(v, off[1:-1])
+    ka, va, pos, cu, _ = oracle.aggregate_topk(ks, vs, [3, 1, 4, 2])
+    want, want_lse = oracle.sync_exchange(q, k, v, lens, ka, va, pos, cu)
+    seg = np.searchsorted(off, np.arange(L), side="right") - 1
+    o_l, lse_l = oracle.local(q, k, v, lens)
+    o_r, lse_r = oracle.sync(q, ka, va, kv_pos=pos, q_pos=off[seg] - 1, kv_head_major=True)
+    o, lse = lse_merge(o_l, lse_l, o_r, lse_r)
+    assert np.abs(o - want).max() < 1e-12 and np.abs(lse - want_lse).max() < 1e-12
+
+
+
 def test_gqa_equals_mha_with_repeated_kv_heads(oracle):
     lens = [6, 5]
     L, Hq, Hkv, d = sum(lens), 6, 2, 8
