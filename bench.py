@@ -536,6 +536,17 @@ def run_cfg4(args):
     def step(i):
         agg(i); sync(i)
 
+    # the paper-experiment variant of the sync block: own segment complete + the sparsified keys of the
+    # earlier participants (fedattn_local + fedattn_sync_remote + fedattn_merge); reported, not part of `value`
+    o_b = torch.empty_like(sets[0]["q"])
+    lse_a = torch.empty((L, Hq), dtype=torch.float32, device=dev); lse_b = torch.empty_like(lse_a)
+
+    def exchange(i):
+        b = sets[i % n_sets]
+        fa.fedattn_local(ctx, shape, b["q"], b["k"], b["v"], cu, b["o"], lse_a)
+        fa.fedattn_sync_remote(ctx, shape, b["q"], cu, b["k_sp"], b["v_sp"], b["pos"], T, True, o_b, lse_b)
+        fa.fedattn_merge(ctx, shape, L, b["o"], lse_a, o_b, lse_b, b["o"], None)
+
     K, W = args.steps, max(args.warmup, 3)
     step(0)
     pos = sets[0]["pos"].to(torch.int64)
@@ -545,6 +556,8 @@ def run_cfg4(args):
     sampler = ClockSampler(0); sampler.start(); time.sleep(0.25)
     ms_agg = _timed(torch, stream, agg, K, W)
     ms_sync = _timed(torch, stream, sync, K, W)
+    ms_exch = _timed(torch, stream, exchange, K, W)
+    f_exch = 4.0 * d * Hq * (sum(n * (n + 1) // 2 for n in seqlens) + sum(seqlens[n] * sum(ksel[:n]) for n in range(N)))
     l0 = ctx.launch_count()
     ms_step = _timed(torch, stream, step, K, W)
     launches = (ctx.launch_count() - l0) * K // (K + W)
@@ -571,7 +584,9 @@ def run_cfg4(args):
             "traffic": TOPK_DRAM_BYTES}
     calls = {"aggregate_topk": {"ms": round(ms_agg, 5), "gbs": round(gbs, 1), "frac_hbm": round(gbs / pk["hbm"], 4),
                                 "graph_ms": round(g_agg, 5), "graph_gbs": round(g_gbs, 1), "graph_frac_hbm": round(g_gbs / pk["hbm"], 4)},
-             "sync_sparse": {"ms": round(ms_sync, 5), "tflops": round(tf, 2), "frac_tensor": round(tf / pk["tensor"], 4)}}
+             "sync_sparse": {"ms": round(ms_sync, 5), "tflops": round(tf, 2), "frac_tensor": round(tf / pk["tensor"], 4)},
+             "sync_exchange_own_complete": {"ms": round(ms_exch, 5), "tflops": round(f_exch / (ms_exch * 1e-3) / 1e12, 2),
+                                            "launches": 3}}
     _line(args, "fedattn_aggregate_gbs", "GB/s", gbs, ms_step, "bf16",
           {"workload": w.name, "participants": N, "tokens_per_participant": seqlens[0], "q_heads": Hq, "kv_heads": Hkv,
            "head_dim": d, "keep_per_kv_head": w.k_sel, "step": "aggregate_topk + sync over the selected KV",

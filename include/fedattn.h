@@ -149,6 +149,33 @@ fedattn_status fedattn_sync(fedattn_ctx *ctx, const fedattn_shape *shape,
                             int64_t total_kv, int32_t kv_head_major,
                             void *o, float *lse, fedattn_stream stream);
 
+/* ---- sync block with sparse KV exchange -----------------------------------------------------
+ * Paper: Sec. VI, discussion of the sparsity-ratio experiment: "sparse KV exchange preserves
+ * self-attention on complete local tokens within each participant while sparsifying remote KVs".
+ * Row i of participant n attends its own keys off_n..i (complete) and the exchanged keys of the
+ * other participants that are not later than i, under ONE softmax.  With contiguous segments the
+ * second set is "aggregated rows positioned before off_n", so the block is computed as
+ *     fedattn_local (o_a, lse_a)  +  fedattn_sync_remote (o_b, lse_b)  ->  fedattn_merge.
+ *
+ * fedattn_sync_remote: like fedattn_sync, but query row i of participant n (segments given by the
+ *   HOST array cu_seqlens_host [N+1]) attends aggregated row j of KV head h iff
+ *   kv_pos[h][j] < off_n.  shape->causal must be 1 (UNSUPPORTED otherwise).  Rows of the first
+ *   participant, and any row with nothing before its segment, get o = 0 and lse = -inf.
+ *   lse is needed for the merge (pass a buffer).
+ * fedattn_merge: o = (e^{lse_a} o_a + e^{lse_b} o_b) / (e^{lse_a} + e^{lse_b}),
+ *   lse = log(e^{lse_a} + e^{lse_b}) for n_rows query rows; o_a, o_b, o dev [n_rows,Hq,d] in
+ *   shape->dtype, lse_a, lse_b dev float [n_rows,Hq], lse dev float or NULL.  o may alias o_a or
+ *   o_b.  Two results that are both empty (-inf) merge to o = 0, lse = -inf. */
+fedattn_status fedattn_sync_remote(fedattn_ctx *ctx, const fedattn_shape *shape,
+                                   const void *q, const int32_t *cu_seqlens_host,
+                                   const void *k_agg, const void *v_agg, const int32_t *kv_pos,
+                                   int64_t total_kv, int32_t kv_head_major,
+                                   void *o, float *lse, fedattn_stream stream);
+
+fedattn_status fedattn_merge(fedattn_ctx *ctx, const fedattn_shape *shape, int64_t n_rows,
+                             const void *o_a, const float *lse_a, const void *o_b, const float *lse_b,
+                             void *o, float *lse, fedattn_stream stream);
+
 /* ---- decode: one new query token per participant over cached KV -------------------------------
  * Paper: Sec. IV-C "Output Generation" (blocks that ran local attention cache local KV, blocks
  * that ran global attention cache the global KV), Sec. III-C (O(L) per step, memory-bound).

@@ -5,5 +5,5 @@ raises if the library has not been built or cannot be loaded."""
 from .binding import (  # noqa: F401
     AGG_CONCAT, AGG_INDEXED, AGG_TOPK_KNORM, BF16, DECODE_LOCAL, DECODE_SYNC, F32,
     FedAttnError, Context, Shape, exported_symbols, fedattn_aggregate_kv, fedattn_decode, fedattn_decode_noalloc,
-    fedattn_local, fedattn_sync, fedattn_workspace_bytes, library_path, status_string,
+    fedattn_local, fedattn_merge, fedattn_sync, fedattn_sync_remote, fedattn_workspace_bytes, library_path, status_string,
 )

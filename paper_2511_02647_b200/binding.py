@@ -18,7 +18,7 @@ DECODE_LOCAL, DECODE_SYNC = 0, 1
 
 _SYMBOLS = ["fedattn_workspace_bytes", "fedattn_create", "fedattn_destroy", "fedattn_status_string",
             "fedattn_poll", "fedattn_launch_count", "fedattn_local", "fedattn_aggregate_kv",
-            "fedattn_sync", "fedattn_decode", "fedattn_decode_noalloc"]
+            "fedattn_sync", "fedattn_sync_remote", "fedattn_merge", "fedattn_decode", "fedattn_decode_noalloc"]
 
 
 class FedAttnError(RuntimeError):
@@ -70,6 +70,10 @@ def _load():
                                          C.POINTER(i32), C.POINTER(i32), vp, vp, vp, vp, vp, vp, vp]
     lib.fedattn_sync.restype = C.c_int
     lib.fedattn_sync.argtypes = [vp, C.POINTER(Shape), vp, i64, vp, vp, vp, vp, i64, i32, vp, vp, vp]
+    lib.fedattn_sync_remote.restype = C.c_int
+    lib.fedattn_sync_remote.argtypes = [vp, C.POINTER(Shape), vp, C.POINTER(i32), vp, vp, vp, i64, i32, vp, vp, vp]
+    lib.fedattn_merge.restype = C.c_int
+    lib.fedattn_merge.argtypes = [vp, C.POINTER(Shape), i64, vp, vp, vp, vp, vp, vp, vp]
     lib.fedattn_decode.restype = C.c_int
     lib.fedattn_decode.argtypes = [vp, C.POINTER(Shape), i32, vp, vp, vp, i64, vp, i32, vp, vp, vp]
     lib.fedattn_decode_noalloc.restype = C.c_int
@@ -180,6 +184,22 @@ def fedattn_sync(ctx: Context, shape: Shape, q, q_pos, k_agg, v_agg, kv_pos, tot
     _check(_lib.fedattn_sync(ctx.handle, C.byref(shape), _ptr(q), int(q.shape[0]), _ptr(q_pos), _ptr(k_agg),
                              _ptr(v_agg), _ptr(kv_pos), int(total_kv), int(bool(kv_head_major)), _ptr(o),
                              _ptr(lse), _stream(stream)), "fedattn_sync")
+
+
+def fedattn_sync_remote(ctx: Context, shape: Shape, q, cu_seqlens_host: Sequence[int], k_agg, v_agg, kv_pos,
+                        total_kv: int, kv_head_major: bool, o, lse, stream=None):
+    cu = _i32_array(cu_seqlens_host)
+    if len(cu) != shape.n_participants + 1:
+        raise ValueError("cu_seqlens must have N+1 entries")
+    _check(_lib.fedattn_sync_remote(ctx.handle, C.byref(shape), _ptr(q), cu, _ptr(k_agg), _ptr(v_agg), _ptr(kv_pos),
+                                    int(total_kv), int(bool(kv_head_major)), _ptr(o), _ptr(lse), _stream(stream)),
+           "fedattn_sync_remote")
+
+
+def fedattn_merge(ctx: Context, shape: Shape, n_rows: int, o_a, lse_a, o_b, lse_b, o, lse=None, stream=None):
+    _check(_lib.fedattn_merge(ctx.handle, C.byref(shape), int(n_rows), _ptr(o_a), _ptr(lse_a), _ptr(o_b), _ptr(lse_b),
+                              _ptr(o), _ptr(lse), _stream(stream)), "fedattn_merge")
+
 
 
 def fedattn_decode(ctx: Context, shape: Shape, mode: int, q, k_cache, v_cache, cache_stride_participant: int,

@@ -282,6 +282,73 @@ fedattn_status fedattn_sync(fedattn_ctx *ctx, const fedattn_shape *shape, const 
     return err == cudaSuccess ? FEDATTN_OK : FEDATTN_ERR_CUDA;
 }
 
+fedattn_status fedattn_sync_remote(fedattn_ctx *ctx, const fedattn_shape *shape, const void *q, const int32_t *cu,
+                                   const void *k_agg, const void *v_agg, const int32_t *kv_pos, int64_t total_kv,
+                                   int32_t kv_head_major, void *o, float *lse, fedattn_stream stream)
+{
+    if (!ctx || !shape_ok(shape) || !cu || total_kv < 0 || total_kv > 0x7fffffffLL) return FEDATTN_ERR_INVALID_ARG;
+    if (kv_head_major != 0 && kv_head_major != 1) return FEDATTN_ERR_INVALID_ARG;
+    if (!shape->causal) return FEDATTN_ERR_UNSUPPORTED;       // "before the segment" needs the causal order
+    const int N = shape->n_participants;
+    if (cu[0] != 0) return FEDATTN_ERR_INVALID_ARG;
+    for (int n = 0; n < N; ++n)
+        if (cu[n + 1] < cu[n]) return FEDATTN_ERR_INVALID_ARG;
+    const int64_t L = cu[N];
+    if (L == 0) return FEDATTN_OK;
+    if (!q || !o || !aligned16(q) || !aligned16(o)) return FEDATTN_ERR_INVALID_ARG;
+    if (total_kv > 0 && (!k_agg || !v_agg || !aligned16(k_agg) || !aligned16(v_agg))) return FEDATTN_ERR_INVALID_ARG;
+    DeviceGuard g(ctx->c.device);
+    if (!g.ok) return FEDATTN_ERR_CUDA;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    cudaError_t err;
+    if (shape->dtype == FEDATTN_BF16 && shape->head_dim == 128 && total_kv > 0 && prefill_sm100_supported(&ctx->c)) {
+        PrefillParams p;
+        memset(&p, 0, sizeof(p));
+        p.q = q; p.k = k_agg; p.v = v_agg; p.o = o; p.lse = lse;
+        p.n_q_rows = L; p.total_kv = total_kv;
+        p.hq = shape->n_q_heads; p.hkv = shape->n_kv_heads;
+        p.scale = eff_scale(shape); p.causal = 1; p.sync = 1; p.remote_only = 1; p.kv_head_major = kv_head_major;
+        p.kv_pos = kv_pos; p.n_seg = N;
+        memcpy(p.cu, cu, sizeof(int32_t) * (N + 1));
+        err = launch_prefill_sm100(&ctx->c, p, s, &ctx->c.launches);
+    } else {
+        GenericParams p;
+        memset(&p, 0, sizeof(p));
+        p.q = q; p.k = k_agg; p.v = v_agg; p.o = o; p.lse = lse;
+        p.n_rows = L; p.hq = shape->n_q_heads; p.hkv = shape->n_kv_heads; p.d = shape->head_dim;
+        p.scale = eff_scale(shape); p.causal = 1; p.mode = kSync; p.remote_only = 1;
+        if (kv_head_major) {
+            p.kv_tok_stride = shape->head_dim;
+            p.kv_head_stride = total_kv * shape->head_dim;
+            p.kv_pos_head_stride = total_kv;
+        } else {
+            p.kv_tok_stride = (int64_t)shape->n_kv_heads * shape->head_dim;
+            p.kv_head_stride = shape->head_dim;
+            p.kv_pos_head_stride = 0;
+        }
+        p.total_kv = total_kv; p.kv_pos = kv_pos;
+        p.n_seg = N;
+        memcpy(p.cu, cu, sizeof(int32_t) * (N + 1));
+        err = launch_attn_generic(p, shape->dtype, s, &ctx->c.launches);
+    }
+    return err == cudaSuccess ? FEDATTN_OK : FEDATTN_ERR_CUDA;
+}
+
+fedattn_status fedattn_merge(fedattn_ctx *ctx, const fedattn_shape *shape, int64_t n_rows, const void *o_a,
+                             const float *lse_a, const void *o_b, const float *lse_b, void *o, float *lse,
+                             fedattn_stream stream)
+{
+    if (!ctx || !shape_ok(shape) || n_rows < 0) return FEDATTN_ERR_INVALID_ARG;
+    if (n_rows == 0) return FEDATTN_OK;
+    if (!o_a || !o_b || !lse_a || !lse_b || !o) return FEDATTN_ERR_INVALID_ARG;
+    if (!aligned16(o_a) || !aligned16(o_b) || !aligned16(o)) return FEDATTN_ERR_INVALID_ARG;
+    DeviceGuard g(ctx->c.device);
+    if (!g.ok) return FEDATTN_ERR_CUDA;
+    cudaError_t err = launch_merge(shape->dtype, n_rows, shape->n_q_heads, shape->head_dim, o_a, lse_a, o_b, lse_b, o, lse,
+                                   static_cast<cudaStream_t>(stream), &ctx->c.launches);
+    return err == cudaSuccess ? FEDATTN_OK : FEDATTN_ERR_CUDA;
+}
+
 fedattn_status fedattn_decode(fedattn_ctx *ctx, const fedattn_shape *shape, int32_t mode, const void *q,
                               const void *k_cache, const void *v_cache, int64_t cache_stride,
                               const int32_t *kv_len, int32_t max_kv_len, void *o, float *lse,

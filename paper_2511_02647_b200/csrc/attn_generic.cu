@@ -45,6 +45,11 @@ attn_generic_kernel(const GenericParams p)
         kv_hi = p.causal ? row + 1 : (int64_t)p.cu[n + 1];
         test_pos = false;
     } else if (p.mode == kSync) {
+        if (p.remote_only) {                         // position = last one before the row's own segment
+            int n = 0;
+            while (n + 1 < p.n_seg && row >= p.cu[n + 1]) ++n;
+            pos = (int64_t)p.cu[n] - 1;
+        }
         kv_hi = p.total_kv;
         if (p.causal && !p.kv_pos) {                 // identity positions: a prefix
             kv_hi = min(kv_hi, pos + 1);

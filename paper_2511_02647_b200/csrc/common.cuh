@@ -42,6 +42,7 @@ struct GenericParams {
     float scale;
     int32_t causal;
     int32_t mode;                 // GenericMode
+    int32_t remote_only;          // kSync: a row's position is the last one before its segment (cu)
     int64_t kv_tok_stride;        // elements between consecutive KV rows of one head
     int64_t kv_head_stride;       // elements between KV heads
     int64_t kv_pos_head_stride;   // ints between heads in kv_pos (0 = shared)
@@ -86,6 +87,7 @@ struct PrefillParams {
     float scale;
     int32_t causal;
     int32_t sync;                 // 0 local, 1 sync
+    int32_t remote_only;          // sync: a row sees the aggregated rows positioned before its segment
     int32_t kv_head_major;
     const int32_t *kv_pos;        // nullable
     int32_t n_seg;
@@ -93,6 +95,10 @@ struct PrefillParams {
 };
 bool prefill_sm100_supported(const Context *ctx);
 cudaError_t launch_prefill_sm100(const Context *ctx, const PrefillParams &p, cudaStream_t s, int64_t *launches);
+
+// ---- merge of two partial attention results through their log-sum-exps ----------------------
+cudaError_t launch_merge(int dtype, int64_t n_rows, int hq, int d, const void *o_a, const float *lse_a, const void *o_b,
+                         const float *lse_b, void *o, float *lse, cudaStream_t s, int64_t *launches);
 
 // ---- bf16 split-KV decode (tensor-core scores, warp-shuffle softmax) ---------------------------
 struct DecodeParams {

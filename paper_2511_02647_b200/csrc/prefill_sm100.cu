@@ -320,6 +320,10 @@ __device__ __forceinline__ int prefix_len(const PrefillParams &p, const Item &it
         return p.causal ? min(pos - p.cu[it.seg] + 1, seg_len) : seg_len;
     }
     if (!p.causal) return T;
+    if (p.remote_only) {                               // what lies before the row's own segment
+        const int before = p.cu[it.seg];
+        return it.kvp ? count_le(it.kvp, T, before - 1) : min(before, T);
+    }
     if (!it.kvp) return min(pos + 1, T);
     return count_le(it.kvp, T, pos);
 }

@@ -96,6 +96,23 @@ class Runner:
         assert self.poll() == 0
         return host(o), (host(lse) if want_lse else None)
 
+    def sync_exchange(self, q, k, v, seqlens, agg):
+        """Sync block with sparse KV exchange: local + remote-only sync + merge.  agg: dict from
+        aggregate() (head-major sparse KV).  Returns (o, lse) as numpy float64."""
+        m = self.m
+        cu = np.concatenate([[0], np.cumsum(seqlens)]).astype(np.int64)
+        qd, kd, vd = dev(q, self.dtype), dev(k, self.dtype), dev(v, self.dtype)
+        L = q.shape[0]
+        o_a = torch.full_like(qd, float("nan")); o_b = torch.full_like(qd, float("nan"))
+        lse_a = torch.full((L, self.hq), float("nan"), device="cuda"); lse_b = torch.full_like(lse_a, float("nan"))
+        o = torch.full_like(qd, float("nan")); lse = torch.full_like(lse_a, float("nan"))
+        T = agg["k_agg"].shape[1]
+        m.fedattn_local(self.ctx, self.shape, qd, kd, vd, cu, o_a, lse_a)
+        m.fedattn_sync_remote(self.ctx, self.shape, qd, cu, agg["k_agg"], agg["v_agg"], agg["kv_pos"], T, True, o_b, lse_b)
+        m.fedattn_merge(self.ctx, self.shape, L, o_a, lse_a, o_b, lse_b, o, lse)
+        assert self.poll() == 0
+        return host(o), host(lse)
+
     def decode(self, q, k_cache, v_cache, kv_len, sync_mode, max_kv_len=None):
         m = self.m
         qd, kd, vd = dev(q, self.dtype), dev(k_cache, self.dtype), dev(v_cache, self.dtype)

@@ -213,6 +213,43 @@ def test_sparse_sync_small_incl_empty_rows_and_excluded_participant(oracle, dtyp
 
 
 # ---------------------------------------------------------------------------------------------
+# sync block with sparse KV exchange: own segment complete + sparsified remote keys
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("dtype,hq,hkv,d", [("bf16", 8, 2, 128), ("f32", 4, 2, 64)])
+def test_sync_exchange_small(oracle, dtype, hq, hkv, d):
+    lens = [140, 90, 260, 33]
+    q, k, v = gen(41, lens, hq, hkv, d, dtype)
+    kp, vp = split(k, lens), split(v, lens)
+    r = Runner(len(lens), hq, hkv, d, dtype, sum(lens))
+    for ksel in ([35, 23, 65, 8], [140, 90, 260, 33], [0, 0, 0, 0], [0, 90, 0, 5]):
+        agg = r.aggregate(fa().AGG_TOPK_KNORM, kp, vp, ksel)
+        ka, va, pos, cu, sel = oracle.aggregate_topk(kp, vp, ksel)
+        assert np.array_equal(agg["sel_idx"].cpu().numpy(), sel)
+        o, lse = r.sync_exchange(q, k, v, lens, agg)
+        oo, ol = oracle.sync_exchange(q, k, v, lens, ka, va, pos, cu)
+        check_close(o, oo, TOL[dtype], "sync exchange %s" % ksel)
+        check_close(lse, ol, 1e-3, "sync exchange lse %s" % ksel)
+
+
+def test_cfg4_sync_exchange_full_size_sampled(oracle):
+    w = fi.cfg4()
+    q, k, v = w.qkv()
+    lens = list(w.seqlens)
+    kp, vp = split(k, lens), split(v, lens)
+    ksel = [w.k_sel] * len(lens)
+    r = Runner(len(lens), w.n_q_heads, w.n_kv_heads, w.head_dim, "bf16", w.total_tokens)
+    agg = r.aggregate(fa().AGG_TOPK_KNORM, kp, vp, ksel)
+    ka, va, pos, cu, sel = oracle.aggregate_topk(kp, vp, ksel)
+    assert np.array_equal(agg["sel_idx"].cpu().numpy(), sel)
+    rows = fi.sample_rows(w.seed, lens, 96)
+    o, lse = r.sync_exchange(q, k, v, lens, agg)
+    oo, ol = oracle.sync_exchange(q, k, v, lens, ka, va, pos, cu, rows=rows)
+    e = check_close(o[rows], oo, TOL["bf16"], "cfg4 sync exchange")
+    check_close(lse[rows], ol, 1e-3, "cfg4 sync exchange lse")
+    assert e / np.abs(oo).max() < 0.05
+
+
+# ---------------------------------------------------------------------------------------------
 # decode
 # ---------------------------------------------------------------------------------------------
 @pytest.mark.parametrize("dtype,d", [("bf16", 128), ("f32", 64), ("bf16", 64)])
