@@ -145,6 +145,27 @@ def flops_decode(w):
 
 
 # ------------------------------------------------------------------------------------------------
+# multi-rank bookkeeping (replicas only: no data-path collective; the ranks only agree on the time)
+# ------------------------------------------------------------------------------------------------
+def max_over_ranks(values, device=None):
+    """Element-wise maximum of a list of floats over all ranks of the default process group
+    (device: where the reduction tensor lives, None for CPU / gloo); identity without a group."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return [float(x) for x in values]
+    t = torch.tensor([float(x) for x in values], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t.tolist()]
+
+
+def replica_throughput(work_per_rank, ms_per_step, world):
+    """Whole-job units per second when `world` independent replicas each do work_per_rank per step
+    and the slowest one needs ms_per_step."""
+    return world * work_per_rank / (ms_per_step * 1e-3)
+
+
+# ------------------------------------------------------------------------------------------------
 # our arm
 # ------------------------------------------------------------------------------------------------
 def run_ours(args):
@@ -302,14 +323,11 @@ def run_ours(args):
     barrier()
     e2e_ms = e0.elapsed_time(e1) / e2e_steps
 
-    # ---- max over ranks ----
-    if world > 1:
-        t = torch.tensor([total_ms, e2e_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms, e2e_ms = float(t[0]), float(t[1])
+    # ---- max over ranks; replicas: every rank did the same work, the job did `world` times as much ----
+    total_ms, e2e_ms = max_over_ranks([total_ms, e2e_ms], dev if world > 1 else None)
     ms_per_step = total_ms / K
-    value = world * step_flops / (ms_per_step * 1e-3) / 1e12
-    e2e_value = world * step_flops / (e2e_ms * 1e-3) / 1e12
+    value = replica_throughput(step_flops, ms_per_step, world) / 1e12
+    e2e_value = replica_throughput(step_flops, e2e_ms, world) / 1e12
 
     if rank == 0:
         pk = peaks()

@@ -141,6 +141,20 @@ def is_sync_block(m: int, H: int) -> bool:
     return m % H == 0
 
 
+def sync_blocks_of_rounds(local_forwards) -> List[int]:
+    """Sync blocks (1-based) of a schedule given as the number of local forwards H_t of every
+    communication round t: round t ends with a sync block, so the sync blocks are the running sums
+    H_0, H_0 + H_1, ...  A constant H_t = H gives the uniform schedule `m mod H == 0`."""
+    blocks, m = [], 0
+    for h in local_forwards:
+        h = int(h)
+        if h <= 0:
+            raise ValueError("every round needs at least one block")
+        m += h
+        blocks.append(m)
+    return blocks
+
+
 def sample_rows(seed: int, seqlens, n_random: int, tile: int = 128) -> np.ndarray:
     """Row subset for sampled parity at full size: every row within +-1 of a segment
     start/end or of a multiple of ``tile`` (both in packed and in segment-relative

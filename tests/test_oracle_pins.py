@@ -450,6 +450,18 @@ def test_block_schedule_matches_printed_marginal_savings():
     assert fi.is_sync_block(32, 32) and not fi.is_sync_block(31, 32)
 
 
+def test_variable_round_schedule_reduces_to_uniform():
+    """Theorem 3's setting: H_t local forwards in round t, sum H_t = M; the uniform case is H_t = H."""
+    M = 32
+    for H in (1, 2, 4, 8, 32):
+        assert fi.sync_blocks_of_rounds([H] * (M // H)) == [m for m in range(1, M + 1) if fi.is_sync_block(m, H)]
+    assert fi.sync_blocks_of_rounds([2, 6, 10, 14]) == [2, 8, 18, 32]        # intervals growing with depth
+    assert sum([14, 10, 6, 2]) == M and fi.sync_blocks_of_rounds([14, 10, 6, 2])[-1] == M
+    with pytest.raises(ValueError):
+        fi.sync_blocks_of_rounds([4, 0, 4])
+
+
+
 def test_input_generators_are_seeded_and_typed():
     w = fi.cfg2()
     a = fi.normal(2, fi.TENSOR_Q, 0, (4, 3), "bf16")
