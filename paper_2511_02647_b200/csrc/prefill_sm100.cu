@@ -63,6 +63,7 @@ struct KernelParams {
     PrefillParams p;
     int32_t ord_seg[kMaxP];          // segments sorted by query-tile count, descending
     int32_t ord_nt[kMaxP];           // their query-tile counts
+    int32_t band_rank[kMaxP + 1];    // tiles ranked above band b (levels ord_nt[b+1] < lv <= ord_nt[b])
     int32_t n_qtiles;                // total query tiles
     int32_t n_items;                 // query tiles x KV heads x head pairs
     int32_t *status;
@@ -343,18 +344,15 @@ __device__ __forceinline__ Item decode_item(const KernelParams &kp, int item)
     it.valid1 = 2 * pair + 1 < g;
     // Heavy tiles first: query tiles are ranked by their index inside their segment, descending
     // (a causal tile's KV-tile count is that index + 1).  Level lv holds tile lv-1 of every segment
-    // that has at least lv tiles; above(lv) = number of tiles on higher levels.
-    auto above = [&](int lv) {
-        int a = 0;
-        for (int i = 0; i < p.n_seg && kp.ord_nt[i] > lv; ++i) a += kp.ord_nt[i] - lv;
-        return a;
-    };
-    int lo = 1, hi = kp.ord_nt[0];                              // largest lv with above(lv) <= tile_rank ... search
-    while (lo < hi) {                                           // smallest lv with above(lv) <= tile_rank
-        const int mid = (lo + hi) >> 1;
-        if (above(mid) <= tile_rank) hi = mid; else lo = mid + 1;
-    }
-    const int seg = kp.ord_seg[tile_rank - above(lo)];
+    // that has at least lv tiles.  With the segments sorted by tile count (ord_nt, descending), the
+    // levels ord_nt[b+1] < lv <= ord_nt[b] form band b, in which every level holds the b+1 longest
+    // segments; band_rank[b] = number of tiles above band b (host-computed).
+    int b = 0;
+    while (b + 1 < p.n_seg && tile_rank >= kp.band_rank[b + 1]) ++b;
+    const int in_band = tile_rank - kp.band_rank[b];
+    const int down = in_band / (b + 1);                         // levels below the band's top
+    const int lo = kp.ord_nt[b] - down;
+    const int seg = kp.ord_seg[in_band - down * (b + 1)];
     it.seg = seg;
     it.q_row0 = p.cu[seg] + (lo - 1) * kTileM;
     it.n_valid = min(kTileM, p.cu[seg + 1] - it.q_row0);
@@ -680,9 +678,11 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                 }
                 continue;
             }
-            const int c_r = prefix_len(p, it, r) - kCols * hf;     // visible keys, counted from this thread's first column
-            // prefix lengths do not decrease with the row, so KV tiles below row 0's prefix are unmasked for all rows
-            const int n_full = prefix_len(p, it, 0) / kTileN;
+            const int c_row = prefix_len(p, it, r);
+            const int c_r = c_row - kCols * hf;                 // visible keys, counted from this thread's first column
+            // prefix lengths do not decrease with the row, so KV tiles below the prefix of the warp's first
+            // row are unmasked for the whole warp (the choice of code path only has to be warp-uniform)
+            const int n_full = __shfl_sync(0xffffffffu, c_row, 0) / kTileN;
             // state of the sub-tile being visited (a) and of the other one (b); swapped after every visit
             float m_a = 0.f, l_a = 0.f, m_b = 0.f, l_b = 0.f;
             const int n_visits = n_tiles * n_sub;
@@ -809,6 +809,11 @@ cudaError_t launch_prefill_sm100(const Context *ctx, const PrefillParams &p, cud
             kp.ord_nt[b - 1] = tn; kp.ord_seg[b - 1] = ts;
         }
     if (n_qtiles > 0x7fffffffLL) return cudaErrorInvalidValue;
+    kp.band_rank[0] = 0;
+    for (int b = 0; b < p.n_seg; ++b) {
+        const int64_t next = b + 1 < p.n_seg ? kp.ord_nt[b + 1] : 0;
+        kp.band_rank[b + 1] = kp.band_rank[b] + (int32_t)((kp.ord_nt[b] - next) * (b + 1));
+    }
     kp.n_qtiles = (int32_t)n_qtiles;
     const int g = p.hq / p.hkv;
     const int64_t items = n_qtiles * p.hkv * ((g + 1) / 2);
