@@ -64,6 +64,8 @@ struct KernelParams {
     int32_t ord_seg[kMaxP];          // segments sorted by query-tile count, descending
     int32_t ord_nt[kMaxP];           // their query-tile counts
     int32_t band_rank[kMaxP + 1];    // tiles ranked above band b (levels ord_nt[b+1] < lv <= ord_nt[b])
+    int32_t group;                   // query heads per KV head
+    uint64_t magic_per_tile, magic_ppg, magic_small[kMaxP];   // ceil(2^40 / d) for d = per_tile, ppg, 1..kMaxP
     int32_t n_qtiles;                // total query tiles
     int32_t n_items;                 // query tiles x KV heads x head pairs
     int32_t *status;
@@ -291,6 +293,9 @@ constexpr uint32_t kIdescBase = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3
 constexpr uint32_t kIdescQK = kIdescBase;                 // A, B K-major
 constexpr uint32_t kIdescPV = kIdescBase | (1u << 16);    // B (V) MN-major
 
+// n / d for 0 <= n < 2^28 and 1 <= d <= 4096, with magic = ceil(2^40 / d)
+__device__ __forceinline__ int fast_div(int n, uint64_t magic) { return (int)(((uint64_t)(uint32_t)n * magic) >> 40); }
+
 // number of entries of the non-decreasing array pos[0..n) that are <= x
 __device__ __forceinline__ int count_le(const int32_t *pos, int n, int x)
 {
@@ -333,12 +338,14 @@ __device__ __forceinline__ Item decode_item(const KernelParams &kp, int item)
 {
     const PrefillParams &p = kp.p;
     Item it;
-    const int g = p.hq / p.hkv;
+    // divisions by launch constants go through host-computed reciprocals (kp.magic_*): this runs once
+    // per item in every role, on the softmax threads' critical path
+    const int g = kp.group;
     const int ppg = (g + 1) >> 1;                               // head pairs per KV head
     const int per_tile = p.hkv * ppg;
-    const int tile_rank = item / per_tile;
+    const int tile_rank = fast_div(item, kp.magic_per_tile);
     const int rem = item - tile_rank * per_tile;
-    it.kvh = rem / ppg;
+    it.kvh = fast_div(rem, kp.magic_ppg);
     const int pair = rem - it.kvh * ppg;
     it.head0 = it.kvh * g + 2 * pair;
     it.valid1 = 2 * pair + 1 < g;
@@ -350,7 +357,7 @@ __device__ __forceinline__ Item decode_item(const KernelParams &kp, int item)
     int b = 0;
     while (b + 1 < p.n_seg && tile_rank >= kp.band_rank[b + 1]) ++b;
     const int in_band = tile_rank - kp.band_rank[b];
-    const int down = in_band / (b + 1);                         // levels below the band's top
+    const int down = fast_div(in_band, kp.magic_small[b]);      // in_band / (b + 1): levels below the band's top
     const int lo = kp.ord_nt[b] - down;
     const int seg = kp.ord_seg[in_band - down * (b + 1)];
     it.seg = seg;
@@ -818,8 +825,13 @@ cudaError_t launch_prefill_sm100(const Context *ctx, const PrefillParams &p, cud
     const int g = p.hq / p.hkv;
     const int64_t items = n_qtiles * p.hkv * ((g + 1) / 2);
     if (items == 0) return cudaSuccess;
-    if (items > 0x7fffffffLL) return cudaErrorInvalidValue;
+    if (items >= (1LL << 28) || (int64_t)p.hkv * ((g + 1) / 2) > 4096) return cudaErrorInvalidValue;   // fast_div range
     kp.n_items = (int32_t)items;
+    auto magic = [](int64_t d) { return (uint64_t)(((1ULL << 40) + (uint64_t)d - 1) / (uint64_t)d); };
+    kp.group = g;
+    kp.magic_per_tile = magic((int64_t)p.hkv * ((g + 1) / 2));
+    kp.magic_ppg = magic((g + 1) / 2);
+    for (int i = 0; i < kMaxP; ++i) kp.magic_small[i] = magic(i + 1);
     const int64_t blocks = items < ctx->sm_count ? items : ctx->sm_count;     // persistent: one CTA per SM
     CUtensorMap mq, mk, mv;
     if (!encode_map(ctx, &mq, p.q, p.n_q_rows, p.hq, false) ||
