@@ -348,6 +348,8 @@ decode_split_kernel(const DecodeParams p, int n_splits, int n_chunks)
     float *sm_l = sm_m + 4 * 16 * kMTiles;
     float *cta_part = reinterpret_cast<float *>(smem + kCtaPartOffset);   // [16 kMTiles rows][kPartialStride]
     constexpr int kRows = 16 * kMTiles;
+    // only the rows that carry a query take part (LOCAL mode stacks g rows into a 16-row tile)
+    const int rows_here = min(kRows, rows_total - chunk * kRows);
     if ((lane & 3) == 0) {
 #pragma unroll
         for (int im = 0; im < kMTiles; ++im) {
@@ -370,14 +372,19 @@ decode_split_kernel(const DecodeParams p, int n_splits, int n_chunks)
         if ((lane & 3) == 0) { sm_l[slice * kRows + ra] = la * fa; sm_l[slice * kRows + rb] = lb * fb; }
         float *w0 = red + ((size_t)slice * kRows + ra) * kPartialStride + 4 + (lane & 3) * 2;
         float *w1 = w0 + 8 * kPartialStride;
+        if (ra < rows_here) {
 #pragma unroll
-        for (int i = 0; i < 16; ++i) {
-            *reinterpret_cast<float2 *>(w0 + i * 8) = make_float2(acc[im][i][0] * fa, acc[im][i][1] * fa);
-            *reinterpret_cast<float2 *>(w1 + i * 8) = make_float2(acc[im][i][2] * fb, acc[im][i][3] * fb);
+            for (int i = 0; i < 16; ++i)
+                *reinterpret_cast<float2 *>(w0 + i * 8) = make_float2(acc[im][i][0] * fa, acc[im][i][1] * fa);
+        }
+        if (rb < rows_here) {
+#pragma unroll
+            for (int i = 0; i < 16; ++i)
+                *reinterpret_cast<float2 *>(w1 + i * 8) = make_float2(acc[im][i][2] * fb, acc[im][i][3] * fb);
         }
     }
     __syncthreads();
-    for (int i = tid; i < kRows * (kD / 4); i += 128) {
+    for (int i = tid; i < rows_here * (kD / 4); i += 128) {
         const int rr = i / (kD / 4), c4 = i - rr * (kD / 4);
         float4 a = *reinterpret_cast<const float4 *>(red + (size_t)rr * kPartialStride + 4 + c4 * 4);
 #pragma unroll
