@@ -153,15 +153,18 @@ __device__ long long g_dtrace[1024 * 8];
 #endif
 
 // grid: x = split, y = KV head, z = cache * n_chunks + chunk   (cache = participant for LOCAL, 0 for SYNC)
-// block: 128 threads.  Warp w takes key slice w (16 keys of every 64-key tile) for all kMTiles
-// 16-row M-tiles of the chunk, so each K/V fragment is read from shared memory once.
+// block: 128 threads = 4 warps over (key slice, M-tile).  kMTiles == 1: 4 key slices of 16 keys of
+// every 64-key tile.  kMTiles == 2: 2 key slices of 32 keys x the 2 M-tiles, one M-tile per warp, so
+// the slice merge at the end moves half as much (K/V fragments are read by two warps instead).
 template <int kMTiles>
 __global__ void __launch_bounds__(128, 2)
 decode_split_kernel(const DecodeParams p, int n_splits, int n_chunks)
 {
+    constexpr int kSlices = 4 / kMTiles;                        // key slices per tile
+    constexpr int kSteps = 4 / kSlices;                         // 16-key steps per warp and tile
     extern __shared__ __align__(1024) uint8_t smem[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int slice = warp;
+    const int slice = warp % kSlices, mt = warp / kSlices;     // this warp's key slice and M-tile
     DTRACE(0);
     const int split = blockIdx.x, kvh = blockIdx.y;
     const int cache = blockIdx.z / n_chunks, chunk = blockIdx.z - cache * n_chunks;
@@ -210,14 +213,10 @@ decode_split_kernel(const DecodeParams p, int n_splits, int n_chunks)
     };
 
     const float sl2 = p.scale * 1.4426950408889634f;
-    float m0[kMTiles], m1[kMTiles], l0[kMTiles], l1[kMTiles];  // rows lane/4 and lane/4 + 8 of each M-tile
-    float acc[kMTiles][16][4];
+    float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;   // rows lane/4 and lane/4 + 8 of this warp's M-tile
+    float acc[16][4];
 #pragma unroll
-    for (int im = 0; im < kMTiles; ++im) {
-        m0[im] = m1[im] = -INFINITY; l0[im] = l1[im] = 0.f;
-#pragma unroll
-        for (int i = 0; i < 16; ++i) acc[im][i][0] = acc[im][i][1] = acc[im][i][2] = acc[im][i][3] = 0.f;
-    }
+    for (int i = 0; i < 16; ++i) acc[i][0] = acc[i][1] = acc[i][2] = acc[i][3] = 0.f;
 
     // Q rows of this chunk -> shared memory (in the third stage's buffer, which the first tile loads do
     // not touch), same swizzle as the K/V tiles; rows past rows_total are zero
@@ -236,21 +235,19 @@ decode_split_kernel(const DecodeParams p, int n_splits, int n_chunks)
         if (s < n_tiles) load_tile(s, s);
         cp_async_commit();
     }
-    // Q fragments (A operand, 16 x 128 per M-tile): 8 k-steps x 4 registers
-    uint32_t qf[kMTiles][8][4];
+    // Q fragments of this warp's M-tile (A operand, 16 x 128): 8 k-steps x 4 registers
+    uint32_t qf[8][4];
     cp_async_wait<kStages - 1>();                               // the Q group; the tile groups may still be in flight
     __syncthreads();
     {
         const uint32_t sQ = smem_u32(smem) + (kStages - 1) * kStageBytes;
 #pragma unroll
-        for (int im = 0; im < kMTiles; ++im)
-#pragma unroll
-            for (int ks = 0; ks < 8; ++ks) {
-                // matrices: (rows 0-7, d 0-7) (rows 8-15, d 0-7) (rows 0-7, d 8-15) (rows 8-15, d 8-15)
-                const int row = im * 16 + (lane & 7) + (((lane >> 3) & 1) << 3);
-                const int ch = ks * 2 + (lane >> 4);
-                ldmatrix_x4(qf[im][ks], sQ + swz(row, ch));
-            }
+        for (int ks = 0; ks < 8; ++ks) {
+            // matrices: (rows 0-7, d 0-7) (rows 8-15, d 0-7) (rows 0-7, d 8-15) (rows 8-15, d 8-15)
+            const int row = mt * 16 + (lane & 7) + (((lane >> 3) & 1) << 3);
+            const int ch = ks * 2 + (lane >> 4);
+            ldmatrix_x4(qf[ks], sQ + swz(row, ch));
+        }
     }
     DTRACE(1);
     for (int t = 0; t < n_tiles; ++t) {
@@ -261,33 +258,25 @@ decode_split_kernel(const DecodeParams p, int n_splits, int n_chunks)
         cp_async_commit();
 
         const uint32_t sK = smem_u32(smem) + (t % kStages) * kStageBytes, sV = sK + kTileBytes;
-        const int krow0 = slice * 16;
-        // ---- S = Q K^T for this warp's 16 keys: two n-tiles of 8 keys per M-tile ----
-        float s0[kMTiles][4], s1[kMTiles][4];
 #pragma unroll
-        for (int im = 0; im < kMTiles; ++im)
+        for (int step = 0; step < kSteps; ++step) {
+            const int krow0 = (slice * kSteps + step) * 16;
+            // ---- S = Q K^T for 16 keys: two n-tiles of 8 keys ----
+            float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-            for (int i = 0; i < 4; ++i) s0[im][i] = s1[im][i] = 0.f;
-#pragma unroll
-        for (int ks = 0; ks < 8; ++ks) {
-            // matrices: (keys 0-7, d 0-7) (keys 0-7, d 8-15) (keys 8-15, d 0-7) (keys 8-15, d 8-15)
-            const int row = krow0 + (lane & 7) + ((lane >> 4) << 3);
-            const int ch = ks * 2 + ((lane >> 3) & 1);
-            uint32_t b[4];
-            ldmatrix_x4(b, sK + swz(row, ch));
-#pragma unroll
-            for (int im = 0; im < kMTiles; ++im) {
-                mma_bf16(s0[im], qf[im][ks], b[0], b[1]);
-                mma_bf16(s1[im], qf[im][ks], b[2], b[3]);
+            for (int ks = 0; ks < 8; ++ks) {
+                // matrices: (keys 0-7, d 0-7) (keys 0-7, d 8-15) (keys 8-15, d 0-7) (keys 8-15, d 8-15)
+                const int row = krow0 + (lane & 7) + ((lane >> 4) << 3);
+                const int ch = ks * 2 + ((lane >> 3) & 1);
+                uint32_t b[4];
+                ldmatrix_x4(b, sK + swz(row, ch));
+                mma_bf16(s0, qf[ks], b[0], b[1]);
+                mma_bf16(s1, qf[ks], b[2], b[3]);
             }
-        }
-        // ---- mask keys past the end, online softmax (rows lane/4 and lane/4+8) ----
-        const int key = (tile_lo + t) * kTileKeys + krow0 + (lane & 3) * 2;
-        const bool ok[4] = {key < len, key + 1 < len, key + 8 < len, key + 9 < len};
-        uint32_t pf[kMTiles][4];
-#pragma unroll
-        for (int im = 0; im < kMTiles; ++im) {
-            float v[8] = {s0[im][0], s0[im][1], s1[im][0], s1[im][1], s0[im][2], s0[im][3], s1[im][2], s1[im][3]};
+            // ---- mask keys past the end, online softmax (rows lane/4 and lane/4+8) ----
+            const int key = (tile_lo + t) * kTileKeys + krow0 + (lane & 3) * 2;
+            const bool ok[4] = {key < len, key + 1 < len, key + 8 < len, key + 9 < len};
+            float v[8] = {s0[0], s0[1], s1[0], s1[1], s0[2], s0[3], s1[2], s1[3]};   // row0: v[0..3], row1: v[4..7]
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 v[i] = ok[i] ? v[i] * sl2 : -INFINITY;
@@ -299,39 +288,35 @@ decode_split_kernel(const DecodeParams p, int n_splits, int n_chunks)
             // The exponent reference of a row moves only when its maximum grew by more than 2^8 (or is
             // still unset); the accumulators are rescaled only then.  The final normalisation uses the
             // same reference, so the result is exact up to rounding.
-            const bool g0 = mx0 > m0[im] + kRescaleThreshold, g1 = mx1 > m1[im] + kRescaleThreshold;
+            const bool g0 = mx0 > m0 + kRescaleThreshold, g1 = mx1 > m1 + kRescaleThreshold;
             if (__any_sync(0xffffffffu, g0 || g1)) {
-                const float mn0 = g0 ? mx0 : m0[im], mn1 = g1 ? mx1 : m1[im];
-                const float a0 = g0 ? ex2(m0[im] - mn0) : 1.f, a1 = g1 ? ex2(m1[im] - mn1) : 1.f;
-                m0[im] = mn0; m1[im] = mn1;
-                l0[im] *= a0; l1[im] *= a1;
+                const float mn0 = g0 ? mx0 : m0, mn1 = g1 ? mx1 : m1;
+                const float a0 = g0 ? ex2(m0 - mn0) : 1.f, a1 = g1 ? ex2(m1 - mn1) : 1.f;
+                m0 = mn0; m1 = mn1;
+                l0 *= a0; l1 *= a1;
 #pragma unroll
-                for (int i = 0; i < 16; ++i) { acc[im][i][0] *= a0; acc[im][i][1] *= a0; acc[im][i][2] *= a1; acc[im][i][3] *= a1; }
+                for (int i = 0; i < 16; ++i) { acc[i][0] *= a0; acc[i][1] *= a0; acc[i][2] *= a1; acc[i][3] *= a1; }
             }
-            const float ms0 = m0[im] == -INFINITY ? 0.f : m0[im], ms1 = m1[im] == -INFINITY ? 0.f : m1[im];
+            const float ms0 = m0 == -INFINITY ? 0.f : m0, ms1 = m1 == -INFINITY ? 0.f : m1;
             float ps0 = 0.f, ps1 = 0.f;
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 v[i] = ex2(v[i] - ms0); ps0 += v[i];
                 v[i + 4] = ex2(v[i + 4] - ms1); ps1 += v[i + 4];
             }
-            l0[im] += ps0; l1[im] += ps1;
+            l0 += ps0; l1 += ps1;
             // P as A operand (16 rows x 16 keys)
-            pf[im][0] = pack_bf16(v[0], v[1]); pf[im][1] = pack_bf16(v[4], v[5]);
-            pf[im][2] = pack_bf16(v[2], v[3]); pf[im][3] = pack_bf16(v[6], v[7]);
-        }
-        // ---- O += P V ----
+            const uint32_t pf[4] = {pack_bf16(v[0], v[1]), pack_bf16(v[4], v[5]), pack_bf16(v[2], v[3]), pack_bf16(v[6], v[7])};
+            // ---- O += P V ----
 #pragma unroll
-        for (int nd = 0; nd < 8; ++nd) {
-            // matrices: (keys 0-7, d 0-7) (keys 8-15, d 0-7) (keys 0-7, d 8-15) (keys 8-15, d 8-15) of d block nd*16
-            const int row = krow0 + (lane & 7) + (((lane >> 3) & 1) << 3);
-            const int ch = nd * 2 + (lane >> 4);
-            uint32_t b[4];
-            ldmatrix_x4_trans(b, sV + swz(row, ch));
-#pragma unroll
-            for (int im = 0; im < kMTiles; ++im) {
-                mma_bf16(acc[im][2 * nd], pf[im], b[0], b[1]);
-                mma_bf16(acc[im][2 * nd + 1], pf[im], b[2], b[3]);
+            for (int nd = 0; nd < 8; ++nd) {
+                // matrices: (keys 0-7, d 0-7) (keys 8-15, d 0-7) (keys 0-7, d 8-15) (keys 8-15, d 8-15) of d block nd*16
+                const int row = krow0 + (lane & 7) + (((lane >> 3) & 1) << 3);
+                const int ch = nd * 2 + (lane >> 4);
+                uint32_t b[4];
+                ldmatrix_x4_trans(b, sV + swz(row, ch));
+                mma_bf16(acc[2 * nd], pf, b[0], b[1]);
+                mma_bf16(acc[2 * nd + 1], pf, b[2], b[3]);
             }
         }
     }
@@ -339,7 +324,7 @@ decode_split_kernel(const DecodeParams p, int n_splits, int n_chunks)
     __syncthreads();
     DTRACE(3);
 
-    // ---- merge the four key slices (warps) into this CTA's partial, kept in shared memory ----
+    // ---- merge the key slices (warps) into this CTA's partial, kept in shared memory ----
     // 1. every warp posts the exponent references of its rows; 2. every thread rescales its own
     // accumulators to the common reference of its rows (in registers) and posts them; 3. the slices
     // are summed with 16-byte reads.
@@ -350,23 +335,19 @@ decode_split_kernel(const DecodeParams p, int n_splits, int n_chunks)
     constexpr int kRows = 16 * kMTiles;
     // only the rows that carry a query take part (LOCAL mode stacks g rows into a 16-row tile)
     const int rows_here = min(kRows, rows_total - chunk * kRows);
+    const int ra = mt * 16 + (lane >> 2), rb = ra + 8;          // this thread's rows inside the CTA
     if ((lane & 3) == 0) {
-#pragma unroll
-        for (int im = 0; im < kMTiles; ++im) {
-            sm_m[slice * kRows + im * 16 + (lane >> 2)] = m0[im];
-            sm_m[slice * kRows + im * 16 + (lane >> 2) + 8] = m1[im];
-        }
+        sm_m[slice * kRows + ra] = m0;
+        sm_m[slice * kRows + rb] = m1;
     }
     __syncthreads();
-#pragma unroll
-    for (int im = 0; im < kMTiles; ++im) {
-        const int ra = im * 16 + (lane >> 2), rb = ra + 8;
+    {
         float ma = -INFINITY, mb = -INFINITY;
 #pragma unroll
-        for (int sl = 0; sl < 4; ++sl) { ma = fmaxf(ma, sm_m[sl * kRows + ra]); mb = fmaxf(mb, sm_m[sl * kRows + rb]); }
-        const float fa = ex2(m0[im] - (ma == -INFINITY ? 0.f : ma)), fb = ex2(m1[im] - (mb == -INFINITY ? 0.f : mb));
+        for (int sl = 0; sl < kSlices; ++sl) { ma = fmaxf(ma, sm_m[sl * kRows + ra]); mb = fmaxf(mb, sm_m[sl * kRows + rb]); }
+        const float fa = ex2(m0 - (ma == -INFINITY ? 0.f : ma)), fb = ex2(m1 - (mb == -INFINITY ? 0.f : mb));
         // quad-reduce l (each lane of a quad summed different keys)
-        float la = l0[im], lb = l1[im];
+        float la = l0, lb = l1;
         la += __shfl_xor_sync(0xffffffffu, la, 1); la += __shfl_xor_sync(0xffffffffu, la, 2);
         lb += __shfl_xor_sync(0xffffffffu, lb, 1); lb += __shfl_xor_sync(0xffffffffu, lb, 2);
         if ((lane & 3) == 0) { sm_l[slice * kRows + ra] = la * fa; sm_l[slice * kRows + rb] = lb * fb; }
@@ -375,12 +356,12 @@ decode_split_kernel(const DecodeParams p, int n_splits, int n_chunks)
         if (ra < rows_here) {
 #pragma unroll
             for (int i = 0; i < 16; ++i)
-                *reinterpret_cast<float2 *>(w0 + i * 8) = make_float2(acc[im][i][0] * fa, acc[im][i][1] * fa);
+                *reinterpret_cast<float2 *>(w0 + i * 8) = make_float2(acc[i][0] * fa, acc[i][1] * fa);
         }
         if (rb < rows_here) {
 #pragma unroll
             for (int i = 0; i < 16; ++i)
-                *reinterpret_cast<float2 *>(w1 + i * 8) = make_float2(acc[im][i][2] * fb, acc[im][i][3] * fb);
+                *reinterpret_cast<float2 *>(w1 + i * 8) = make_float2(acc[i][2] * fb, acc[i][3] * fb);
         }
     }
     __syncthreads();
@@ -388,7 +369,7 @@ decode_split_kernel(const DecodeParams p, int n_splits, int n_chunks)
         const int rr = i / (kD / 4), c4 = i - rr * (kD / 4);
         float4 a = *reinterpret_cast<const float4 *>(red + (size_t)rr * kPartialStride + 4 + c4 * 4);
 #pragma unroll
-        for (int sl = 1; sl < 4; ++sl) {
+        for (int sl = 1; sl < kSlices; ++sl) {
             const float4 v = *reinterpret_cast<const float4 *>(red + ((size_t)sl * kRows + rr) * kPartialStride + 4 + c4 * 4);
             a.x += v.x; a.y += v.y; a.z += v.z; a.w += v.w;
         }
@@ -397,7 +378,7 @@ decode_split_kernel(const DecodeParams p, int n_splits, int n_chunks)
         if (c4 == 0) {
             float mm = -INFINITY, ll = 0.f;
 #pragma unroll
-            for (int sl = 0; sl < 4; ++sl) { mm = fmaxf(mm, sm_m[sl * kRows + rr]); ll += sm_l[sl * kRows + rr]; }
+            for (int sl = 0; sl < kSlices; ++sl) { mm = fmaxf(mm, sm_m[sl * kRows + rr]); ll += sm_l[sl * kRows + rr]; }
             dst[0] = mm; dst[1] = ll;
         }
     }
