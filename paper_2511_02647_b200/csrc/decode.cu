@@ -437,18 +437,23 @@ decode_split_kernel(const DecodeParams p, int n_splits, int n_chunks)
             if (c4 == 0) { dst[0] = mm; dst[1] = ll; }
         }
     }
-    cluster.sync();                                             // peers are done reading this CTA's partial
+    // This CTA is done reading its peers; it may not exit before they are done reading it.  Arrive now,
+    // wait at the very end: what follows does not touch distributed shared memory.
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
     DTRACE(5);
-    if (ncl == 1 || my_rows == 0) return;
 
     // ---- several clusters per (cache, KV head): the last to arrive for these rows merges them ----
     __shared__ int s_flag;
-    const int source = blockIdx.z * gridDim.y + kvh;
-    const bool last = arrive_last(p.counters + source * kMaxCluster + rank, ncl, &s_flag);
-    DTRACE(6);
-    if (!last) return;
-    merge_slots<128>(p, ncl, cache, kvh, row0 + rank, cs, my_rows);
-    DTRACE(7);
+    if (ncl > 1 && my_rows > 0) {                               // CTA-uniform
+        const int source = blockIdx.z * gridDim.y + kvh;
+        const bool last = arrive_last(p.counters + source * kMaxCluster + rank, ncl, &s_flag);
+        DTRACE(6);
+        if (last) {
+            merge_slots<128>(p, ncl, cache, kvh, row0 + rank, cs, my_rows);
+            DTRACE(7);
+        }
+    }
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
 #ifdef FEDATTN_DTRACE
