@@ -114,6 +114,7 @@ struct DecodeParams {
     float *partial;               // scratch: per-split partial results
     size_t partial_bytes;
     int32_t *counters;            // kDecodeCounters arrival counters, all zero between calls
+    int32_t g_shift;              // log2(hq / hkv) when that is a power of two, else -1 (set by the launcher)
 };
 size_t decode_scratch_bytes(int n_part, int hq, int d, int sm_count);
 cudaError_t launch_decode_bf16(const Context *ctx, const DecodeParams &p, cudaStream_t s, int64_t *launches);

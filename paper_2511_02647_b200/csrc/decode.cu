@@ -187,8 +187,12 @@ decode_split_kernel(const DecodeParams p, int n_splits, int n_chunks)
     // stacked row -> (participant, query head)
     auto q_ptr = [&](int srow) -> const __nv_bfloat16 * {
         if (srow >= rows_total) return nullptr;
-        const int part = p.sync ? srow / g : cache;
-        const int head = kvh * g + (p.sync ? srow % g : srow);
+        int part = cache, sub = srow;
+        if (p.sync) {                                           // srow = part * g + sub
+            if (p.g_shift >= 0) { part = srow >> p.g_shift; sub = srow & (g - 1); }
+            else { part = srow / g; sub = srow - part * g; }
+        }
+        const int head = kvh * g + sub;
         return reinterpret_cast<const __nv_bfloat16 *>(p.q) + ((size_t)part * p.hq + head) * kD;
     };
 
@@ -472,10 +476,14 @@ size_t decode_scratch_bytes(int n_part, int hq, int d, int /*sm_count*/)
 // Grid rule shared by both entry points.  Splits are chosen so that the whole grid is resident at
 // once (two CTAs per SM): a grid slightly larger than that would run a nearly empty second wave.
 // The splits of one (cache, KV head) form clusters of cs = 1, 2, 4 or 8 CTAs along grid.x.
-static cudaError_t launch_decode_split(const DecodeParams &p, int sm_count, int max_slots, cudaStream_t s,
+static cudaError_t launch_decode_split(const DecodeParams &p_in, int sm_count, int max_slots, cudaStream_t s,
                                        int64_t *launches)
 {
+    DecodeParams p = p_in;
     const int g = p.hq / p.hkv;
+    p.g_shift = -1;
+    for (int sh = 0; sh < 16; ++sh)
+        if ((1 << sh) == g) p.g_shift = sh;
     const int rows_total = p.sync ? p.n_part * g : g;
     const int m_tiles = rows_total > 16 ? 2 : 1;
     const int n_chunks = (rows_total + 16 * m_tiles - 1) / (16 * m_tiles);
