@@ -45,7 +45,11 @@ constexpr int kD = 128;              // head dim
 constexpr int kSplit = 2;
 constexpr int kCols = kTileN / kSplit;
 constexpr int kSoftmaxThreads = 128 * kSplit;
-constexpr int kThreads = kSoftmaxThreads + 64;   // then one TMA producer warp and one MMA issuer warp
+constexpr int kThreads = kSoftmaxThreads + 128;  // then a warpgroup holding the TMA producer warp and the MMA issuer warp
+// Registers move from that warpgroup to the softmax warpgroups once the roles split (setmaxnreg):
+// 384 threads start with 168 each; afterwards 2 x 128 x kSoftmaxRegs + 128 x kOtherRegs <= 64 K.
+constexpr int kSoftmaxRegs = 216, kOtherRegs = 64;
+static_assert(kSoftmaxThreads * kSoftmaxRegs + 128 * kOtherRegs <= 65536, "register budget");
 constexpr int kProducerWarp = 4 * kSplit, kMmaWarp = 4 * kSplit + 1;
 static_assert(kSplit == 2 || kSplit == 4, "column split");
 constexpr uint32_t kTileBytes = kTileM * kD * 2;      // 32 KB: one Q, K or V tile
@@ -424,7 +428,10 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
+    // every warp of a warpgroup executes the same setmaxnreg (first thing in its role); the increase
+    // waits for the decrease
     if (warp == kProducerWarp) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kOtherRegs));
         // ================= TMA producer =================
         if (lane == 0) {
             asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&map_q) : "memory");
@@ -472,6 +479,7 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             }
         }
     } else if (warp == kMmaWarp) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kOtherRegs));
         // ================= MMA issuer =================
         // Issue order per item  S0(0) S1(0) | PV0(0) S0(1) | PV1(0) S1(1) | PV0(1) S0(2) | ...  : while one
         // sub-tile's softmax runs, the tensor pipe works on the other sub-tile.
@@ -551,7 +559,10 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             ++qn;
             if (it.valid1) { git1 += n; ++qn1; }
         }
+    } else if (warp >= 4 * kSplit) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kOtherRegs));      // the two idle warps of that warpgroup
     } else {
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kSoftmaxRegs));
         // ================= softmax + epilogue =================
         // All softmax warpgroups work on the same S tile: thread = (query row r = TMEM lane, column part hf).
         // Warpgroup hf owns keys kCols hf .. kCols hf + kCols - 1 of every S tile and the same head-dim
