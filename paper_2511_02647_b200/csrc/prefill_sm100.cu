@@ -20,7 +20,9 @@
 // Warp roles: warps 0-7 softmax/epilogue.  Both warpgroups work on the same S tile, split by
 // columns: thread = (query row = TMEM lane, column half); the halves of a row exchange their
 // maxima through shared memory once per tile.  Warp 8 TMA producer (+ TMEM allocation), warp 9
-// MMA issuer (the whole warp walks the loop, one elected lane issues).  3/8 of the exponentials
+// MMA issuer (the whole warp walks the loop, one elected lane issues); warps 10-11 only fill that
+// warpgroup, which hands most of its registers to the softmax warpgroups (setmaxnreg works on whole
+// warpgroups).  3/8 of the exponentials
 // of unmasked tiles are evaluated by a polynomial on the FMA pipe, because for this tile shape the
 // ex2 unit is exactly as slow as the tensor pipe.  Every wait is bounded; on expiry the CTA sets
 // the status word, stops waiting and runs to its normal end (TMEM is always released).
