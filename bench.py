@@ -54,10 +54,10 @@ N_SETS = 3            # rotating input sets: ~600 MB touched per cycle, larger t
 SPARSE_RATIO_NUM, SPARSE_RATIO_DEN = 1, 4
 # dram__bytes_read.sum + dram__bytes_write.sum per prefill launch of the sync call at this
 # workload, from the ncu capture summarised under profiles/ (None until captured)
-PREFILL_SYNC_DRAM_BYTES = 134_893_568
+PREFILL_SYNC_DRAM_BYTES = 135_579_904
 # the same for one decode call (cfg5) and for one sparse aggregation (cfg4)
-DECODE_DRAM_BYTES = 139_544_000     # mean of the local (140.0 MB) and sync (138.1 MB) captures
-TOPK_DRAM_BYTES = 42_155_264
+DECODE_DRAM_BYTES = 138_348_800     # mean of the local (138.5 MB) and sync (138.2 MB) captures
+TOPK_DRAM_BYTES = 42_363_136       # mean of two captured launches
 
 
 def env_rank():
