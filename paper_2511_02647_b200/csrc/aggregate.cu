@@ -93,8 +93,9 @@ __device__ __forceinline__ double sq_acc_bf16x2(double s, uint32_t w)
 {
     const double lo = (double)__uint_as_float(w << 16);
     const double hi = (double)__uint_as_float(w & 0xffff0000u);
-    s = __dadd_rn(s, __dmul_rn(lo, lo));
-    s = __dadd_rn(s, __dmul_rn(hi, hi));
+    // x * x is exact in fp64, so the fused multiply-add rounds exactly once, like the separate add
+    s = __fma_rn(lo, lo, s);
+    s = __fma_rn(hi, hi, s);
     return s;
 }
 
@@ -190,10 +191,10 @@ topk_fused_kernel(const PartsParams pp, int hkv, int vpr /* 16-byte vectors per 
                         const uint4 u = mine[v];
                         const float x0 = __uint_as_float(u.x), x1 = __uint_as_float(u.y), x2 = __uint_as_float(u.z),
                                     x3 = __uint_as_float(u.w);
-                        sc = __dadd_rn(sc, __dmul_rn((double)x0, (double)x0));
-                        sc = __dadd_rn(sc, __dmul_rn((double)x1, (double)x1));
-                        sc = __dadd_rn(sc, __dmul_rn((double)x2, (double)x2));
-                        sc = __dadd_rn(sc, __dmul_rn((double)x3, (double)x3));
+                        sc = __fma_rn((double)x0, (double)x0, sc);
+                        sc = __fma_rn((double)x1, (double)x1, sc);
+                        sc = __fma_rn((double)x2, (double)x2, sc);
+                        sc = __fma_rn((double)x3, (double)x3, sc);
                     }
                 }
                 keys[c0 + tid] = (unsigned long long)__double_as_longlong(sc);
