@@ -639,8 +639,9 @@ def run_cfg3(args):
     M = w.n_blocks
 
     def block(m, H):
+        # H: the uniform interval, or the explicit set of sync blocks of a non-uniform schedule
         b = sets[m % n_sets]
-        if fi.is_sync_block(m, H):
+        if (m in H) if isinstance(H, frozenset) else fi.is_sync_block(m, H):
             fa.fedattn_aggregate_kv(ctx, shape, fa.AGG_CONCAT, b["kp"], b["vp"], seqlens, None, None, b["kg"], b["vg"], None, None, None)
             fa.fedattn_sync(ctx, shape, b["q"], None, b["kg"], b["vg"], None, L, False, b["o"])
         else:
@@ -662,6 +663,17 @@ def run_cfg3(args):
                          "tflops": round(fl / (ms * 1e-3) / 1e12, 2)}
     launches = (ctx.launch_count() - l0) * K // (K + W)
     time.sleep(0.25); clocks = sampler.stop()
+    # Non-uniform schedules with four exchanges each (Theorem 3: H_t local forwards in round t): exchanges
+    # in the shallow or the deep half, intervals growing or shrinking with depth.  The paper does not
+    # print its intervals; these are stand-ins of that form.
+    named = {"shallow_half": fi.sync_blocks_of_rounds([4, 4, 4, 4]), "deep_half": [20, 24, 28, 32],
+             "progressive": fi.sync_blocks_of_rounds([2, 4, 8, 18]), "regressive": fi.sync_blocks_of_rounds([18, 8, 4, 2])}
+    for name, blocks in named.items():
+        sset = frozenset(blocks)
+        ms = _timed(torch, stream, lambda i, sset=sset: [block(m, sset) for m in range(1, M + 1)], K, W)
+        fl = len(sset) * f_sync + (M - len(sset)) * f_local
+        per_h[name] = {"ms": round(ms, 4), "sync_blocks": sorted(sset), "ms_per_block": round(ms / M, 4),
+                       "tflops": round(fl / (ms * 1e-3) / 1e12, 2)}
     assert ctx.poll() == 0
 
     def e2e_step(i):                                           # one sync block through host buffers

@@ -113,6 +113,16 @@ class Runner:
         assert self.poll() == 0
         return host(o), host(lse)
 
+    def merge(self, o_a, lse_a, o_b, lse_b):
+        """LSE merge of two partial attention results over disjoint key sets (numpy in, numpy out)."""
+        oa, ob = dev(o_a.astype(np.float32), self.dtype), dev(o_b.astype(np.float32), self.dtype)
+        la = torch.from_numpy(np.ascontiguousarray(lse_a, dtype=np.float32)).cuda()
+        lb = torch.from_numpy(np.ascontiguousarray(lse_b, dtype=np.float32)).cuda()
+        o = torch.full_like(oa, float("nan")); lse = torch.full_like(la, float("nan"))
+        self.m.fedattn_merge(self.ctx, self.shape, int(o_a.shape[0]), oa, la, ob, lb, o, lse)
+        assert self.poll() == 0
+        return host(o), host(lse)
+
     def decode(self, q, k_cache, v_cache, kv_len, sync_mode, max_kv_len=None):
         m = self.m
         qd, kd, vd = dev(q, self.dtype), dev(k_cache, self.dtype), dev(v_cache, self.dtype)

@@ -250,6 +250,54 @@ def test_cfg4_sync_exchange_full_size_sampled(oracle):
 
 
 # ---------------------------------------------------------------------------------------------
+# a block in which only some participants exchange KV (adaptive aggregation): the others stay local
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("dtype,hq,hkv,d", [("bf16", 8, 2, 128), ("f32", 4, 2, 64)])
+def test_block_with_a_subset_of_participants_exchanging(oracle, dtype, hq, hkv, d):
+    lens = [130, 70, 200, 45]
+    off = np.concatenate([[0], np.cumsum(lens)])
+    q, k, v = gen(61, lens, hq, hkv, d, dtype)
+    kp, vp = split(k, lens), split(v, lens)
+    r = Runner(len(lens), hq, hkv, d, dtype, sum(lens))
+    o_loc, lse_loc = r.local(q, k, v, lens)
+    oo_loc, ol_loc = oracle.local(q, k, v, lens)
+    for members in ([0, 2], [1, 2, 3], [3]):
+        ksel = [lens[n] if n in members else 0 for n in range(len(lens))]      # members send every row
+        agg = r.aggregate(fa().AGG_TOPK_KNORM, kp, vp, ksel)
+        ka, va, pos, cu, sel = oracle.aggregate_topk(kp, vp, ksel)
+        assert np.array_equal(agg["kv_pos"].cpu().numpy(), pos) and np.array_equal(agg["cu_kv"].cpu().numpy(), cu)
+        rows = np.concatenate([np.arange(off[n], off[n + 1]) for n in members]).astype(np.int32)
+        o, lse = r.sync(q[rows], agg["k_agg"], agg["v_agg"], agg["kv_pos"], q_pos=rows, head_major=True)
+        oo, ol = oracle.sync(q[rows], ka, va, kv_pos=pos, q_pos=rows, kv_head_major=True)
+        check_close(o, oo, TOL[dtype], "subset exchange %s" % members)
+        check_close(lse, ol, 1e-3, "subset exchange lse %s" % members)
+        rest = np.setdiff1d(np.arange(sum(lens)), rows)
+        check_close(o_loc[rest], oo_loc[rest], TOL[dtype], "subset exchange, local rows %s" % members)
+    # a participant that exchanges with nobody else computes its local attention
+    n0 = np.arange(off[3], off[4])
+    check_close(o, oo_loc[n0], TOL[dtype], "lone member equals local")
+
+
+# ---------------------------------------------------------------------------------------------
+# sparse local attention: every participant keeps a seeded sample of its tokens
+# ---------------------------------------------------------------------------------------------
+def test_sparse_local_attention_on_sampled_tokens(oracle):
+    lens = [300, 129, 515]
+    hq, hkv, d = 8, 2, 128
+    q, k, v = gen(71, lens, hq, hkv, d, "bf16")
+    off = np.concatenate([[0], np.cumsum(lens)])
+    rng = np.random.default_rng(71)
+    keep = [np.sort(rng.choice(n, size=(n + 1) // 2, replace=False)) + off[i] for i, n in enumerate(lens)]
+    rows = np.concatenate(keep)
+    kept = [len(x) for x in keep]
+    r = Runner(len(lens), hq, hkv, d, "bf16", sum(lens))
+    o, lse = r.local(q[rows], k[rows], v[rows], kept)
+    oo, ol = oracle.local(q[rows], k[rows], v[rows], kept)
+    check_close(o, oo, TOL["bf16"], "sparse local")
+    check_close(lse, ol, 1e-3, "sparse local lse")
+
+
+# ---------------------------------------------------------------------------------------------
 # decode
 # ---------------------------------------------------------------------------------------------
 @pytest.mark.parametrize("dtype,d", [("bf16", 128), ("f32", 64), ("bf16", 64)])
@@ -270,6 +318,31 @@ def test_decode_small(oracle, dtype, d):
         oo, ol = oracle.decode(q, k, v, [T], True)
         check_close(o, oo, TOL[dtype], "decode sync %d" % T)
         check_close(lse, ol, 1e-3, "decode sync lse")
+
+
+@pytest.mark.parametrize("dtype,d", [("bf16", 128), ("f32", 64)])
+def test_decode_sync_block_with_private_suffix(oracle, dtype, d):
+    """Sync-block decode when every participant has generated tokens of its own after the shared
+    global cache: attention over the union = sync decode over the global cache, local decode over
+    the private suffix, merged by their log-sum-exps."""
+    n, T, cap, hq, hkv = 4, 700, 40, 8, 2
+    _, kg, vg = fi.Workload("dg", 51, (T,), hq, hkv, d, dtype).qkv()
+    ws = fi.Workload("dx", 52, (cap,) * n, hq, hkv, d, dtype)
+    _, ks, vs = ws.qkv()
+    q = ws.decode_q(0)
+    ksc, vsc = ks.reshape(n, cap, hkv, d), vs.reshape(n, cap, hkv, d)
+    r = Runner(n, hq, hkv, d, dtype, max(T, n * cap))
+    for sfx in ([40, 0, 7, 1], [0, 0, 0, 0]):
+        o_g, lse_g = r.decode(q, kg, vg, [T], True, max_kv_len=T)
+        o_s, lse_s = r.decode(q, ksc, vsc, sfx, False, max_kv_len=cap)
+        o, lse = r.merge(o_g, lse_g, o_s, lse_s)
+        cat_k = np.concatenate([np.broadcast_to(kg, (n,) + kg.shape), ksc], axis=1)
+        cat_v = np.concatenate([np.broadcast_to(vg, (n,) + vg.shape), vsc], axis=1)
+        # the suffix of participant i follows the T global rows directly only when it is read as rows
+        # T .. T + sfx[i] - 1, which is how the concatenated cache is laid out
+        oo, ol = oracle.decode(q, cat_k, cat_v, [T + s for s in sfx], False)
+        check_close(o, oo, TOL[dtype], "decode with suffix %s" % sfx)
+        check_close(lse, ol, 1e-3, "decode with suffix lse %s" % sfx)
 
 
 def test_decode_many_splits_clusters_and_row_chunks(oracle):

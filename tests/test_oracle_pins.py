@@ -462,6 +462,55 @@ def test_variable_round_schedule_reduces_to_uniform():
 
 
 
+def test_participant_subset_exchange_reduces_to_local_and_to_dense_sync(oracle):
+    """Adaptive aggregation (a participant mask per round): members send every row, the others none.
+    One member alone sees only its own keys, i.e. its local attention; all members give the dense
+    sync block; in between, a member's row sees exactly the members' keys at or before its position."""
+    lens = [5, 3, 6, 4]
+    L, Hq, Hkv, d = sum(lens), 4, 2, 4
+    off = np.concatenate([[0], np.cumsum(lens)])
+    q, k, v = randn(L, Hq, d), randn(L, Hkv, d), randn(L, Hkv, d)
+    cuts = np.cumsum(lens)[:-1]
+    ks, vs = np.split(k, cuts), np.split(v, cuts)
+    o_loc, lse_loc = oracle.local(q, k, v, lens)
+    o_den, lse_den = oracle.sync(q, k, v)
+    for members in ([2], [0, 1, 2, 3], [1, 3]):
+        ksel = [lens[n] if n in members else 0 for n in range(4)]
+        ka, va, pos, cu, sel = oracle.aggregate_topk(ks, vs, ksel)
+        want_pos = np.concatenate([np.arange(off[n], off[n + 1]) for n in members])
+        assert np.array_equal(pos, np.tile(want_pos, (Hkv, 1))) and cu[-1] == len(want_pos)
+        rows = want_pos.astype(np.int32)
+        o, lse = oracle.sync(q[rows], ka, va, kv_pos=pos, q_pos=rows, kv_head_major=True)
+        if len(members) == 1:
+            assert np.allclose(o, o_loc[rows], atol=1e-12) and np.allclose(lse, lse_loc[rows], atol=1e-12)
+        elif len(members) == 4:
+            assert np.allclose(o, o_den, atol=1e-12) and np.allclose(lse, lse_den, atol=1e-12)
+        else:
+            g = Hq // Hkv
+            ob, lb = brute_attention(q[rows], lambda j, kvh: k[j, kvh], lambda j, kvh: v[j, kvh],
+                                     lambda i, h: ([int(j) for j in want_pos if j <= rows[i]], h // g),
+                                     1.0 / math.sqrt(d))
+            assert np.allclose(o, ob, atol=1e-12) and np.allclose(lse, lb, atol=1e-12)
+
+
+def test_decode_over_global_cache_plus_private_suffix_is_the_merge_of_two_decodes(oracle):
+    """A sync-block decode step after generation has begun: the shared global cache followed by the
+    participant's own new rows.  Softmax over a disjoint union = log-sum-exp merge of the parts."""
+    n, T, cap, Hq, Hkv, d = 3, 11, 4, 4, 2, 4
+    kg, vg = randn(T, Hkv, d), randn(T, Hkv, d)
+    ksx, vsx = randn(n, cap, Hkv, d), randn(n, cap, Hkv, d)
+    q = randn(n, Hq, d)
+    sfx = [4, 0, 2]
+    o_g, lse_g = oracle.decode(q, kg, vg, [T], True)
+    o_s, lse_s = oracle.decode(q, ksx, vsx, sfx, False)
+    assert np.all(o_s[1] == 0) and np.all(np.isneginf(lse_s[1]))
+    cat_k = np.concatenate([np.broadcast_to(kg, (n,) + kg.shape), ksx], axis=1)
+    cat_v = np.concatenate([np.broadcast_to(vg, (n,) + vg.shape), vsx], axis=1)
+    o, lse = oracle.decode(q, cat_k, cat_v, [T + s for s in sfx], False)
+    om, lm = lse_merge(o_g, lse_g, o_s, lse_s)
+    assert np.allclose(o, om, atol=1e-12) and np.allclose(lse, lm, atol=1e-12)
+
+
 def test_input_generators_are_seeded_and_typed():
     w = fi.cfg2()
     a = fi.normal(2, fi.TENSOR_Q, 0, (4, 3), "bf16")
