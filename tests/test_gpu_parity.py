@@ -411,6 +411,14 @@ def _full_size_local_sync(oracle, w, n_random, block=0):
     assert e / np.abs(oo).max() < 0.05
 
 
+def test_long_segments_many_kv_tiles_sampled(oracle):
+    """One 33 k-token participant next to a short one: 258 KV tiles per query tile at the end of the
+    walk, ragged last tile, barrier phases and ring stages wrapping many times; odd group size (3 query
+    heads per KV head: the last head pair of a KV head is a single head)."""
+    w = fi.Workload("long", 77, (32768 + 77, 131), 6, 2, 128, "bf16")
+    _full_size_local_sync(oracle, w, 48)
+
+
 def test_cfg2_full_size_sampled(oracle):
     _full_size_local_sync(oracle, fi.cfg2(), 256)
 
