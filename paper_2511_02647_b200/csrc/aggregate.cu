@@ -87,8 +87,9 @@ cudaError_t launch_concat(const PartsParams &pp, int hkv, int d, int elt_bytes, 
 // square of a bf16/fp32 value is exact in fp64, so only the summation order matters and it is
 // fixed here.  Output index: Hkv * off[n] + h * L_n + j.
 // s + x^2 for the two bf16 values packed in w, low half first; each square is exact in fp64.
-// (Squaring in fp32 and widening the result by integer bit moves avoids the slow fp32->fp64
-// conversion but was measured slower: the extra integer and range-check instructions cost more.)
+// (Widening by integer bit moves instead of the fp32->fp64 conversion, for all or for half of the
+// terms, was measured no faster: four integer instructions cost the integer pipe what one
+// conversion costs the conversion unit, and the phase waits for its data more than for either.)
 __device__ __forceinline__ double sq_acc_bf16x2(double s, uint32_t w)
 {
     const double lo = (double)__uint_as_float(w << 16);
@@ -102,12 +103,13 @@ __device__ __forceinline__ double sq_acc_bf16x2(double s, uint32_t w)
 // ---- top-k scores + selection + gather, one launch ----------------------------------------------
 // grid (KV head, participant, slice); the slices of one (head, participant) form a thread-block
 // cluster.
-//  1. Scores.  Slice r takes a contiguous share of the participant's tokens.  It copies their K rows
-//     of this head (row_bytes each, strided by the token pitch) into shared memory with 16-byte
-//     cp.async, each row padded by 16 bytes, and thread i walks row i: s = sum_c x_c^2 accumulated in
-//     fp64 in increasing c.  Each square of a bf16/fp32 value is exact in fp64, so only the order
-//     matters and it is fixed.  Scores are non-negative doubles, so their bit patterns order like
-//     unsigned integers; they are kept as such keys in shared memory.
+//  1. Scores.  Slice r takes a contiguous share of the participant's tokens.  Every warp copies the K
+//     rows of this head for 32 tokens at a time (row_bytes each, strided by the token pitch) into a
+//     ring of its own in shared memory with 16-byte cp.async, 128 bytes of every row per step, and
+//     lane i walks row i: s = sum_c x_c^2 accumulated in fp64 in increasing c.  Each square of a
+//     bf16/fp32 value is exact in fp64, so only the order matters and it is fixed.  Scores are
+//     non-negative doubles, so their bit patterns order like unsigned integers; they are kept as such
+//     keys in shared memory.
 //  2. Every slice collects the other slices' keys through distributed shared memory.
 //  3. Selection, repeated by every slice: an 8-bit-per-pass radix select, started at the highest bit
 //     in which two keys differ, finds the k-th largest score tau and how many rows equal to tau are
@@ -119,22 +121,25 @@ __device__ __forceinline__ double sq_acc_bf16x2(double s, uint32_t w)
 //     indices and global positions.
 constexpr int kSelThreads = 256;
 constexpr int kSelMaxLen = 4096;
-constexpr int kStageRows = 128;            // K rows staged per pass and buffer
 constexpr int kMaxSlices = 8;              // portable cluster size
 
 template <int kDtype>
 __global__ void __launch_bounds__(kSelThreads)
 topk_fused_kernel(const PartsParams pp, int hkv, int vpr /* 16-byte vectors per (row, head) */,
+                  int n_stages /* buffers in every warp's staging ring, 2..4 */,
+                  int max_len /* longest participant: sizes the key arrays */,
                   uint4 *k_agg, uint4 *v_agg, int32_t *kv_pos, int32_t *cu_kv, int32_t *sel_idx_out)
 {
-    extern __shared__ __align__(16) uint8_t stage[];           // [2][kStageRows][row_bytes + 16]
-    __shared__ unsigned long long keys[kSelMaxLen];
+    // dynamic shared memory: keys [max_len] u64 | kept rows [max_len] u16 | staging [8 warps][n_stages][32 rows][128 B]
+    extern __shared__ __align__(16) uint8_t dyn_smem[];
+    unsigned long long *keys = reinterpret_cast<unsigned long long *>(dyn_smem);
+    uint16_t *my_rows = reinterpret_cast<uint16_t *>(dyn_smem + (size_t)max_len * 8);   // kept indices of this CTA's slice (< 4096)
+    uint8_t *stage = dyn_smem + (((size_t)max_len * 10 + 15) & ~(size_t)15);
     __shared__ int hist[256];
     __shared__ int warp_tot[kSelThreads / 32];
     __shared__ int sh_bin, sh_krem, sh_count;
     __shared__ unsigned long long sh_tau;
     __shared__ unsigned long long warp_or[kSelThreads / 32], warp_and[kSelThreads / 32];
-    __shared__ uint16_t my_rows[kSelMaxLen];                  // kept indices of this CTA's slice (< 4096)
 
     namespace cg = cooperative_groups;
     cg::cluster_group cluster = cg::this_cluster();
@@ -148,59 +153,80 @@ topk_fused_kernel(const PartsParams pp, int hkv, int vpr /* 16-byte vectors per 
 
     // ---- 1. scores of this slice's tokens ----
     {
-        const int row_bytes = vpr * 16, stride = row_bytes + 16;
+        // Every warp runs a pipeline of its own, without CTA-wide barriers: it takes the row groups
+        // (32 rows, one per lane) w, w + 8, ... of the slice, copies a group's K rows of this head into its
+        // private ring of n_stages buffers in column blocks of up to 8 chunks (128 bytes per row, chunks
+        // XOR-swizzled by the row so that lane i walks row i without bank conflicts), and walks block
+        // after block with the chain carried in a register.  n_stages - 1 blocks per warp are in flight
+        // while one is walked; the conversion unit, the narrow pipe of this phase, is shared by all the
+        // warps of the SM and stays busy because they drift apart.
+        const int row_bytes = vpr * 16;
         const int per = (len + n_slices - 1) / n_slices;
         const int r0 = min(slice * per, len), r1 = min(r0 + per, len);
         const uint8_t *src = reinterpret_cast<const uint8_t *>(pp.k[n]) + (size_t)h * row_bytes;
         const size_t pitch = (size_t)hkv * row_bytes;          // bytes between consecutive tokens
-        const uint32_t sbase = (uint32_t)__cvta_generic_to_shared(stage);
-        // two buffers of kStageRows rows: the copy of the next pass is in flight during the chains of this one
-        auto copy_pass = [&](int c0, int buf) {
-            const int rows = min(kStageRows, r1 - c0);
-            for (int q = tid; q < rows * vpr; q += kSelThreads) {
-                const int r = q / vpr, ch = q - r * vpr;
-                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(sbase + (buf * kStageRows + r) * stride + ch * 16),
-                             "l"(src + (size_t)(c0 + r) * pitch + ch * 16) : "memory");
+        constexpr int kBlk = 8;                                // chunks per column block
+        constexpr int kBufBytes = 32 * kBlk * 16;              // one buffer: 32 rows x 128 bytes
+        const uint32_t wbase = (uint32_t)__cvta_generic_to_shared(stage) + warp * n_stages * kBufBytes;
+        const uint8_t *wstage = stage + (size_t)warp * n_stages * kBufBytes;
+        const int n_blk = (vpr + kBlk - 1) / kBlk;             // column blocks per row
+        const int n_grp = (r1 - r0 + 31) / 32;                 // row groups of the slice
+        const int my_grp = n_grp > warp ? (n_grp - warp + kSelThreads / 32 - 1) / (kSelThreads / 32) : 0;
+        const int n_u = my_grp * n_blk;                        // (group, block) units of this warp, in order
+        auto copy_unit = [&](int u) {                          // always commits a group, possibly empty
+            if (u < n_u) {
+                const int g = warp + (u / n_blk) * (kSelThreads / 32), blk = u % n_blk;
+                const int c0 = r0 + g * 32, rows = min(32, r1 - c0);
+                const int nc = min(kBlk, vpr - blk * kBlk);    // chunks of this block
+                const uint32_t buf = wbase + (u % n_stages) * kBufBytes;
+                for (int q = lane; q < rows * nc; q += 32) {
+                    const int r = nc == kBlk ? q >> 3 : q / nc, ch = q - r * nc;
+                    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;"
+                                 ::"r"(buf + r * (kBlk * 16) + ((ch ^ (r & (kBlk - 1))) << 4)),
+                                   "l"(src + (size_t)(c0 + r) * pitch + (blk * kBlk + ch) * 16) : "memory");
+                }
             }
             asm volatile("cp.async.commit_group;" ::: "memory");
         };
-        if (r0 < r1) copy_pass(r0, 0);
-        int buf = 0;
-        for (int c0 = r0; c0 < r1; c0 += kStageRows, buf ^= 1) {
-            const int rows = min(kStageRows, r1 - c0);
-            if (c0 + kStageRows < r1) {
-                copy_pass(c0 + kStageRows, buf ^ 1);           // that buffer's chains ended before the last barrier
-                asm volatile("cp.async.wait_group 1;" ::: "memory");
-            } else {
-                asm volatile("cp.async.wait_group 0;" ::: "memory");
-            }
-            __syncthreads();
-            if (tid < rows) {
-                const uint4 *mine = reinterpret_cast<const uint4 *>(stage + (size_t)(buf * kStageRows + tid) * stride);
-                double sc = 0.0;
+        for (int u = 0; u < n_stages - 1; ++u) copy_unit(u);
+        double sc = 0.0;
+        for (int u = 0; u < n_u; ++u) {
+            copy_unit(u + n_stages - 1);                       // into the buffer walked one unit ago
+            if (n_stages == 2) asm volatile("cp.async.wait_group 1;" ::: "memory");
+            else if (n_stages == 3) asm volatile("cp.async.wait_group 2;" ::: "memory");
+            else asm volatile("cp.async.wait_group 3;" ::: "memory");
+            __syncwarp();
+            const int g = warp + (u / n_blk) * (kSelThreads / 32), blk = u % n_blk;
+            const int row = r0 + g * 32 + lane;
+            const int nc = min(kBlk, vpr - blk * kBlk);
+            if (blk == 0) sc = 0.0;
+            if (row < r1) {
+                const uint4 *mine = reinterpret_cast<const uint4 *>(wstage + (size_t)(u % n_stages) * kBufBytes + lane * (kBlk * 16));
+                const int sw = lane & (kBlk - 1);
                 if (kDtype == FEDATTN_BF16) {
-                    for (int v = 0; v < vpr; ++v) {
-                        const uint4 w = mine[v];
+                    for (int v = 0; v < nc; ++v) {
+                        const uint4 w = mine[v ^ sw];
                         sc = sq_acc_bf16x2(sc, w.x);
                         sc = sq_acc_bf16x2(sc, w.y);
                         sc = sq_acc_bf16x2(sc, w.z);
                         sc = sq_acc_bf16x2(sc, w.w);
                     }
                 } else {
-                    for (int v = 0; v < vpr; ++v) {
-                        const uint4 u = mine[v];
-                        const float x0 = __uint_as_float(u.x), x1 = __uint_as_float(u.y), x2 = __uint_as_float(u.z),
-                                    x3 = __uint_as_float(u.w);
+                    for (int v = 0; v < nc; ++v) {
+                        const uint4 u4 = mine[v ^ sw];
+                        const float x0 = __uint_as_float(u4.x), x1 = __uint_as_float(u4.y), x2 = __uint_as_float(u4.z),
+                                    x3 = __uint_as_float(u4.w);
                         sc = __fma_rn((double)x0, (double)x0, sc);
                         sc = __fma_rn((double)x1, (double)x1, sc);
                         sc = __fma_rn((double)x2, (double)x2, sc);
                         sc = __fma_rn((double)x3, (double)x3, sc);
                     }
                 }
-                keys[c0 + tid] = (unsigned long long)__double_as_longlong(sc);
+                if (blk == n_blk - 1) keys[row] = (unsigned long long)__double_as_longlong(sc);
             }
-            __syncthreads();                                   // this buffer may be refilled two passes on
+            __syncwarp();                                      // the buffer is refilled n_stages - 1 units on
         }
+        asm volatile("cp.async.wait_group 0;" ::: "memory");   // only empty groups are left
         // ---- 2. the other slices' keys ----
         cluster.sync();
         for (int q = 1; q < n_slices; ++q) {
@@ -397,14 +423,25 @@ cudaError_t launch_topk_fused(const PartsParams &pp, int hkv, int d, int dtype, 
 {
     if (pp.cu_kv[pp.n] == 0 && !cu_kv) return cudaSuccess;
     const int elt = dtype == FEDATTN_BF16 ? 2 : 4;
-    const int smem = 2 * kStageRows * (d * elt + 16);
+    const int vpr = d * elt / 16;
+    int max_len = 0;
+    for (int i = 0; i < pp.n; ++i) max_len = max(max_len, pp.off[i + 1] - pp.off[i]);
+    if (max_len > kSelMaxLen) return cudaErrorInvalidValue;
+    // Shared memory per CTA: keys (8 B) and kept rows (2 B) per token of the longest participant, then
+    // the staging buffers.  As many buffers (2..4) as still let two CTAs share an SM: what is in flight
+    // from HBM is all but one of them.
+    const int stage_bytes = (kSelThreads / 32) * 32 * 128;    // one buffer per warp: 32 rows x 128 bytes
+    const int fixed = (max_len * 10 + 15) & ~15;
+    const int two_per_sm = (228 * 1024) / 2 - 1024 /*reserved per CTA*/ - 2048 /*static*/;
+    int n_stages = (two_per_sm - fixed) / stage_bytes;
+    n_stages = n_stages < 2 ? 2 : (n_stages > 4 ? 4 : n_stages);
+    const int smem = fixed + n_stages * stage_bytes;
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(topk_fused_kernel<FEDATTN_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             2 * kStageRows * (FEDATTN_MAX_HEAD_DIM * 2 + 16));
+        const int most = 227 * 1024 - 2048;
+        cudaError_t e = cudaFuncSetAttribute(topk_fused_kernel<FEDATTN_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
         if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(topk_fused_kernel<FEDATTN_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     2 * kStageRows * (FEDATTN_MAX_HEAD_DIM * 4 + 16));
+            e = cudaFuncSetAttribute(topk_fused_kernel<FEDATTN_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
@@ -423,12 +460,11 @@ cudaError_t launch_topk_fused(const PartsParams &pp, int hkv, int d, int dtype, 
     attr.val.clusterDim.x = 1; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = slices;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    const int vpr = d * elt / 16;
     cudaError_t e = dtype == FEDATTN_BF16
-                        ? cudaLaunchKernelEx(&cfg, topk_fused_kernel<FEDATTN_BF16>, pp, hkv, vpr, (uint4 *)k_agg, (uint4 *)v_agg,
-                                             kv_pos, cu_kv, sel_idx_out)
-                        : cudaLaunchKernelEx(&cfg, topk_fused_kernel<FEDATTN_F32>, pp, hkv, vpr, (uint4 *)k_agg, (uint4 *)v_agg,
-                                             kv_pos, cu_kv, sel_idx_out);
+                        ? cudaLaunchKernelEx(&cfg, topk_fused_kernel<FEDATTN_BF16>, pp, hkv, vpr, n_stages, max_len,
+                                             (uint4 *)k_agg, (uint4 *)v_agg, kv_pos, cu_kv, sel_idx_out)
+                        : cudaLaunchKernelEx(&cfg, topk_fused_kernel<FEDATTN_F32>, pp, hkv, vpr, n_stages, max_len,
+                                             (uint4 *)k_agg, (uint4 *)v_agg, kv_pos, cu_kv, sel_idx_out);
     ++*launches;
     return e != cudaSuccess ? e : cudaGetLastError();
 }

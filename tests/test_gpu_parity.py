@@ -158,6 +158,30 @@ def test_topk_max_length_many_slices_and_degenerate_scores(oracle):
         assert np.array_equal(host(agg["k_agg"]), ka) and np.array_equal(host(agg["v_agg"]), va)
 
 
+@pytest.mark.parametrize("d", [128, 64, 40])
+def test_topk_zero_and_subnormal_terms(oracle, d):
+    """Rows with exact zeros, bf16 subnormals and all-zero rows (padding): their scores must still be
+    the exact chain, also where rows differ only by such terms (scores of the order of 1e-80)."""
+    lens = [300, 97]
+    hkv = 2
+    _, k, v = gen(23, lens, hkv, hkv, d, "bf16")
+    rng = np.random.default_rng(23)
+    k[rng.random(k.shape) < 0.05] = 0.0                               # scattered zeros, any column
+    tiny = np.float32(2.0 ** -130)                                    # a bf16 subnormal
+    k[10:40] = 0.0                                                    # all-zero rows
+    k[20:30, :, d - 1] = tiny * np.arange(1, 11, dtype=np.float32)[:, None]   # ... some with one subnormal term
+    k[40:50, :, ::2] = tiny                                           # rows of zeros and subnormals only
+    k[305:320, :, d // 2:] = 0.0                                      # half-zero rows in the second participant
+    kp, vp = split(k, lens), split(v, lens)
+    r = Runner(len(lens), hkv, hkv, d, "bf16", sum(lens))
+    for ksel in ([280, 50], [295, 97], [5, 1]):
+        agg = r.aggregate(fa().AGG_TOPK_KNORM, kp, vp, ksel)
+        ka, va, pos, cu, sel = oracle.aggregate_topk(kp, vp, ksel)
+        assert agg["status"] == 0
+        assert np.array_equal(agg["sel_idx"].cpu().numpy(), sel), ksel
+        assert np.array_equal(host(agg["k_agg"]), ka) and np.array_equal(host(agg["v_agg"]), va)
+
+
 def test_topk_fp32_head_dim_128(oracle):
     lens = [700, 300]
     hkv, d = 8, 128
