@@ -235,7 +235,11 @@ topk_fused_kernel(const PartsParams pp, int hkv, int vpr /* 16-byte vectors per 
             const unsigned long long *pk = cluster.map_shared_rank(keys, peer);
             for (int j = p0 + tid; j < p1; j += kSelThreads) keys[j] = pk[j];
         }
-        cluster.sync();                                       // nobody reads this CTA's shared memory after this
+        // This CTA is done reading its peers; it may not exit before they are done reading it.  Arrive
+        // now, wait at the very end: nothing after this touches distributed shared memory, and nobody
+        // writes the keys a peer may still be reading.
+        asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+        __syncthreads();                                      // the collected keys, for this CTA's own threads
     }
 
     // ---- 3. selection ----
@@ -415,6 +419,7 @@ topk_fused_kernel(const PartsParams pp, int hkv, int vpr /* 16-byte vectors per 
         if (kv_pos) kv_pos[out_row0 + r] = pp.off[n] + my_rows[r];
         if (sel_idx_out) sel_idx_out[out_row0 + r] = my_rows[r];
     }
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
 cudaError_t launch_topk_fused(const PartsParams &pp, int hkv, int d, int dtype, void *k_agg, void *v_agg,
