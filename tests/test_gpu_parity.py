@@ -510,6 +510,16 @@ def test_invalid_arguments_are_rejected():
     with pytest.raises(m.FedAttnError):
         m.fedattn_decode(r.ctx, r.shape, 3, q[:2], kv, kv, 0, torch.zeros(2, dtype=torch.int32, device="cuda"), 8,
                          o[:2])                                               # unknown decode mode
+    lse = torch.zeros((64, 4), dtype=torch.float32, device="cuda")
+    with pytest.raises(m.FedAttnError) as e:
+        m.fedattn_sync_remote(r.ctx, m.Shape(2, 4, 2, 128, m.BF16, 0), q, [0, 40, 64], kv, kv, None, 64, False, o, lse)
+    assert e.value.code == 2                                                  # needs the causal order: unsupported
+    with pytest.raises(m.FedAttnError):
+        m.fedattn_sync_remote(r.ctx, r.shape, q, [0, 40, 30], kv, kv, None, 64, False, o, lse)   # non-monotone offsets
+    with pytest.raises(m.FedAttnError):
+        m.fedattn_merge(r.ctx, r.shape, -1, o, lse, o, lse, o, lse)           # negative row count
+    with pytest.raises(m.FedAttnError):
+        m.fedattn_merge(r.ctx, r.shape, 64, o, None, o, lse, o, lse)          # a partial result without its lse
     assert r.ctx.launch_count() == before and r.poll() == 0
     m.fedattn_local(r.ctx, r.shape, q, kv, kv, [0, 40, 64], o)                # still usable
     assert r.poll() == 0 and r.ctx.launch_count() > before
