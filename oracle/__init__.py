@@ -154,6 +154,22 @@ def aggregate_topk(k_parts, v_parts, k_sel):
     return aggregate_indexed(k_parts, v_parts, k_sel, sel_idx) + (sel_idx,)
 
 
+def aggregate_topk_token(k_parts, v_parts, k_sel):
+    """Sparse aggregation with token-level selection (the selection matrix of the paper's adaptive
+    aggregation picks whole tokens): one score per token, the squared norm of its whole key row
+    [Hkv * d] accumulated in fp64 in memory order, same order and tie rule as the per-head selector;
+    every KV head keeps the same tokens.  The definition is the per-head one applied to the row
+    viewed as a single head.  Returns (k_agg [T,Hkv,d], v_agg, kv_pos [T], cu_kv [N+1], sel_idx [T])."""
+    k_parts = [_f64(x) for x in k_parts]
+    v_parts = [_f64(x) for x in v_parts]
+    hkv, d = k_parts[0].shape[1:]
+    flat_k = [x.reshape(x.shape[0], 1, hkv * d) for x in k_parts]
+    flat_v = [x.reshape(x.shape[0], 1, hkv * d) for x in v_parts]
+    k_agg, v_agg, kv_pos, cu_kv, sel = aggregate_topk(flat_k, flat_v, k_sel)
+    T = k_agg.shape[1]
+    return k_agg.reshape(T, hkv, d), v_agg.reshape(T, hkv, d), kv_pos[0], cu_kv, sel[0]
+
+
 def sync(q, k_agg, v_agg, kv_pos=None, q_pos=None, kv_head_major: bool = False,
          scale: float = 0.0, causal: bool = True, rows: Optional[Sequence[int]] = None):
     """Global attention of packed queries Q [L,Hq,d] over the aggregated KV

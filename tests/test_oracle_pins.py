@@ -240,6 +240,45 @@ def test_topk_constructed_norms(oracle):
     assert list(oracle.topk_knorm(kp, 1)[0]) == [2]
 
 
+def test_token_level_selection_bruteforce_and_special_cases(oracle):
+    """Token-level selection: one score per token over all KV heads, the same tokens for every head."""
+    lens = [9, 6, 7]
+    Hkv, d = 3, 4
+    ks = [fi.round_to_bf16(randn(n, Hkv, d).astype(np.float32)).astype(np.float64) for n in lens]
+    vs = [randn(n, Hkv, d) for n in lens]
+    ks[0][4] = ks[0][1]                          # a tie between tokens 1 and 4
+    ks[2][5] = ks[2][0][::-1]                    # heads permuted: the same terms in another order
+    off = np.concatenate([[0], np.cumsum(lens)])
+    ksel = [4, 0, 3]
+    k_agg, v_agg, kv_pos, cu, sel = oracle.aggregate_topk_token(ks, vs, ksel)
+    assert k_agg.shape == (7, Hkv, d) and kv_pos.shape == (7,) and np.array_equal(cu, [0, 4, 4, 7])
+    at = 0
+    for n, kk in enumerate(ksel):
+        # nested-loop score in memory order (head, then channel), python floats = the fp64 chain
+        score = []
+        for j in range(lens[n]):
+            acc = 0.0
+            for h in range(Hkv):
+                for c in range(d):
+                    acc = acc + float(ks[n][j, h, c]) * float(ks[n][j, h, c])
+            score.append(acc)
+        want = rank_select(score, kk)
+        assert list(sel[at:at + kk]) == want
+        for t, j in enumerate(want):
+            assert np.array_equal(k_agg[at + t], ks[n][j]) and np.array_equal(v_agg[at + t], vs[n][j])
+            assert kv_pos[at + t] == off[n] + j
+        at += kk
+    # one KV head: token-level and per-head selection coincide
+    k1 = [x[:, :1] for x in ks]; v1 = [x[:, :1] for x in vs]
+    a = oracle.aggregate_topk_token(k1, v1, ksel)
+    b = oracle.aggregate_topk(k1, v1, ksel)
+    assert np.array_equal(a[0], b[0][0][:, None, :]) and np.array_equal(a[2], b[2][0]) and np.array_equal(a[4], b[4][0])
+    # every token kept: the concatenation
+    ka, va, pos, cu2 = oracle.aggregate_concat(ks, vs)
+    k_all, v_all, pos_all, _, _ = oracle.aggregate_topk_token(ks, vs, lens)
+    assert np.array_equal(k_all, ka) and np.array_equal(v_all, va) and np.array_equal(pos_all, pos)
+
+
 def test_sparse_aggregation_layout_and_special_cases(oracle):
     lens = [6, 4, 5]
     Hkv, d = 2, 4
