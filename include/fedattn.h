@@ -111,18 +111,26 @@ fedattn_status fedattn_local(fedattn_ctx *ctx, const fedattn_shape *shape,
  *                           lower index first.  Kept rows are emitted in ascending index order.
  *   FEDATTN_AGG_INDEXED     as TOPK but the kept local indices are given in sel_idx_in
  *                           (dev int32 [Hkv, T], T = sum k_sel, block n at cu_kv[n], ascending).
+ *   FEDATTN_AGG_TOPK_TOKEN  token-level selection (the selection matrix pi_n picks whole tokens):
+ *                           one score per token, the squared norm of its whole key row [Hkv*d]
+ *                           (fp64, memory order), same tie rule; every KV head keeps the same
+ *                           tokens.  Outputs are token-major: k_agg, v_agg dev [T, Hkv, d];
+ *                           kv_pos dev int32 [T]; sel_idx_out dev int32 [T]; to be passed to
+ *                           fedattn_sync with kv_head_major = 0.
  *   Sparse outputs are head-major: k_agg, v_agg dev [Hkv, T, d]; kv_pos dev int32 [Hkv, T] =
  *   off_n + local index; sel_idx_out dev int32 [Hkv, T] local indices (TOPK; nullable);
  *   cu_kv dev int32 [N+1] = prefix sum of k_sel.  Dropped rows are removed, not zeroed.
  *
  *   k_parts, v_parts: host arrays of N dev pointers, participant n's [L_n,Hkv,d] (may be slices
  *   of one packed buffer).  seqlens_host host int32 [N].  k_sel_host host int32 [N], 0 <= k_sel[n]
- *   <= L_n (ignored for CONCAT).  TOPK needs L_n <= 4096 per participant (else UNSUPPORTED).
+ *   <= L_n (ignored for CONCAT).  Both TOPK modes need L_n <= 4096 per participant (else
+ *   UNSUPPORTED).
  *   kv_pos and cu_kv may be NULL when not wanted. */
 typedef enum {
     FEDATTN_AGG_CONCAT = 0,
     FEDATTN_AGG_TOPK_KNORM = 1,
-    FEDATTN_AGG_INDEXED = 2
+    FEDATTN_AGG_INDEXED = 2,
+    FEDATTN_AGG_TOPK_TOKEN = 3
 } fedattn_agg_mode;
 
 fedattn_status fedattn_aggregate_kv(fedattn_ctx *ctx, const fedattn_shape *shape, int32_t mode,

@@ -13,7 +13,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.environ.get("FEDATTN_LIBRARY") or os.path.join(_PKG, "lib", "libfedattn.so")
 
 F32, BF16 = 0, 1
-AGG_CONCAT, AGG_TOPK_KNORM, AGG_INDEXED = 0, 1, 2
+AGG_CONCAT, AGG_TOPK_KNORM, AGG_INDEXED, AGG_TOPK_TOKEN = 0, 1, 2, 3
 DECODE_LOCAL, DECODE_SYNC = 0, 1
 
 _SYMBOLS = ["fedattn_workspace_bytes", "fedattn_create", "fedattn_destroy", "fedattn_status_string",

@@ -188,7 +188,8 @@ fedattn_status fedattn_aggregate_kv(fedattn_ctx *ctx, const fedattn_shape *shape
                                     int32_t *sel_idx_out, fedattn_stream stream)
 {
     if (!ctx || !shape_ok(shape) || !k_parts || !v_parts || !seqlens) return FEDATTN_ERR_INVALID_ARG;
-    if (mode != FEDATTN_AGG_CONCAT && mode != FEDATTN_AGG_TOPK_KNORM && mode != FEDATTN_AGG_INDEXED)
+    if (mode != FEDATTN_AGG_CONCAT && mode != FEDATTN_AGG_TOPK_KNORM && mode != FEDATTN_AGG_INDEXED &&
+        mode != FEDATTN_AGG_TOPK_TOKEN)
         return FEDATTN_ERR_INVALID_ARG;
     const int N = shape->n_participants;
     PartsParams pp;
@@ -213,7 +214,7 @@ fedattn_status fedattn_aggregate_kv(fedattn_ctx *ctx, const fedattn_shape *shape
     if (mode == FEDATTN_AGG_INDEXED && T > 0 && !sel_idx_in) return FEDATTN_ERR_INVALID_ARG;
     const int64_t out_rows = mode == FEDATTN_AGG_CONCAT ? L : T;
     if (out_rows > 0 && (!k_agg || !v_agg || !aligned16(k_agg) || !aligned16(v_agg))) return FEDATTN_ERR_INVALID_ARG;
-    if (mode == FEDATTN_AGG_TOPK_KNORM)
+    if (mode == FEDATTN_AGG_TOPK_KNORM || mode == FEDATTN_AGG_TOPK_TOKEN)
         for (int n = 0; n < N; ++n)
             if (seqlens[n] > 4096) return FEDATTN_ERR_UNSUPPORTED;
     DeviceGuard g(ctx->c.device);
@@ -227,6 +228,12 @@ fedattn_status fedattn_aggregate_kv(fedattn_ctx *ctx, const fedattn_shape *shape
     }
     if (mode == FEDATTN_AGG_TOPK_KNORM) {
         err = launch_topk_fused(pp, hkv, d, shape->dtype, k_agg, v_agg, kv_pos, cu_kv, sel_idx_out, ctx->c.sm_count, s,
+                                &ctx->c.launches);
+        return err == cudaSuccess ? FEDATTN_OK : FEDATTN_ERR_CUDA;
+    }
+    if (mode == FEDATTN_AGG_TOPK_TOKEN) {
+        // the per-head kernel on the token row viewed as one head of Hkv * d channels: token-major output
+        err = launch_topk_fused(pp, 1, hkv * d, shape->dtype, k_agg, v_agg, kv_pos, cu_kv, sel_idx_out, ctx->c.sm_count, s,
                                 &ctx->c.launches);
         return err == cudaSuccess ? FEDATTN_OK : FEDATTN_ERR_CUDA;
     }

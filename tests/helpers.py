@@ -66,6 +66,15 @@ class Runner:
                        cu_kv=torch.full((self.n + 1,), -1, dtype=torch.int32, device="cuda"), sel_idx=None)
             m.fedattn_aggregate_kv(self.ctx, self.shape, mode, kd, vd, seqlens, None, None, out["k_agg"],
                                    out["v_agg"], out["kv_pos"], out["cu_kv"], None)
+        elif mode == m.AGG_TOPK_TOKEN:
+            T = int(sum(k_sel))
+            out = dict(k_agg=torch.zeros((T, self.hkv, self.d), dtype=td, device="cuda"),
+                       v_agg=torch.zeros((T, self.hkv, self.d), dtype=td, device="cuda"),
+                       kv_pos=torch.full((T,), -1, dtype=torch.int32, device="cuda"),
+                       cu_kv=torch.full((self.n + 1,), -1, dtype=torch.int32, device="cuda"),
+                       sel_idx=torch.full((T,), -1, dtype=torch.int32, device="cuda"))
+            m.fedattn_aggregate_kv(self.ctx, self.shape, mode, kd, vd, seqlens, list(k_sel), None, out["k_agg"],
+                                   out["v_agg"], out["kv_pos"], out["cu_kv"], out["sel_idx"])
         else:
             T = int(sum(k_sel))
             out = dict(k_agg=torch.zeros((self.hkv, T, self.d), dtype=td, device="cuda"),

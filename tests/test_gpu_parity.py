@@ -182,6 +182,28 @@ def test_topk_zero_and_subnormal_terms(oracle, d):
         assert np.array_equal(host(agg["k_agg"]), ka) and np.array_equal(host(agg["v_agg"]), va)
 
 
+@pytest.mark.parametrize("dtype,hq,hkv,d", [("bf16", 8, 2, 128), ("bf16", 32, 8, 128), ("f32", 4, 2, 64)])
+def test_token_level_selection_and_sync_over_it(oracle, dtype, hq, hkv, d):
+    """Token-level selection: one score per token over all KV heads (a chain of Hkv * d terms), indices
+    bit-exact; the token-major sparse KV then feeds the sync attention with a shared kv_pos."""
+    lens = [300, 97, 513]
+    q, k, v = gen(24, lens, hq, hkv, d, dtype)
+    k[310:330] = k[305]                                               # equal scores across tokens
+    kp, vp = split(k, lens), split(v, lens)
+    r = Runner(len(lens), hq, hkv, d, dtype, sum(lens))
+    for ksel in ([75, 24, 128], [300, 0, 1], [0, 0, 0]):
+        agg = r.aggregate(fa().AGG_TOPK_TOKEN, kp, vp, ksel)
+        ka, va, pos, cu, sel = oracle.aggregate_topk_token(kp, vp, ksel)
+        assert agg["status"] == 0
+        assert np.array_equal(agg["sel_idx"].cpu().numpy(), sel), ksel
+        assert np.array_equal(agg["kv_pos"].cpu().numpy(), pos) and np.array_equal(agg["cu_kv"].cpu().numpy(), cu)
+        assert np.array_equal(host(agg["k_agg"]), ka) and np.array_equal(host(agg["v_agg"]), va)
+        o, lse = r.sync(q, agg["k_agg"], agg["v_agg"], agg["kv_pos"], head_major=False)
+        oo, ol = oracle.sync(q, ka, va, kv_pos=pos)
+        check_close(o, oo, TOL[dtype], "sync over token-level selection %s" % ksel)
+        check_close(lse, ol, 1e-3, "sync over token-level selection lse %s" % ksel)
+
+
 def test_topk_fp32_head_dim_128(oracle):
     lens = [700, 300]
     hkv, d = 8, 128
