@@ -620,6 +620,17 @@ def run_cfg4(args):
                         max(3, min(K, 10)), n_sets)
 
     g_agg = _graph_timed(torch, agg, 2 * n_sets)
+    # token-level selection (one score per token over all KV heads): same bytes, token-major output
+    k_tok = torch.empty((T, Hkv, d), dtype=bf, device=dev); v_tok = torch.empty_like(k_tok)
+    pos_tok = torch.empty((T,), dtype=torch.int32, device=dev); sel_tok = torch.empty_like(pos_tok)
+
+    def agg_token(i):
+        b = sets[i % n_sets]
+        fa.fedattn_aggregate_kv(ctx, shape, fa.AGG_TOPK_TOKEN, b["kp"], b["vp"], seqlens, ksel, None, k_tok, v_tok,
+                                pos_tok, None, sel_tok)
+    ms_tok = _timed(torch, stream, agg_token, K, W)
+    g_tok = _graph_timed(torch, agg_token, 2 * n_sets)
+    assert ctx.poll() == 0
     kv_bytes = 2 * L * Hkv * d * 2
     agg_bytes = kv_bytes // 2 + (kv_bytes // 2) * T // L + kv_bytes * T // L     # K once + selected V + selected K,V written
     pk = peaks()
@@ -632,6 +643,9 @@ def run_cfg4(args):
             "traffic": TOPK_DRAM_BYTES}
     calls = {"aggregate_topk": {"ms": round(ms_agg, 5), "gbs": round(gbs, 1), "frac_hbm": round(gbs / pk["hbm"], 4),
                                 "graph_ms": round(g_agg, 5), "graph_gbs": round(g_gbs, 1), "graph_frac_hbm": round(g_gbs / pk["hbm"], 4)},
+             "aggregate_topk_token": {"ms": round(ms_tok, 5), "graph_ms": round(g_tok, 5),
+                                      "graph_gbs": round(agg_bytes / (g_tok * 1e-3) / 1e9, 1),
+                                      "graph_frac_hbm": round(agg_bytes / (g_tok * 1e-3) / 1e9 / pk["hbm"], 4)},
              "sync_sparse": {"ms": round(ms_sync, 5), "tflops": round(tf, 2), "frac_tensor": round(tf / pk["tensor"], 4)},
              "sync_exchange_own_complete": {"ms": round(ms_exch, 5), "tflops": round(f_exch / (ms_exch * 1e-3) / 1e12, 2),
                                             "launches": 3}}
