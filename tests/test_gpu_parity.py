@@ -391,6 +391,28 @@ def test_decode_sync_block_with_private_suffix(oracle, dtype, d):
         check_close(lse, ol, 1e-3, "decode with suffix lse %s" % sfx)
 
 
+def test_decode_logits_growing_and_falling_along_the_cache(oracle):
+    """Logits that grow (or fall) by far more than 2^8 from tile to tile and from split to split: the
+    exponent reference moves inside a CTA's walk, and the partials that are merged differ by hundreds
+    of binades (later or earlier splits carry all the weight)."""
+    n, cap, hq, hkv, d = 2, 5000, 8, 2, 128
+    w = fi.Workload("dg", 33, (cap,) * n, hq, hkv, d, "bf16")
+    _, k, v = w.qkv()
+    q = fi.round_to_bf16(np.abs(w.decode_q(0)))
+    ramp = (np.arange(n * cap, dtype=np.float32) % cap / 40.0)[:, None, None]
+    for kk in (fi.round_to_bf16(np.abs(k) * ramp), fi.round_to_bf16(np.abs(k) * ramp[::-1])):
+        kc, vc = kk.reshape(n, cap, hkv, d), v.reshape(n, cap, hkv, d)
+        r = Runner(n, hq, hkv, d, "bf16", n * cap)
+        o, lse = r.decode(q, kc, vc, [cap, 3777], False, max_kv_len=cap)
+        oo, ol = oracle.decode(q, kc, vc, [cap, 3777], False)
+        check_close(o, oo, TOL["bf16"], "decode local, ramped logits")
+        assert np.abs(lse - ol).max() / np.abs(ol).max() < 1e-3
+        o, lse = r.decode(q, kk, v, [n * cap], True, max_kv_len=n * cap)
+        oo, ol = oracle.decode(q, kk, v, [n * cap], True)
+        check_close(o, oo, TOL["bf16"], "decode sync, ramped logits")
+        assert np.abs(lse - ol).max() / np.abs(ol).max() < 1e-3
+
+
 def test_decode_many_splits_clusters_and_row_chunks(oracle):
     """Long caches: the splits of a (cache, KV head) span several clusters, so the cross-cluster merge
     runs; ragged lengths leave some splits empty; 48 stacked rows per KV head need two row chunks."""
