@@ -277,6 +277,35 @@ def test_sync_exchange_small(oracle, dtype, hq, hkv, d):
         check_close(lse, ol, 1e-3, "sync exchange lse %s" % ksel)
 
 
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_merge_of_partial_results_closed_form_and_empty_parts(dtype):
+    """fedattn_merge against the closed form (softmax over a disjoint union of key sets): weights
+    exp(lse - max) normalised; a part with lse = -inf carries no weight; two empty parts give 0, -inf."""
+    rng = np.random.default_rng(9)
+    L, hq, d = 70, 4, 128 if dtype == "bf16" else 64
+    o_a = fi.round_to_bf16(rng.standard_normal((L, hq, d)).astype(np.float32)) if dtype == "bf16" else rng.standard_normal((L, hq, d)).astype(np.float32)
+    o_b = fi.round_to_bf16(rng.standard_normal((L, hq, d)).astype(np.float32)) if dtype == "bf16" else rng.standard_normal((L, hq, d)).astype(np.float32)
+    lse_a = (rng.standard_normal((L, hq)) * 30).astype(np.float32)
+    lse_b = (rng.standard_normal((L, hq)) * 30).astype(np.float32)
+    lse_a[3] = -np.inf; o_a[3] = 0                    # empty first part
+    lse_b[5] = -np.inf; o_b[5] = 0                    # empty second part
+    lse_a[7] = lse_b[7] = -np.inf; o_a[7] = o_b[7] = 0    # both empty
+    lse_b[9] = lse_a[9]                               # equal weights: the mean
+    r = Runner(2, hq, hq, d, dtype, L)
+    o, lse = r.merge(o_a.astype(np.float64), lse_a, o_b.astype(np.float64), lse_b)
+    la, lb = lse_a.astype(np.float64), lse_b.astype(np.float64)
+    m = np.maximum(la, lb); m = np.where(np.isfinite(m), m, 0.0)
+    wa, wb = np.exp(la - m), np.exp(lb - m)
+    z = wa + wb
+    want = (o_a * wa[..., None] + o_b * wb[..., None]) / np.where(z > 0, z, 1.0)[..., None]
+    with np.errstate(divide="ignore"):
+        want_lse = m + np.log(z)
+    check_close(o, want, TOL[dtype], "merge o")
+    check_close(lse, want_lse, 1e-4 * 30, "merge lse")
+    assert np.all(o[7] == 0) and np.all(np.isneginf(lse[7]))
+    check_close(o[9], 0.5 * (o_a[9].astype(np.float64) + o_b[9]), TOL[dtype], "merge, equal weights")
+
+
 def test_cfg4_sync_exchange_full_size_sampled(oracle):
     w = fi.cfg4()
     q, k, v = w.qkv()
