@@ -155,6 +155,51 @@ def sync_blocks_of_rounds(local_forwards) -> List[int]:
     return blocks
 
 
+def random_subset(seed: int, participant: int, head: int, length: int, k: int) -> np.ndarray:
+    """k distinct local token indices of a participant of ``length`` tokens, drawn uniformly without
+    replacement from ``(seed, participant, head)`` and returned ascending: the random selector of a
+    sparse KV exchange.  The draw is an input of the method, not part of it."""
+    if not 0 <= k <= length:
+        raise ValueError("need 0 <= k <= length")
+    rng = np.random.default_rng([int(seed), TENSOR_MISC, 991, int(participant), int(head)])
+    return np.sort(rng.choice(int(length), size=int(k), replace=False)).astype(np.int32)
+
+
+def random_selection(seed: int, seqlens, k_sel, n_kv_heads: int) -> np.ndarray:
+    """Per-head random selection for every participant in the layout the indexed aggregation
+    takes: int32 [Hkv, sum k_sel], participant n's block at the prefix sum of k_sel, ascending."""
+    rows = [np.concatenate([random_subset(seed, n, h, int(ln), int(k)) for n, (ln, k) in enumerate(zip(seqlens, k_sel))]
+                           + [np.zeros(0, np.int32)]) for h in range(n_kv_heads)]
+    return np.stack(rows).astype(np.int32)
+
+
+def index_sets(seed: int, seqlens, kind: str) -> List[np.ndarray]:
+    """A partition of the global positions 0..L-1 into one ascending index set per participant
+    (participant n gets seqlens[n] positions).  kind = "contiguous": consecutive segments in
+    participant order; "interleaved": global position t goes to the participants in round-robin
+    order, skipping those that are full; "random": a seeded random assignment."""
+    seqlens = [int(x) for x in seqlens]
+    L = int(sum(seqlens))
+    if kind == "contiguous":
+        owner = np.repeat(np.arange(len(seqlens)), seqlens)
+    elif kind == "interleaved":
+        left = list(seqlens)
+        owner = np.empty(L, dtype=np.int64)
+        n = 0
+        for t in range(L):
+            while left[n % len(seqlens)] == 0:
+                n += 1
+            owner[t] = n % len(seqlens)
+            left[n % len(seqlens)] -= 1
+            n += 1
+    elif kind == "random":
+        owner = np.repeat(np.arange(len(seqlens)), seqlens)
+        _rng(seed, TENSOR_MISC, 4242).shuffle(owner)
+    else:
+        raise ValueError(kind)
+    return [np.nonzero(owner == n)[0].astype(np.int32) for n in range(len(seqlens))]
+
+
 def sample_rows(seed: int, seqlens, n_random: int, tile: int = 128) -> np.ndarray:
     """Row subset for sampled parity at full size: every row within +-1 of a segment
     start/end or of a multiple of ``tile`` (both in packed and in segment-relative

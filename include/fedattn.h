@@ -17,8 +17,15 @@
  *     stream) and the call returns without synchronising.
  *   - Errors are return codes.  Arguments are validated on the host before anything is
  *     launched; a rejected call launches nothing.  A device-side anomaly (a bounded wait that
- *     ran out, an out-of-range index in INDEXED mode) sets a status word in the workspace that
- *     fedattn_poll reads; the kernel still terminates and the context stays usable.
+ *     ran out, an out-of-range or unsorted index in INDEXED mode, positions in an order the call
+ *     cannot handle) sets a status word in the workspace that fedattn_poll reads; the kernel still
+ *     terminates and the context stays usable.  Outputs of the call that raised the status are
+ *     undefined.  After FEDATTN_ERR_TIMEOUT the bf16 head_dim 128 attention calls enqueued before
+ *     the next fedattn_poll do no work and leave their outputs untouched (they would otherwise
+ *     each wait out the same limit); poll, then repeat them.
+ *   - Q, K and V must be finite.  Rows outside a query's allowed set carry weight exactly 0, but
+ *     a tile that straddles a segment boundary multiplies those weights with the neighbour's V
+ *     rows, and 0 * Inf or 0 * NaN is NaN.
  *   - Layouts are row-major with head_dim contiguous.  Packed queries Q[L, Hq, d]; packed keys
  *     and values K,V[L, Hkv, d]; L = sum of segment lengths; query head h reads KV head
  *     h / (Hq / Hkv).  dtype is FEDATTN_F32 or FEDATTN_BF16 for all of Q, K, V, O of a call;
@@ -49,7 +56,8 @@ typedef enum {
     FEDATTN_ERR_WORKSPACE = 3,   /* workspace missing, misaligned or too small */
     FEDATTN_ERR_CUDA = 4,        /* a CUDA runtime/driver call failed */
     FEDATTN_ERR_TIMEOUT = 5,     /* device status: a bounded wait inside a kernel ran out */
-    FEDATTN_ERR_INDEX = 6        /* device status: INDEXED selection index out of range */
+    FEDATTN_ERR_INDEX = 6,       /* device status: INDEXED selection index out of range or not ascending */
+    FEDATTN_ERR_ORDER = 7        /* device status: kv_pos not non-decreasing in a call that needs it */
 } fedattn_status;
 
 typedef enum { FEDATTN_F32 = 0, FEDATTN_BF16 = 1 } fedattn_dtype;
@@ -83,8 +91,17 @@ const char *fedattn_status_string(fedattn_status s);
  * an anomaly) and clears it. */
 fedattn_status fedattn_poll(fedattn_ctx *ctx, fedattn_stream stream);
 
-/* Number of kernels this context has launched so far (for launch accounting). */
+/* Number of kernels this context has launched so far (for launch accounting), and how many of
+ * them were launches of the tensor-core (tcgen05) attention kernel. */
 int64_t fedattn_launch_count(const fedattn_ctx *ctx);
+int64_t fedattn_tensor_core_launch_count(const fedattn_ctx *ctx);
+
+/* Self-test of the bounded-wait protocol that every in-kernel wait follows.  Launches one small
+ * kernel that waits, with the library's own wait routine and a limit of `max_polls` polls
+ * (1..65536), on a barrier that nothing ever signals.  The wait runs out, the kernel raises
+ * FEDATTN_ERR_TIMEOUT in the status word and returns normally: no trap, no fault, the context
+ * stays usable.  For tests of the poll-and-repeat protocol described above. */
+fedattn_status fedattn_selftest_wait_timeout(fedattn_ctx *ctx, int32_t max_polls, fedattn_stream stream);
 
 /* ---- local attention: Phase I, o_n = Attention(q_n, k_n, v_n) ----------------------------------
  * Paper: Sec. IV-B "Phase I: Local Self-Attention", eq. (update_local_o), Algorithm 1 inner loop;
@@ -149,8 +166,14 @@ fedattn_status fedattn_aggregate_kv(fedattn_ctx *ctx, const fedattn_shape *shape
  *   q dev [L,Hq,d] (all participants' rows, packed; L = n_q_rows).
  *   k_agg, v_agg dev: kv_head_major == 0: [T,Hkv,d], kv_pos dev int32 [T] or NULL (= 0..T-1);
  *                     kv_head_major == 1: [Hkv,T,d], kv_pos dev int32 [Hkv,T] or NULL.
- *   kv_pos must be non-decreasing along T (aggregate_kv always produces that).
- *   q_pos dev int32 [L] or NULL.  o dev [L,Hq,d]; lse dev float [L,Hq] or NULL. */
+ *   q_pos dev int32 [L] or NULL.  o dev [L,Hq,d]; lse dev float [L,Hq] or NULL.
+ *   Order of positions.  With q_pos == NULL, kv_pos must be non-decreasing along T (what
+ *   fedattn_aggregate_kv produces for contiguous segments); the bf16 head_dim 128 kernel then
+ *   masks by a prefix count, checks the order as it goes and raises FEDATTN_ERR_ORDER (outputs
+ *   undefined) when it does not hold.  With q_pos given, query and key positions may come in ANY
+ *   order (general index sets L_n of Sec. IV-A, e.g. interleaved participants; a subset of the
+ *   participants' rows): every (query, key) pair is tested on its own positions.  To attend an
+ *   unsorted kv_pos from packed queries, pass q_pos = 0..L-1 explicitly. */
 fedattn_status fedattn_sync(fedattn_ctx *ctx, const fedattn_shape *shape,
                             const void *q, int64_t n_q_rows, const int32_t *q_pos,
                             const void *k_agg, const void *v_agg, const int32_t *kv_pos,
@@ -158,18 +181,20 @@ fedattn_status fedattn_sync(fedattn_ctx *ctx, const fedattn_shape *shape,
                             void *o, float *lse, fedattn_stream stream);
 
 /* ---- sync block with sparse KV exchange -----------------------------------------------------
- * Paper: Sec. VI, discussion of the sparsity-ratio experiment: "sparse KV exchange preserves
- * self-attention on complete local tokens within each participant while sparsifying remote KVs".
- * Row i of participant n attends its own keys off_n..i (complete) and the exchanged keys of the
- * other participants that are not later than i, under ONE softmax.  With contiguous segments the
- * second set is "aggregated rows positioned before off_n", so the block is computed as
+ * Paper: Sec. VI, discussion of the sparsity-ratio experiment (the own segment stays complete,
+ * only the keys and values received from the other participants are sparsified); Sec. III-B
+ * lets the attention operator stand for the masked or the unmasked (bidirectional) form.
+ * Row i of participant n attends its own keys (off_n..i when causal, the whole segment otherwise)
+ * and the exchanged keys of the OTHER participants that its mask allows, under ONE softmax.  With
+ * contiguous segments the second set is "aggregated rows positioned before off_n" (causal) or
+ * "aggregated rows positioned outside [off_n, off_{n+1})" (bidirectional), so the block is
  *     fedattn_local (o_a, lse_a)  +  fedattn_sync_remote (o_b, lse_b)  ->  fedattn_merge.
  *
  * fedattn_sync_remote: like fedattn_sync, but query row i of participant n (segments given by the
  *   HOST array cu_seqlens_host [N+1]) attends aggregated row j of KV head h iff
- *   kv_pos[h][j] < off_n.  shape->causal must be 1 (UNSUPPORTED otherwise).  Rows of the first
- *   participant, and any row with nothing before its segment, get o = 0 and lse = -inf.
- *   lse is needed for the merge (pass a buffer).
+ *   kv_pos[h][j] < off_n, or, when shape->causal == 0, also iff kv_pos[h][j] >= off_{n+1}.
+ *   kv_pos must be non-decreasing along T (NULL = 0..T-1).  A row with no such key gets o = 0 and
+ *   lse = -inf.  lse is needed for the merge (pass a buffer).
  * fedattn_merge: o = (e^{lse_a} o_a + e^{lse_b} o_b) / (e^{lse_a} + e^{lse_b}),
  *   lse = log(e^{lse_a} + e^{lse_b}) for n_rows query rows; o_a, o_b, o dev [n_rows,Hq,d] in
  *   shape->dtype, lse_a, lse_b dev float [n_rows,Hq], lse dev float or NULL.  o may alias o_a or
@@ -221,7 +246,9 @@ fedattn_status fedattn_decode(fedattn_ctx *ctx, const fedattn_shape *shape, int3
  * call) and their contents after a call are unspecified.  The few arrival counters beside them
  * must be zero when a call starts: they are zero when the library is loaded and every completed
  * call leaves them at zero.  All calls on one device share these arrays: two calls that may
- * overlap on the GPU (different streams, no ordering) race on them. */
+ * overlap on the GPU (different streams, no ordering) race on them.  The first call on a device
+ * also fills a small host-side table without locking: do not let two host threads make their
+ * first call on the same device at the same moment. */
 fedattn_status fedattn_decode_noalloc(const fedattn_shape *shape, int32_t mode,
                                       const void *q, const void *k_cache, const void *v_cache,
                                       int64_t cache_stride_participant, const int32_t *kv_len,

@@ -198,10 +198,11 @@ def sync(q, k_agg, v_agg, kv_pos=None, q_pos=None, kv_head_major: bool = False,
 
 
 def sync_exchange(q, k, v, seqlens, k_agg, v_agg, kv_pos, cu_kv, scale: float = 0.0,
-                  rows: Optional[Sequence[int]] = None):
-    """Sync block with sparse KV exchange: every participant attends its own complete (causal)
-    segment plus the exchanged, sparsified keys of the other participants that are not later than
-    the query.  q [L,Hq,d]; k, v [L,Hkv,d] local; k_agg, v_agg [Hkv,T,d] head-major aggregate with
+                  rows: Optional[Sequence[int]] = None, causal: bool = True):
+    """Sync block with sparse KV exchange: every participant attends its own complete segment
+    (causally, or all of it when ``causal`` is False) plus the exchanged, sparsified keys of the
+    other participants (those not later than the query, or all of them when ``causal`` is False).
+    q [L,Hq,d]; k, v [L,Hkv,d] local; k_agg, v_agg [Hkv,T,d] head-major aggregate with
     kv_pos [Hkv,T] and participant ranges cu_kv [N+1]."""
     q, k, v, k_agg, v_agg = _f64(q), _f64(k), _f64(v), _f64(k_agg), _f64(v_agg)
     L, hq, d = q.shape
@@ -215,7 +216,8 @@ def sync_exchange(q, k, v, seqlens, k_agg, v_agg, kv_pos, cu_kv, scale: float = 
     _load().fedattn_oracle_sync_exchange(_p(q), _p(k), _p(v), _p(off), C.c_int32(len(off) - 1),
                                          _p(k_agg), _p(v_agg), _p(kvp), _p(cu), C.c_int64(T),
                                          C.c_int32(hq), C.c_int32(hkv), C.c_int32(d),
-                                         C.c_double(_scale(scale, d)), _p(r), C.c_int64(n_rows), _p(o), _p(lse))
+                                         C.c_double(_scale(scale, d)), C.c_int32(int(causal)), _p(r),
+                                         C.c_int64(n_rows), _p(o), _p(lse))
     return o, lse
 
 

@@ -293,13 +293,14 @@ void fedattn_oracle_sync(const double *q, int64_t n_q, const int32_t *q_pos,
 
 /*
  * Sync block with sparse KV exchange as the paper's experiment describes it (Sec. VI, the
- * discussion of the sparsity-ratio figure: "sparse KV exchange preserves self-attention on
- * complete local tokens within each participant while sparsifying remote KVs"): row i of
- * participant n attends
- *     A = its own keys  { j : off_n <= j <= i }                       (complete, causal), and
- *     B = the exchanged keys of the OTHER participants that are not later than i,
- *         { t outside [cu_kv[n], cu_kv[n+1]) : kv_pos[kvh][t] <= i }  (sparsified, causal on the
- *         global position),
+ * discussion of the sparsity-ratio figure: every participant keeps self-attention over its own
+ * complete segment, only what it receives from the others is sparsified): row i of participant
+ * n attends
+ *     A = its own keys  { j : off_n <= j <= i }  (causal)  or the whole segment (causal == 0), and
+ *     B = the exchanged keys of the OTHER participants,
+ *         { t outside [cu_kv[n], cu_kv[n+1]) : kv_pos[kvh][t] <= i }  (causal on the global
+ *         position), or every such t when causal == 0 (Sec. III-B: the attention operator stands
+ *         for the masked or the bidirectional form),
  * with one softmax over A u B.  k, v: packed local tensors [L, Hkv, d]; k_agg, v_agg: head-major
  * aggregate [Hkv, T, d] with kv_pos [Hkv, T] and participant ranges cu_kv [N+1].
  * rows / o / lse as in fedattn_oracle_local.
@@ -308,7 +309,7 @@ void fedattn_oracle_sync_exchange(const double *q, const double *k, const double
                                   const int32_t *off, int32_t n_participants,
                                   const double *k_agg, const double *v_agg, const int32_t *kv_pos,
                                   const int32_t *cu_kv, int64_t total_kv,
-                                  int32_t hq, int32_t hkv, int32_t d, double scale,
+                                  int32_t hq, int32_t hkv, int32_t d, double scale, int32_t causal,
                                   const int64_t *rows, int64_t n_rows, double *o, double *lse)
 {
     const int32_t g = hq / hkv;
@@ -330,7 +331,8 @@ void fedattn_oracle_sync_exchange(const double *q, const double *k, const double
                 double *orow = o + (r * hq + h) * d;
                 int64_t na = 0;
                 double mx = -INFINITY;
-                for (int64_t j = off[n]; j <= i; ++j) {            /* set A */
+                const int64_t last_own = causal ? i : (int64_t)off[n + 1] - 1;
+                for (int64_t j = off[n]; j <= last_own; ++j) {     /* set A */
                     const double *kr = k + (j * hkv + kvh) * d;
                     double s = 0.0;
                     for (int32_t c = 0; c < d; ++c)
@@ -344,7 +346,7 @@ void fedattn_oracle_sync_exchange(const double *q, const double *k, const double
                 for (int64_t t = 0; t < total_kv; ++t) {           /* set B */
                     if (t >= cu_kv[n] && t < cu_kv[n + 1])
                         continue;
-                    if (kv_pos[(int64_t)kvh * total_kv + t] > i)
+                    if (causal && kv_pos[(int64_t)kvh * total_kv + t] > i)
                         continue;
                     const double *kr = k_agg + ((int64_t)kvh * total_kv + t) * d;
                     double s = 0.0;

@@ -430,6 +430,126 @@ def test_sync_exchange_is_local_merged_with_remote_only_sync(oracle):
 
 
 
+@pytest.mark.parametrize("ksel", [[2, 1, 0, 3], [3, 4, 2, 4], [0, 0, 0, 0]])
+def test_sync_exchange_bidirectional_bruteforce_and_limits(oracle, ksel):
+    """causal = 0: a row attends its whole own segment and every exchanged key of the other
+    participants (Sec. III-B: attention without the mask).  Brute force over a tagged union; with
+    every key exchanged it is bidirectional attention over the whole sequence, with none it is the
+    bidirectional local block."""
+    lens = [3, 4, 2, 4]
+    L, Hq, Hkv, d = sum(lens), 4, 2, 4
+    q, k, v = randn(L, Hq, d), randn(L, Hkv, d), randn(L, Hkv, d)
+    off = np.concatenate([[0], np.cumsum(lens)])
+    ks, vs = np.split(k, off[1:-1]), np.split(v, off[1:-1])
+    sel = fi.random_selection(77, lens, ksel, Hkv)
+    ka, va, pos, cu = oracle.aggregate_indexed(ks, vs, ksel, sel)
+    o, lse = oracle.sync_exchange(q, k, v, lens, ka, va, pos, cu, causal=False)
+    g, T = Hq // Hkv, ka.shape[1]
+    seg = np.searchsorted(off, np.arange(L), side="right") - 1
+
+    def allowed(i, h):
+        n = seg[i]
+        own = [("l", j) for j in range(off[n], off[n + 1])]
+        remote = [("a", t) for t in range(T) if not (cu[n] <= t < cu[n + 1])]
+        return own + remote, h // g
+
+    K = lambda key, kh: k[key[1], kh] if key[0] == "l" else ka[kh, key[1]]
+    V = lambda key, kh: v[key[1], kh] if key[0] == "l" else va[kh, key[1]]
+    bo, bl = brute_attention(q, K, V, allowed, 1 / math.sqrt(d))
+    assert np.abs(o - bo).max() < 1e-12 and np.abs(lse - bl).max() < 1e-12
+    if ksel == lens:
+        dense, dense_lse = oracle.sync(q, k, v, causal=False)
+        assert np.abs(o - dense).max() < 1e-12 and np.abs(lse - dense_lse).max() < 1e-12
+    if sum(ksel) == 0:
+        loc, loc_lse = oracle.local(q, k, v, lens, causal=False)
+        assert np.abs(o - loc).max() < 1e-13 and np.abs(lse - loc_lse).max() < 1e-13
+    # the decomposition the CUDA path uses: bidirectional local block merged with a remote-only pass
+    o_l, lse_l = oracle.local(q, k, v, lens, causal=False)
+    o_r = np.zeros_like(o_l); lse_r = np.full_like(lse_l, -np.inf)
+    for n in range(len(lens)):
+        keep = np.array([t for t in range(T) if not (cu[n] <= t < cu[n + 1])], dtype=np.int64)
+        if len(keep) and lens[n]:
+            rows = np.arange(off[n], off[n + 1])
+            o_r[rows], lse_r[rows] = oracle.sync(q[rows], ka[:, keep], va[:, keep], kv_head_major=True, causal=False)
+    om, lm = lse_merge(o_l, lse_l, o_r, lse_r)
+    assert np.abs(om - o).max() < 1e-12 and np.abs(lm - lse).max() < 1e-12
+
+
+def test_random_selection_feeds_the_exchange_block(oracle):
+    """The sparsity-ratio experiment samples the exchanged KV rows at random (Sec. VI): a seeded draw
+    per (participant, KV head) goes through the indexed aggregation into the exchange block.  Pinned
+    by brute force over the tagged union, by the draw's own invariants, and by the two limits."""
+    lens = [5, 3, 6, 4]
+    L, Hq, Hkv, d = sum(lens), 4, 2, 4
+    q, k, v = randn(L, Hq, d), randn(L, Hkv, d), randn(L, Hkv, d)
+    off = np.concatenate([[0], np.cumsum(lens)])
+    ks, vs = np.split(k, off[1:-1]), np.split(v, off[1:-1])
+    ksel = [2, 1, 3, 2]                                   # ratio 1/2, rounded
+    sel = fi.random_selection(5, lens, ksel, Hkv)
+    cu = np.concatenate([[0], np.cumsum(ksel)])
+    for h in range(Hkv):
+        for n in range(len(lens)):
+            blk = sel[h, cu[n]:cu[n + 1]]
+            assert np.all(np.diff(blk) > 0) and (len(blk) == 0 or (blk[0] >= 0 and blk[-1] < lens[n]))
+    assert not np.array_equal(sel[0], sel[1])             # heads draw independently
+    assert np.array_equal(sel, fi.random_selection(5, lens, ksel, Hkv))   # seeded
+    ka, va, pos, cu2 = oracle.aggregate_indexed(ks, vs, ksel, sel)
+    assert np.array_equal(cu2, cu)
+    o, lse = oracle.sync_exchange(q, k, v, lens, ka, va, pos, cu)
+    g, T = Hq // Hkv, ka.shape[1]
+    seg = np.searchsorted(off, np.arange(L), side="right") - 1
+
+    def allowed(i, h):
+        n, kvh = seg[i], h // g
+        own = [("l", j) for j in range(off[n], i + 1)]
+        remote = [("r", (m, int(j))) for m in range(len(lens)) if m != n
+                  for j in sel[kvh, cu[m]:cu[m + 1]] if off[m] + j <= i]
+        return own + remote, kvh
+
+    K = lambda key, kh: k[key[1], kh] if key[0] == "l" else ks[key[1][0]][key[1][1], kh]
+    V = lambda key, kh: v[key[1], kh] if key[0] == "l" else vs[key[1][0]][key[1][1], kh]
+    bo, bl = brute_attention(q, K, V, allowed, 1 / math.sqrt(d))
+    assert np.abs(o - bo).max() < 1e-12 and np.abs(lse - bl).max() < 1e-12
+    full = fi.random_selection(5, lens, lens, Hkv)        # ratio 1: every row, i.e. the dense sync block
+    ka, va, pos, cu3 = oracle.aggregate_indexed(ks, vs, lens, full)
+    dense, dense_lse = oracle.sync(q, k, v)
+    o1, l1 = oracle.sync_exchange(q, k, v, lens, ka, va, pos, cu3)
+    assert np.abs(o1 - dense).max() < 1e-13 and np.abs(l1 - dense_lse).max() < 1e-13
+
+
+@pytest.mark.parametrize("kind", ["interleaved", "random", "contiguous"])
+def test_general_index_sets_sync_equals_centralised_attention(oracle, kind):
+    """Sec. IV-A: the participants hold general ordered index sets L_n of the global sequence.  With
+    explicit positions for queries and aggregated keys, syncing reproduces centralised attention on
+    the sequence in its global order (the H = 1 reduction), whatever the partition; the concatenated
+    kv_pos is then not monotone.  Checked against torch's fp64 causal attention on the re-ordered
+    sequence and, for one participant's rows alone, against brute force."""
+    lens = [5, 2, 6, 3]
+    L, Hq, Hkv, d = sum(lens), 4, 2, 8
+    sets = fi.index_sets(9, lens, kind)
+    assert np.array_equal(np.sort(np.concatenate(sets)), np.arange(L))
+    pos = np.concatenate(sets).astype(np.int32)            # packed row r holds global position pos[r]
+    if kind != "contiguous":
+        assert np.any(np.diff(pos) < 0)
+    q, k, v = randn(L, Hq, d), randn(L, Hkv, d), randn(L, Hkv, d)      # in packed (participant) order
+    o, lse = oracle.sync(q, k, v, kv_pos=pos, q_pos=pos)
+    inv = np.argsort(pos)                                   # packed row of global position t
+    g = Hq // Hkv
+    tq = torch.from_numpy(q[inv]).permute(1, 0, 2)
+    tk = torch.from_numpy(np.repeat(k[inv], g, axis=1)).permute(1, 0, 2)
+    tv = torch.from_numpy(np.repeat(v[inv], g, axis=1)).permute(1, 0, 2)
+    want = torch.nn.functional.scaled_dot_product_attention(tq, tk, tv, is_causal=True).permute(1, 0, 2).numpy()
+    assert np.abs(o[inv] - want).max() < 1e-12
+    n = 2                                                   # one participant's rows against the global KV
+    r0 = sum(lens[:n])
+    rows = np.arange(r0, r0 + lens[n])
+    o_n, lse_n = oracle.sync(q[rows], k, v, kv_pos=pos, q_pos=pos[rows])
+    bo, bl = brute_attention(q[rows], lambda j, kvh: k[j, kvh], lambda j, kvh: v[j, kvh],
+                             lambda i, h: ([j for j in range(L) if pos[j] <= pos[rows[i]]], h // g), 1 / math.sqrt(d))
+    assert np.abs(o_n - bo).max() < 1e-12 and np.abs(lse_n - bl).max() < 1e-12
+    assert np.abs(o_n - o[rows]).max() < 1e-13
+
+
 def test_gqa_equals_mha_with_repeated_kv_heads(oracle):
     lens = [6, 5]
     L, Hq, Hkv, d = sum(lens), 6, 2, 8
