@@ -17,7 +17,8 @@ AGG_CONCAT, AGG_TOPK_KNORM, AGG_INDEXED, AGG_TOPK_TOKEN = 0, 1, 2, 3
 DECODE_LOCAL, DECODE_SYNC = 0, 1
 
 _SYMBOLS = ["fedattn_workspace_bytes", "fedattn_create", "fedattn_destroy", "fedattn_status_string",
-            "fedattn_poll", "fedattn_launch_count", "fedattn_local", "fedattn_aggregate_kv",
+            "fedattn_poll", "fedattn_launch_count", "fedattn_tensor_core_launch_count",
+            "fedattn_selftest_wait_timeout", "fedattn_local", "fedattn_aggregate_kv",
             "fedattn_sync", "fedattn_sync_remote", "fedattn_merge", "fedattn_decode", "fedattn_decode_noalloc"]
 
 
@@ -63,6 +64,10 @@ def _load():
     lib.fedattn_poll.argtypes = [vp, vp]
     lib.fedattn_launch_count.restype = i64
     lib.fedattn_launch_count.argtypes = [vp]
+    lib.fedattn_tensor_core_launch_count.restype = i64
+    lib.fedattn_tensor_core_launch_count.argtypes = [vp]
+    lib.fedattn_selftest_wait_timeout.restype = C.c_int
+    lib.fedattn_selftest_wait_timeout.argtypes = [vp, i32, vp]
     lib.fedattn_local.restype = C.c_int
     lib.fedattn_local.argtypes = [vp, C.POINTER(Shape), vp, vp, vp, C.POINTER(i32), vp, vp, vp]
     lib.fedattn_aggregate_kv.restype = C.c_int
@@ -143,6 +148,14 @@ class Context:
 
     def launch_count(self) -> int:
         return int(_lib.fedattn_launch_count(self._h))
+
+    def tensor_core_launch_count(self) -> int:
+        return int(_lib.fedattn_tensor_core_launch_count(self._h))
+
+    def selftest_wait_timeout(self, max_polls: int = 64, stream=None):
+        """Launches the kernel whose bounded wait runs out (raises the TIMEOUT status word)."""
+        _check(_lib.fedattn_selftest_wait_timeout(self._h, int(max_polls), _stream(stream)),
+               "fedattn_selftest_wait_timeout")
 
     def close(self):
         if self._h:

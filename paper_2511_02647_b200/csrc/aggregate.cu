@@ -83,9 +83,6 @@ cudaError_t launch_concat(const PartsParams &pp, int hkv, int d, int elt_bytes, 
 }
 
 // ---- key-norm scores -----------------------------------------------------------------------------
-// One thread per (token, KV head): s = sum_c x_c^2 accumulated in fp64 in increasing c.  Each
-// square of a bf16/fp32 value is exact in fp64, so only the summation order matters and it is
-// fixed here.  Output index: Hkv * off[n] + h * L_n + j.
 // s + x^2 for the two bf16 values packed in w, low half first; each square is exact in fp64.
 // (Widening by integer bit moves instead of the fp32->fp64 conversion, for all or for half of the
 // terms, was measured no faster: four integer instructions cost the integer pipe what one
@@ -238,8 +235,9 @@ topk_fused_kernel(const PartsParams pp, int hkv, int vpr /* 16-byte vectors per 
         // This CTA is done reading its peers; it may not exit before they are done reading it.  Arrive
         // now, wait at the very end: nothing after this touches distributed shared memory, and nobody
         // writes the keys a peer may still be reading.
+        __syncthreads();                                      // the collected keys, for this CTA's own threads; also
+                                                              // reconverges every warp for the aligned arrive
         asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-        __syncthreads();                                      // the collected keys, for this CTA's own threads
     }
 
     // ---- 3. selection ----
@@ -423,8 +421,8 @@ topk_fused_kernel(const PartsParams pp, int hkv, int vpr /* 16-byte vectors per 
 }
 
 cudaError_t launch_topk_fused(const PartsParams &pp, int hkv, int d, int dtype, void *k_agg, void *v_agg,
-                              int32_t *kv_pos, int32_t *cu_kv, int32_t *sel_idx_out, int sm_count, cudaStream_t s,
-                              int64_t *launches)
+                              int32_t *kv_pos, int32_t *cu_kv, int32_t *sel_idx_out, int device, int sm_count,
+                              cudaStream_t s, int64_t *launches)
 {
     if (pp.cu_kv[pp.n] == 0 && !cu_kv) return cudaSuccess;
     const int elt = dtype == FEDATTN_BF16 ? 2 : 4;
@@ -441,14 +439,14 @@ cudaError_t launch_topk_fused(const PartsParams &pp, int hkv, int d, int dtype, 
     int n_stages = (two_per_sm - fixed) / stage_bytes;
     n_stages = n_stages < 2 ? 2 : (n_stages > 4 ? 4 : n_stages);
     const int smem = fixed + n_stages * stage_bytes;
-    static bool attr_set = false;
-    if (!attr_set) {
+    static bool attr_set[64] = {};                            // the attribute is per device
+    if (!attr_set[device & 63]) {
         const int most = 227 * 1024 - 2048;
         cudaError_t e = cudaFuncSetAttribute(topk_fused_kernel<FEDATTN_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
         if (e == cudaSuccess)
             e = cudaFuncSetAttribute(topk_fused_kernel<FEDATTN_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
         if (e != cudaSuccess) return e;
-        attr_set = true;
+        attr_set[device & 63] = true;
     }
     // slices per (head, participant): a power of two <= 8 (one cluster), about two CTAs per SM in total
     const int pairs = hkv * pp.n;
@@ -493,9 +491,11 @@ gather_kernel(const PartsParams pp, int hkv, int64_t vpr /* 16-byte vectors per 
         const int n = find_segment(pp.cu_kv, pp.n, t);
         const int32_t j = sel_idx[rowid];
         const int32_t len = pp.off[n + 1] - pp.off[n];
-        if (j < 0 || j >= len) {
+        // in range, and strictly above its predecessor inside the same (head, participant) block: the
+        // aggregate's positions must come out ascending, which the attention over it relies on
+        if (j < 0 || j >= len || (t > pp.cu_kv[n] && sel_idx[rowid - 1] >= j)) {
             if (vi == 0) atomicMax(status, (int32_t)FEDATTN_ERR_INDEX);
-            continue;
+            if (j < 0 || j >= len) continue;
         }
         const uint4 *src = reinterpret_cast<const uint4 *>(is_v ? pp.v[n] : pp.k[n]) +
                            ((int64_t)j * hkv + h) * vpr + vi;
@@ -510,12 +510,12 @@ gather_kernel(const PartsParams pp, int hkv, int64_t vpr /* 16-byte vectors per 
 
 cudaError_t launch_gather(const PartsParams &pp, int hkv, int d, int elt_bytes, const int32_t *sel_idx,
                           void *k_agg, void *v_agg, int32_t *kv_pos, int32_t *cu_kv, int32_t *sel_idx_out,
-                          int32_t *status, cudaStream_t s, int64_t *launches)
+                          int32_t *status, int sm_count, cudaStream_t s, int64_t *launches)
 {
     const int64_t vpr = (int64_t)d * elt_bytes / 16;
     const int64_t total = (int64_t)hkv * pp.cu_kv[pp.n] * vpr;
     int64_t blocks = (total + 255) / 256;
-    if (blocks > 148 * 16) blocks = 148 * 16;
+    if (blocks > (int64_t)sm_count * 16) blocks = (int64_t)sm_count * 16;
     if (blocks < 1) blocks = 1;
     gather_kernel<<<dim3((unsigned)blocks, 2), 256, 0, s>>>(pp, hkv, vpr, sel_idx, (uint4 *)k_agg, (uint4 *)v_agg,
                                                             kv_pos, cu_kv, sel_idx_out, status);

@@ -37,12 +37,6 @@ inline int elt_bytes(const fedattn_shape *s) { return s->dtype == FEDATTN_BF16 ?
 
 inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
-size_t topk_scratch_bytes(int hkv, int64_t tokens)
-{
-    return align_up((size_t)hkv * (size_t)tokens * sizeof(double), 256) +
-           align_up((size_t)hkv * (size_t)tokens * sizeof(int32_t), 256);
-}
-
 struct DeviceGuard {
     int prev = -1;
     bool ok = true;
@@ -68,7 +62,8 @@ const char *fedattn_status_string(fedattn_status s)
     case FEDATTN_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
     case FEDATTN_ERR_CUDA: return "CUDA call failed";
     case FEDATTN_ERR_TIMEOUT: return "a bounded in-kernel wait ran out";
-    case FEDATTN_ERR_INDEX: return "selection index out of range";
+    case FEDATTN_ERR_INDEX: return "selection index out of range or not ascending";
+    case FEDATTN_ERR_ORDER: return "key positions not in non-decreasing order";
     }
     return "unknown status";
 }
@@ -76,10 +71,11 @@ const char *fedattn_status_string(fedattn_status s)
 size_t fedattn_workspace_bytes(const fedattn_shape *shape, int64_t max_total_tokens, int64_t max_total_kv)
 {
     if (!shape_ok(shape) || max_total_tokens < 0 || max_total_kv < 0) return 0;
-    size_t need = topk_scratch_bytes(shape->n_kv_heads, max_total_tokens > max_total_kv ? max_total_tokens
-                                                                                        : max_total_kv);
-    const size_t dec = decode_scratch_bytes(shape->n_participants, shape->n_q_heads, shape->head_dim, 0);
-    if (dec > need) need = dec;
+    // scratch, shared by calls that are ordered on one stream: the split-KV partials of the decode
+    // kernel, or the position tables of a sync call with explicit query positions
+    size_t need = decode_scratch_bytes(shape->n_participants, shape->n_q_heads, shape->head_dim, 0);
+    const size_t tab = position_table_bytes(shape->n_kv_heads, max_total_tokens, max_total_kv);
+    if (tab > need) need = tab;
     return kStatusBytes + align_up(need, 256);
 }
 
@@ -106,6 +102,7 @@ fedattn_status fedattn_create(fedattn_ctx **out, int device, void *workspace, si
     c.scratch = c.workspace + kStatusBytes;
     c.scratch_bytes = workspace_bytes - kStatusBytes;
     c.launches = 0;
+    c.tc_launches = 0;
     c.encode_tiled = nullptr;
     if (prop.major == 10) {
         void *fn = nullptr;
@@ -125,6 +122,18 @@ fedattn_status fedattn_create(fedattn_ctx **out, int device, void *workspace, si
 void fedattn_destroy(fedattn_ctx *ctx) { delete ctx; }
 
 int64_t fedattn_launch_count(const fedattn_ctx *ctx) { return ctx ? ctx->c.launches : 0; }
+
+int64_t fedattn_tensor_core_launch_count(const fedattn_ctx *ctx) { return ctx ? ctx->c.tc_launches : 0; }
+
+fedattn_status fedattn_selftest_wait_timeout(fedattn_ctx *ctx, int32_t max_polls, fedattn_stream stream)
+{
+    if (!ctx || max_polls < 1 || max_polls > 65536) return FEDATTN_ERR_INVALID_ARG;
+    if (!prefill_sm100_supported(&ctx->c)) return FEDATTN_ERR_UNSUPPORTED;
+    DeviceGuard g(ctx->c.device);
+    if (!g.ok) return FEDATTN_ERR_CUDA;
+    return launch_wait_selftest(&ctx->c, max_polls, static_cast<cudaStream_t>(stream)) == cudaSuccess ? FEDATTN_OK
+                                                                                                       : FEDATTN_ERR_CUDA;
+}
 
 fedattn_status fedattn_poll(fedattn_ctx *ctx, fedattn_stream stream)
 {
@@ -165,7 +174,7 @@ fedattn_status fedattn_local(fedattn_ctx *ctx, const fedattn_shape *shape, const
         p.scale = eff_scale(shape); p.causal = shape->causal; p.sync = 0; p.kv_head_major = 0;
         p.kv_pos = nullptr; p.n_seg = N;
         memcpy(p.cu, cu, sizeof(int32_t) * (N + 1));
-        err = launch_prefill_sm100(&ctx->c, p, s, &ctx->c.launches);
+        err = launch_prefill_sm100(&ctx->c, p, s);
     } else {
         GenericParams p;
         memset(&p, 0, sizeof(p));
@@ -227,18 +236,18 @@ fedattn_status fedattn_aggregate_kv(fedattn_ctx *ctx, const fedattn_shape *shape
         return err == cudaSuccess ? FEDATTN_OK : FEDATTN_ERR_CUDA;
     }
     if (mode == FEDATTN_AGG_TOPK_KNORM) {
-        err = launch_topk_fused(pp, hkv, d, shape->dtype, k_agg, v_agg, kv_pos, cu_kv, sel_idx_out, ctx->c.sm_count, s,
-                                &ctx->c.launches);
+        err = launch_topk_fused(pp, hkv, d, shape->dtype, k_agg, v_agg, kv_pos, cu_kv, sel_idx_out, ctx->c.device,
+                                ctx->c.sm_count, s, &ctx->c.launches);
         return err == cudaSuccess ? FEDATTN_OK : FEDATTN_ERR_CUDA;
     }
     if (mode == FEDATTN_AGG_TOPK_TOKEN) {
         // the per-head kernel on the token row viewed as one head of Hkv * d channels: token-major output
-        err = launch_topk_fused(pp, 1, hkv * d, shape->dtype, k_agg, v_agg, kv_pos, cu_kv, sel_idx_out, ctx->c.sm_count, s,
-                                &ctx->c.launches);
+        err = launch_topk_fused(pp, 1, hkv * d, shape->dtype, k_agg, v_agg, kv_pos, cu_kv, sel_idx_out, ctx->c.device,
+                                ctx->c.sm_count, s, &ctx->c.launches);
         return err == cudaSuccess ? FEDATTN_OK : FEDATTN_ERR_CUDA;
     }
     const int32_t *sel = sel_idx_in;
-    err = launch_gather(pp, hkv, d, eb, sel, k_agg, v_agg, kv_pos, cu_kv, sel_idx_out, ctx->c.status, s,
+    err = launch_gather(pp, hkv, d, eb, sel, k_agg, v_agg, kv_pos, cu_kv, sel_idx_out, ctx->c.status, ctx->c.sm_count, s,
                         &ctx->c.launches);
     return err == cudaSuccess ? FEDATTN_OK : FEDATTN_ERR_CUDA;
 }
@@ -257,8 +266,7 @@ fedattn_status fedattn_sync(fedattn_ctx *ctx, const fedattn_shape *shape, const 
     if (!g.ok) return FEDATTN_ERR_CUDA;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     cudaError_t err;
-    if (shape->dtype == FEDATTN_BF16 && shape->head_dim == 128 && !q_pos && total_kv > 0 &&
-        prefill_sm100_supported(&ctx->c)) {
+    if (shape->dtype == FEDATTN_BF16 && shape->head_dim == 128 && total_kv > 0 && prefill_sm100_supported(&ctx->c)) {
         PrefillParams p;
         memset(&p, 0, sizeof(p));
         p.q = q; p.k = k_agg; p.v = v_agg; p.o = o; p.lse = lse;
@@ -266,8 +274,14 @@ fedattn_status fedattn_sync(fedattn_ctx *ctx, const fedattn_shape *shape, const 
         p.hq = shape->n_q_heads; p.hkv = shape->n_kv_heads;
         p.scale = eff_scale(shape); p.causal = shape->causal; p.sync = 1; p.kv_head_major = kv_head_major;
         p.kv_pos = kv_pos; p.n_seg = 1;
+        if (q_pos && shape->causal) {
+            // explicit query positions: every (query, key) pair is tested on its own positions, in any order
+            if (ctx->c.scratch_bytes < position_table_bytes(p.hkv, n_q_rows, total_kv)) return FEDATTN_ERR_WORKSPACE;
+            p.general = 1; p.q_pos = q_pos;
+            p.tab = reinterpret_cast<int32_t *>(ctx->c.scratch);
+        }
         p.cu[0] = 0; p.cu[1] = (int32_t)n_q_rows;
-        err = launch_prefill_sm100(&ctx->c, p, s, &ctx->c.launches);
+        err = launch_prefill_sm100(&ctx->c, p, s);
     } else {
         GenericParams p;
         memset(&p, 0, sizeof(p));
@@ -295,7 +309,6 @@ fedattn_status fedattn_sync_remote(fedattn_ctx *ctx, const fedattn_shape *shape,
 {
     if (!ctx || !shape_ok(shape) || !cu || total_kv < 0 || total_kv > 0x7fffffffLL) return FEDATTN_ERR_INVALID_ARG;
     if (kv_head_major != 0 && kv_head_major != 1) return FEDATTN_ERR_INVALID_ARG;
-    if (!shape->causal) return FEDATTN_ERR_UNSUPPORTED;       // "before the segment" needs the causal order
     const int N = shape->n_participants;
     if (cu[0] != 0) return FEDATTN_ERR_INVALID_ARG;
     for (int n = 0; n < N; ++n)
@@ -314,16 +327,16 @@ fedattn_status fedattn_sync_remote(fedattn_ctx *ctx, const fedattn_shape *shape,
         p.q = q; p.k = k_agg; p.v = v_agg; p.o = o; p.lse = lse;
         p.n_q_rows = L; p.total_kv = total_kv;
         p.hq = shape->n_q_heads; p.hkv = shape->n_kv_heads;
-        p.scale = eff_scale(shape); p.causal = 1; p.sync = 1; p.remote_only = 1; p.kv_head_major = kv_head_major;
+        p.scale = eff_scale(shape); p.causal = shape->causal; p.sync = 1; p.remote_only = 1; p.kv_head_major = kv_head_major;
         p.kv_pos = kv_pos; p.n_seg = N;
         memcpy(p.cu, cu, sizeof(int32_t) * (N + 1));
-        err = launch_prefill_sm100(&ctx->c, p, s, &ctx->c.launches);
+        err = launch_prefill_sm100(&ctx->c, p, s);
     } else {
         GenericParams p;
         memset(&p, 0, sizeof(p));
         p.q = q; p.k = k_agg; p.v = v_agg; p.o = o; p.lse = lse;
         p.n_rows = L; p.hq = shape->n_q_heads; p.hkv = shape->n_kv_heads; p.d = shape->head_dim;
-        p.scale = eff_scale(shape); p.causal = 1; p.mode = kSync; p.remote_only = 1;
+        p.scale = eff_scale(shape); p.causal = shape->causal; p.mode = kSync; p.remote_only = 1;
         if (kv_head_major) {
             p.kv_tok_stride = shape->head_dim;
             p.kv_head_stride = total_kv * shape->head_dim;
@@ -352,7 +365,7 @@ fedattn_status fedattn_merge(fedattn_ctx *ctx, const fedattn_shape *shape, int64
     DeviceGuard g(ctx->c.device);
     if (!g.ok) return FEDATTN_ERR_CUDA;
     cudaError_t err = launch_merge(shape->dtype, n_rows, shape->n_q_heads, shape->head_dim, o_a, lse_a, o_b, lse_b, o, lse,
-                                   static_cast<cudaStream_t>(stream), &ctx->c.launches);
+                                   ctx->c.sm_count, static_cast<cudaStream_t>(stream), &ctx->c.launches);
     return err == cudaSuccess ? FEDATTN_OK : FEDATTN_ERR_CUDA;
 }
 

@@ -38,6 +38,8 @@ attn_generic_kernel(const GenericParams p)
     int64_t pos = p.q_pos ? p.q_pos[row] : row;
     int64_t kv_base = (int64_t)kvh * p.kv_head_stride;
     bool test_pos = p.causal != 0;
+    int64_t own_lo = 0, own_hi = 0;                  // remote-only, bidirectional: positions of the row's own segment
+    bool test_own = false;
     if (p.mode == kLocal) {
         int n = 0;
         while (n + 1 < p.n_seg && row >= p.cu[n + 1]) ++n;
@@ -45,10 +47,15 @@ attn_generic_kernel(const GenericParams p)
         kv_hi = p.causal ? row + 1 : (int64_t)p.cu[n + 1];
         test_pos = false;
     } else if (p.mode == kSync) {
-        if (p.remote_only) {                         // position = last one before the row's own segment
+        if (p.remote_only) {
             int n = 0;
             while (n + 1 < p.n_seg && row >= p.cu[n + 1]) ++n;
-            pos = (int64_t)p.cu[n] - 1;
+            if (p.causal) {
+                pos = (int64_t)p.cu[n] - 1;          // position = last one before the row's own segment
+            } else {                                 // everything positioned outside the row's own segment
+                own_lo = p.cu[n]; own_hi = p.cu[n + 1];
+                test_own = true;
+            }
         }
         kv_hi = p.total_kv;
         if (p.causal && !p.kv_pos) {                 // identity positions: a prefix
@@ -81,6 +88,10 @@ attn_generic_kernel(const GenericParams p)
         const int64_t j = j0 + lane;
         bool ok = j < kv_hi;
         if (ok && test_pos) ok = (int64_t)(kvp ? kvp[j] : j) <= pos;
+        if (ok && test_own) {
+            const int64_t pj = kvp ? kvp[j] : j;
+            ok = pj < own_lo || pj >= own_hi;
+        }
         float s = -INFINITY;
         if (ok) {
             const T *kr = K + j * p.kv_tok_stride;

@@ -27,6 +27,7 @@ struct Context {
     char *scratch;         // dev, workspace + kStatusBytes
     size_t scratch_bytes;
     int64_t launches;
+    int64_t tc_launches;   // launches of the tcgen05 attention kernel among them
     void *encode_tiled;    // cuTensorMapEncodeTiled entry point (driver), or nullptr
 };
 
@@ -42,7 +43,8 @@ struct GenericParams {
     float scale;
     int32_t causal;
     int32_t mode;                 // GenericMode
-    int32_t remote_only;          // kSync: a row's position is the last one before its segment (cu)
+    int32_t remote_only;          // kSync: a row sees the keys positioned before its segment (cu) and, when
+                                  // causal == 0, those positioned after it
     int64_t kv_tok_stride;        // elements between consecutive KV rows of one head
     int64_t kv_head_stride;       // elements between KV heads
     int64_t kv_pos_head_stride;   // ints between heads in kv_pos (0 = shared)
@@ -70,11 +72,11 @@ cudaError_t launch_concat(const PartsParams &pp, int hkv, int d, int elt_bytes, 
                           int32_t *kv_pos, int32_t *cu_kv, cudaStream_t s, int sm_count, int64_t *launches);
 
 cudaError_t launch_topk_fused(const PartsParams &pp, int hkv, int d, int dtype, void *k_agg, void *v_agg,
-                              int32_t *kv_pos, int32_t *cu_kv, int32_t *sel_idx_out, int sm_count, cudaStream_t s,
-                              int64_t *launches);
+                              int32_t *kv_pos, int32_t *cu_kv, int32_t *sel_idx_out, int device, int sm_count,
+                              cudaStream_t s, int64_t *launches);
 cudaError_t launch_gather(const PartsParams &pp, int hkv, int d, int elt_bytes, const int32_t *sel_idx,
                           void *k_agg, void *v_agg, int32_t *kv_pos, int32_t *cu_kv, int32_t *sel_idx_out,
-                          int32_t *status, cudaStream_t s, int64_t *launches);
+                          int32_t *status, int sm_count, cudaStream_t s, int64_t *launches);
 
 // ---- bf16 prefill on tensor cores (tcgen05 + TMEM + TMA), head_dim 128 ------------------------
 struct PrefillParams {
@@ -87,18 +89,26 @@ struct PrefillParams {
     float scale;
     int32_t causal;
     int32_t sync;                 // 0 local, 1 sync
-    int32_t remote_only;          // sync: a row sees the aggregated rows positioned before its segment
+    int32_t remote_only;          // sync: a row sees the aggregated rows positioned before its segment (and, when
+                                  // causal == 0, those positioned after it)
     int32_t kv_head_major;
     const int32_t *kv_pos;        // nullable
+    int32_t general;              // sync, causal: every (query, key) pair is tested on explicit positions
+    const int32_t *q_pos;         // general: nullable (= row index)
+    int32_t *tab;                 // general: scratch for the position tables (position_table_bytes)
     int32_t n_seg;
     int32_t cu[kMaxP + 1];        // query segments (local: also the KV segments)
 };
 bool prefill_sm100_supported(const Context *ctx);
-cudaError_t launch_prefill_sm100(const Context *ctx, const PrefillParams &p, cudaStream_t s, int64_t *launches);
+// scratch bytes of the per-tile position tables of a general-position sync call
+size_t position_table_bytes(int hkv, int64_t n_q_rows, int64_t total_kv);
+cudaError_t launch_prefill_sm100(Context *ctx, const PrefillParams &p, cudaStream_t s);
+// one small kernel whose bounded wait runs out after max_polls polls (raises FEDATTN_ERR_TIMEOUT)
+cudaError_t launch_wait_selftest(Context *ctx, int max_polls, cudaStream_t s);
 
 // ---- merge of two partial attention results through their log-sum-exps ----------------------
 cudaError_t launch_merge(int dtype, int64_t n_rows, int hq, int d, const void *o_a, const float *lse_a, const void *o_b,
-                         const float *lse_b, void *o, float *lse, cudaStream_t s, int64_t *launches);
+                         const float *lse_b, void *o, float *lse, int sm_count, cudaStream_t s, int64_t *launches);
 
 // ---- bf16 split-KV decode (tensor-core scores, warp-shuffle softmax) ---------------------------
 struct DecodeParams {

@@ -489,7 +489,6 @@ static cudaError_t launch_decode_split(const DecodeParams &p_in, int sm_count, i
     const int n_chunks = (rows_total + 16 * m_tiles - 1) / (16 * m_tiles);
     const int caches = p.sync ? 1 : p.n_part;
     const int sources = caches * p.hkv * n_chunks;
-    if (sources * kMaxCluster > kDecodeCounters) return cudaErrorInvalidValue;
     const int tiles = (p.max_kv_len + kTileKeys - 1) / kTileKeys;
     int n_splits = 2 * sm_count / sources;                     // rounded down: one wave
     if (n_splits > tiles / 2) n_splits = tiles / 2;            // at least two tiles per split
@@ -499,6 +498,9 @@ static cudaError_t launch_decode_split(const DecodeParams &p_in, int sm_count, i
     int ncl = n_splits / cs;
     if (ncl > max_slots) ncl = max_slots;
     if (ncl > kMaxSlots) ncl = kMaxSlots;
+    // several clusters per source meet through the arrival counters (kMaxCluster per source); with more
+    // sources than counters every source keeps to one cluster, which needs none
+    if (ncl > 1 && (int64_t)sources * kMaxCluster > kDecodeCounters) ncl = 1;
     n_splits = ncl * cs;
     if (ncl > 1 && (size_t)p.n_part * p.hq * ncl * kPartialStride * sizeof(float) > p.partial_bytes)
         return cudaErrorInvalidValue;

@@ -60,12 +60,12 @@ merge_kernel(int64_t n_items /* rows * hq * d / 8 */, int d8, const T *o_a, cons
 }
 
 cudaError_t launch_merge(int dtype, int64_t n_rows, int hq, int d, const void *o_a, const float *lse_a, const void *o_b,
-                         const float *lse_b, void *o, float *lse, cudaStream_t s, int64_t *launches)
+                         const float *lse_b, void *o, float *lse, int sm_count, cudaStream_t s, int64_t *launches)
 {
     const int64_t n_items = n_rows * hq * (d / 8);
     if (n_items == 0) return cudaSuccess;
     int64_t blocks = (n_items + 255) / 256;
-    if (blocks > 148 * 16) blocks = 148 * 16;
+    if (blocks > (int64_t)sm_count * 16) blocks = (int64_t)sm_count * 16;
     if (dtype == FEDATTN_BF16)
         merge_kernel<__nv_bfloat16><<<(unsigned)blocks, 256, 0, s>>>(n_items, d / 8, (const __nv_bfloat16 *)o_a, lse_a,
                                                                      (const __nv_bfloat16 *)o_b, lse_b, (__nv_bfloat16 *)o, lse);

@@ -77,8 +77,26 @@ struct KernelParams {
     uint64_t magic_per_tile, magic_ppg, magic_small[kMaxP];   // ceil(2^40 / d) for d = per_tile, ppg, 1..kMaxP
     int32_t n_qtiles;                // total query tiles
     int32_t n_items;                 // query tiles x KV heads x head pairs
+    int32_t n_kt;                    // KV tiles: ceil(total_kv / kTileN)
     int32_t *status;
 };
+
+// Position tables of a general-position call (ints, in this order): minimum and maximum position of
+// every query tile; then per KV position array (one per KV head when head-major, else one) the
+// running minimum over the tiles j, j+1, ... (suffix minimum) and the running maximum over the tiles
+// 0 .. j (prefix maximum) of the tile's key positions.  Both runs are monotone in j, so "tiles that
+// can hold a visible key" and "tiles whose keys are all visible" are prefixes found by bisection.
+// A ragged last KV tile counts as never fully visible (maximum = INT_MAX).
+struct PosTables {
+    const int32_t *q_min, *q_max, *suf_min, *pre_max;
+};
+__device__ __host__ __forceinline__ PosTables pos_tables(const int32_t *tab, int n_qtiles, int n_arrays, int n_kt)
+{
+    PosTables t;
+    t.q_min = tab; t.q_max = tab + n_qtiles;
+    t.suf_min = tab + 2 * (size_t)n_qtiles; t.pre_max = t.suf_min + (size_t)n_arrays * n_kt;
+    return t;
+}
 
 #ifdef FEDATTN_TRACE
 // Debug build only: cycle stamps of one CTA's pipeline events, [tile][event].
@@ -123,10 +141,11 @@ __device__ __forceinline__ bool mbar_test_wait(uint64_t *bar, uint32_t parity)
                  : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
     return ok != 0;
 }
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag, int32_t *status)
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag, int32_t *status,
+                                          uint32_t limit = kWaitLimit)
 {
     if (mbar_test_wait(bar, parity)) return true;        // phase already over: skip the suspending wait
-    for (uint32_t it = 0; it < kWaitLimit; ++it) {
+    for (uint32_t it = 0; it < limit; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
     }
@@ -321,9 +340,13 @@ __device__ __forceinline__ int count_le(const int32_t *pos, int n, int x)
 // One unit of work: a 128-row query tile x one pair of query heads that share a KV head.
 struct Item {
     int kvh, head0, q_row0, n_valid, seg, kv_begin, n_tiles;
+    // The walk visits KV tiles 0 .. n_a-1 and then t_b0, t_b0+1, ...  (n_a == n_tiles unless the allowed
+    // keys are two ranges: bidirectional remote-only attention, keys [0, a) and [b, T)).
+    int n_a, t_b0, a, b;
     bool valid1;                       // the pair's second head exists (odd group size: last pair is single)
     const int32_t *kvp;                // positions of this KV head's aggregated rows (sparse sync), or null
 };
+__device__ __forceinline__ int tile_of(const Item &it, int j) { return j < it.n_a ? j : it.t_b0 + (j - it.n_a); }
 
 // allowed-prefix length c(row): keys kv_begin .. kv_begin + c - 1 are visible to query row r of the tile
 __device__ __forceinline__ int prefix_len(const PrefillParams &p, const Item &it, int r)
@@ -334,11 +357,11 @@ __device__ __forceinline__ int prefix_len(const PrefillParams &p, const Item &it
         const int seg_len = p.cu[it.seg + 1] - p.cu[it.seg];
         return p.causal ? min(pos - p.cu[it.seg] + 1, seg_len) : seg_len;
     }
-    if (!p.causal) return T;
     if (p.remote_only) {                               // what lies before the row's own segment
         const int before = p.cu[it.seg];
         return it.kvp ? count_le(it.kvp, T, before - 1) : min(before, T);
     }
+    if (!p.causal) return T;
     if (!it.kvp) return min(pos + 1, T);
     return count_le(it.kvp, T, pos);
 }
@@ -374,7 +397,26 @@ __device__ __forceinline__ Item decode_item(const KernelParams &kp, int item)
     it.n_valid = min(kTileM, p.cu[seg + 1] - it.q_row0);
     it.kvp = p.kv_pos ? p.kv_pos + (p.kv_head_major ? (int64_t)it.kvh * p.total_kv : 0) : nullptr;
     it.kv_begin = p.sync ? 0 : p.cu[seg];
-    it.n_tiles = (prefix_len(p, it, it.n_valid - 1) + kTileN - 1) / kTileN;
+    it.t_b0 = 0; it.a = 0; it.b = 0;
+    if (p.general) {
+        // tiles up to the last one that holds a key position <= the tile's largest query position
+        const PosTables pt = pos_tables(p.tab, kp.n_qtiles, p.kv_head_major ? p.hkv : 1, kp.n_kt);
+        const int32_t *suf = pt.suf_min + (p.kv_head_major ? (size_t)it.kvh * kp.n_kt : 0);
+        it.n_tiles = count_le(suf, kp.n_kt, __ldg(pt.q_max + (it.q_row0 >> 7)));
+        it.n_a = it.n_tiles;
+    } else if (p.sync && p.remote_only && !p.causal) {
+        // keys [0, a) lie before the row's segment, keys [b, T) after it
+        const int T = (int)p.total_kv, n_t = (T + kTileN - 1) / kTileN;
+        it.a = prefix_len(p, it, 0);
+        const int after = p.cu[seg + 1];
+        it.b = it.kvp ? count_le(it.kvp, T, after - 1) : min(after, T);
+        it.n_a = (it.a + kTileN - 1) / kTileN;
+        it.t_b0 = it.b >= T ? n_t : max(it.b / kTileN, it.n_a);
+        it.n_tiles = it.n_a + (n_t - it.t_b0);
+    } else {
+        it.n_tiles = (prefix_len(p, it, it.n_valid - 1) + kTileN - 1) / kTileN;
+        it.n_a = it.n_tiles;
+    }
     return it;
 }
 
@@ -404,7 +446,6 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int n_items = kp.n_items;
-    const int n_rounds = (n_items + (int)gridDim.x - 1) / (int)gridDim.x;
     // Static schedule: round k hands item k*G + c to CTA c, in reversed CTA order on odd rounds, so
     // that with items sorted by cost every CTA gets a similar total.
     auto item_of = [&](int k) -> int {
@@ -432,6 +473,9 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    // A timeout that an earlier kernel reported and nobody has polled yet: this launch does no work
+    // (every wait would run out again) and leaves its outputs untouched.
+    const int n_rounds = *abort_flag ? 0 : (n_items + (int)gridDim.x - 1) / (int)gridDim.x;
 
     // every warp of a warpgroup executes the same setmaxnreg (first thing in its role); the increase
     // waits for the decrease
@@ -458,7 +502,7 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                 }
                 for (int j = 0; j < it.n_tiles; ++j) {
                     const int gt = git + j, st = gt & 1, use = gt >> 1;
-                    const int row = it.kv_begin + j * kTileN;
+                    const int row = it.kv_begin + tile_of(it, j) * kTileN;
                     const int c1 = p.kv_head_major ? row : it.kvh, c2 = p.kv_head_major ? it.kvh : row;
                     if (gt >= 2) mbar_wait(k_empty + st, (use - 1) & 1, abort_flag, kp.status);
                     TRACE(j, 7);
@@ -566,6 +610,17 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         }
     } else if (warp >= 4 * kSplit) {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kOtherRegs));      // the two idle warps of that warpgroup
+        // One of them checks what the prefix-count mask relies on: key positions that never decrease
+        // along the aggregated rows of a head.  The CTAs share the pairs (i, i + 1) among them.
+        if (warp == kMmaWarp + 1 && p.kv_pos && !p.general && p.sync && (p.causal || p.remote_only) && p.total_kv > 1) {
+            const int64_t per = p.total_kv - 1, total = per * (p.kv_head_major ? p.hkv : 1);
+            bool bad = false;
+            for (int64_t i = (int64_t)blockIdx.x * 32 + lane; i < total; i += (int64_t)gridDim.x * 32) {
+                const int64_t a = i / per, e = a * p.total_kv + (i - a * per);
+                bad |= __ldg(p.kv_pos + e) > __ldg(p.kv_pos + e + 1);
+            }
+            if (bad) atomicMax(kp.status, (int32_t)FEDATTN_ERR_ORDER);
+        }
     } else {
         asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kSoftmaxRegs));
         // ================= softmax + epilogue =================
@@ -587,12 +642,17 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         auto wg_sync = [&]() { asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "n"(32 * kSplit) : "memory"); };
         const bool o_aligned32 = (reinterpret_cast<uintptr_t>(p.o) & 31) == 0;
 
-        // One visit = the softmax of one S tile of one sub-tile.  kPartial: some row of the tile has masked
-        // columns (they become -inf and every exponential goes through ex2.approx, which maps -inf to 0);
-        // otherwise a fixed subset of the columns takes the polynomial so that the ex2 unit, which is as
-        // slow as the tensor pipe for this tile shape, is not the bottleneck.
-        auto visit = [&](auto partial_tag, int t, int j, int gt, int lim, float &m_used, float &l) {
-            constexpr bool kPartial = decltype(partial_tag)::value;
+        // One visit = the softmax of one S tile of one sub-tile.  Mask kinds: 0 none (every key of the tile
+        // is visible to every row); 1 prefix (this thread's columns c < a0 are visible); 2 two ranges
+        // (c < a0, or a1 <= c < a2); 3 explicit positions (column c is key a1 + c, visible iff it exists and
+        // its position is <= a0 = the row's position).  Masked columns become -inf and every exponential of
+        // a masked tile goes through ex2.approx, which maps -inf to 0; in unmasked tiles a fixed subset of
+        // the columns takes the polynomial so that the ex2 unit, which is as slow as the tensor pipe for this
+        // tile shape, is not the bottleneck.
+        auto visit = [&](auto mask_tag, int t, int j, int gt, int a0, int a1, int a2, const int32_t *kvp, float &m_used,
+                         float &l) {
+            constexpr int kMask = decltype(mask_tag)::value;
+            constexpr bool kPartial = kMask != 0;
             const uint32_t tS = tmem_base + lane_base + kColS + t * 128 + kCols * hf;   // fp32 S, this part
             const uint32_t tP = tS;                                                      // bf16 P, this part
             const uint32_t tO = tmem_base + lane_base + kColO + t * 128 + kCols * hf;
@@ -603,10 +663,22 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
 #pragma unroll
             for (int c = 0; c < kCols; c += 32) FEDATTN_TMEM_LD32(tS + c, (s + c));
             tmem_wait_ld();
-            if (kPartial) {
+            if (kMask == 1) {
 #pragma unroll
                 for (int c = 0; c < kCols; ++c)
-                    if (c >= lim) s[c] = 0xff800000u;           // -inf; columns < lim are visible
+                    if (c >= a0) s[c] = 0xff800000u;            // -inf; columns < a0 are visible
+            } else if (kMask == 2) {
+#pragma unroll
+                for (int c = 0; c < kCols; ++c)
+                    if (c >= a0 && !(c >= a1 && c < a2)) s[c] = 0xff800000u;
+            } else if (kMask == 3) {
+                const int T = (int)p.total_kv;
+#pragma unroll
+                for (int c = 0; c < kCols; ++c) {
+                    const int key = a1 + c;                     // the same address in every lane: one broadcast load
+                    const int kpos = kvp ? __ldg(kvp + min(key, T - 1)) : key;
+                    if (key >= T || kpos > a0) s[c] = 0xff800000u;
+                }
             }
             // partial row maximum: 8 independent chains, then a tree
             float mx[8];
@@ -701,11 +773,24 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                 }
                 continue;
             }
-            const int c_row = prefix_len(p, it, r);
+            const bool two_range = p.sync && p.remote_only && !p.causal;
+            int c_row = 0, n_full = 0, p_row = 0;
+            if (p.general) {
+                // every (query, key) pair on its own positions; the tiles whose keys all lie at or below the
+                // tile's smallest query position (a prefix of the walk, see PosTables) need no test
+                const PosTables pt = pos_tables(p.tab, kp.n_qtiles, p.kv_head_major ? p.hkv : 1, kp.n_kt);
+                const int32_t *pre = pt.pre_max + (p.kv_head_major ? (size_t)it.kvh * kp.n_kt : 0);
+                n_full = count_le(pre, kp.n_kt, __ldg(pt.q_min + (it.q_row0 >> 7)));
+                const int row = it.q_row0 + min(r, it.n_valid - 1);
+                p_row = p.q_pos ? __ldg(p.q_pos + row) : row;
+            } else {
+                c_row = prefix_len(p, it, r);
+                // prefix lengths do not decrease with the row, so KV tiles below the prefix of the warp's first
+                // row are unmasked for the whole warp (the choice of code path only has to be warp-uniform)
+                n_full = __shfl_sync(0xffffffffu, c_row, 0) / kTileN;
+            }
             const int c_r = c_row - kCols * hf;                 // visible keys, counted from this thread's first column
-            // prefix lengths do not decrease with the row, so KV tiles below the prefix of the warp's first
-            // row are unmasked for the whole warp (the choice of code path only has to be warp-uniform)
-            const int n_full = __shfl_sync(0xffffffffu, c_row, 0) / kTileN;
+            const int T = (int)p.total_kv;
             // state of the sub-tile being visited (a) and of the other one (b); swapped after every visit
             float m_a = 0.f, l_a = 0.f, m_b = 0.f, l_b = 0.f;
             const int n_visits = n_tiles * n_sub;
@@ -713,8 +798,20 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                 const int t = n_sub == 2 ? (v & 1) : 0;
                 const int j = n_sub == 2 ? (v >> 1) : v;
                 const int gt = (t ? gsub1 : gsub0) + j;
-                if (j < n_full) visit(std::false_type{}, t, j, gt, kCols, m_a, l_a);
-                else visit(std::true_type{}, t, j, gt, c_r - j * kTileN, m_a, l_a);
+                if (two_range) {
+                    const int k0 = tile_of(it, j) * kTileN;     // first key of the tile
+                    if (k0 + kTileN <= it.a || (k0 >= it.b && k0 + kTileN <= T))
+                        visit(std::integral_constant<int, 0>{}, t, j, gt, 0, 0, 0, nullptr, m_a, l_a);
+                    else
+                        visit(std::integral_constant<int, 2>{}, t, j, gt, c_r - k0, it.b - k0 - kCols * hf, T - k0 - kCols * hf,
+                              nullptr, m_a, l_a);
+                } else if (j < n_full) {
+                    visit(std::integral_constant<int, 0>{}, t, j, gt, 0, 0, 0, nullptr, m_a, l_a);
+                } else if (p.general) {
+                    visit(std::integral_constant<int, 3>{}, t, j, gt, p_row, j * kTileN + kCols * hf, 0, it.kvp, m_a, l_a);
+                } else {
+                    visit(std::integral_constant<int, 1>{}, t, j, gt, c_r - j * kTileN, 0, 0, nullptr, m_a, l_a);
+                }
                 if (n_sub == 2) {
                     float x = m_a; m_a = m_b; m_b = x;
                     x = l_a; l_a = l_b; l_b = x;
@@ -778,6 +875,100 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     }
 }
 
+// ---- position tables of a general-position call -------------------------------------------------------
+// grid: one block per KV position array (n_arrays of them), then one block for the query positions.
+// A warp reduces one 128-entry tile at a time (one 16-byte load per lane when the array allows it).  The
+// KV blocks then turn the per-tile values into the running suffix minimum / prefix maximum in place.
+constexpr int kTabThreads = 1024;
+
+__device__ __forceinline__ void tile_min_max(const int32_t *pos, int64_t n, int64_t tile, int lane, int &mn, int &mx)
+{
+    mn = INT32_MAX; mx = INT32_MIN;
+    const int64_t i0 = tile * kTileN + lane * 4;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const int64_t i = i0 + e;
+        if (i < n) {
+            const int v = pos ? __ldg(pos + i) : (int)i;
+            mn = min(mn, v); mx = max(mx, v);
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        mn = min(mn, __shfl_xor_sync(0xffffffffu, mn, o));
+        mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    }
+}
+
+__global__ void __launch_bounds__(kTabThreads)
+position_tables_kernel(const int32_t *q_pos, int64_t n_q, const int32_t *kv_pos, int64_t total_kv, int n_arrays,
+                       int n_qtiles, int n_kt, int32_t *tab)
+{
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, n_warps = kTabThreads / 32;
+    const PosTables pt = pos_tables(tab, n_qtiles, n_arrays, n_kt);
+    if ((int)blockIdx.x == n_arrays) {
+        int32_t *q_min = tab, *q_max = tab + n_qtiles;
+        for (int64_t t = warp; t < n_qtiles; t += n_warps) {
+            int mn, mx;
+            tile_min_max(q_pos, n_q, t, lane, mn, mx);
+            if (lane == 0) { q_min[t] = mn; q_max[t] = mx; }
+        }
+        return;
+    }
+    const int a = blockIdx.x;
+    const int32_t *pos = kv_pos ? kv_pos + (size_t)a * total_kv : nullptr;
+    int32_t *suf = const_cast<int32_t *>(pt.suf_min) + (size_t)a * n_kt, *pre = const_cast<int32_t *>(pt.pre_max) + (size_t)a * n_kt;
+    for (int64_t t = warp; t < n_kt; t += n_warps) {
+        int mn, mx;
+        tile_min_max(pos, total_kv, t, lane, mn, mx);
+        if ((t + 1) * kTileN > total_kv) mx = INT32_MAX;      // ragged tile: never fully visible
+        if (lane == 0) { suf[t] = mn; pre[t] = mx; }
+    }
+    __syncthreads();
+    if (warp == 0) {                                           // prefix maximum, 32 tiles per step
+        int carry = INT32_MIN;
+        for (int t0 = 0; t0 < n_kt; t0 += 32) {
+            int v = t0 + lane < n_kt ? pre[t0 + lane] : INT32_MIN;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int u = __shfl_up_sync(0xffffffffu, v, o);
+                if (lane >= o) v = max(v, u);
+            }
+            v = max(v, carry);
+            if (t0 + lane < n_kt) pre[t0 + lane] = v;
+            carry = __shfl_sync(0xffffffffu, v, 31);
+        }
+    } else if (warp == 1) {                                    // suffix minimum, from the last tile backwards
+        int carry = INT32_MAX;
+        for (int t0 = ((n_kt - 1) / 32) * 32; t0 >= 0; t0 -= 32) {
+            int v = t0 + lane < n_kt ? suf[t0 + lane] : INT32_MAX;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int u = __shfl_down_sync(0xffffffffu, v, o);
+                if (lane + o < 32) v = min(v, u);
+            }
+            v = min(v, carry);
+            if (t0 + lane < n_kt) suf[t0 + lane] = v;
+            carry = __shfl_sync(0xffffffffu, v, 0);
+        }
+    }
+}
+
+// ---- self-test of the bounded wait ---------------------------------------------------------------------
+// Waits with mbar_wait, the routine every role above waits with, on a barrier that nothing signals.
+__global__ void wait_selftest_kernel(int32_t *status, uint32_t max_polls)
+{
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    mbar_wait(&bar, 0, &abort_flag, status, max_polls);        // phase 0 never completes: runs out, flags the status
+}
+
 // ---- host ---------------------------------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
@@ -813,12 +1004,26 @@ static bool encode_map(const Context *ctx, CUtensorMap *map, const void *base, i
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-cudaError_t launch_prefill_sm100(const Context *ctx, const PrefillParams &p, cudaStream_t s, int64_t *launches)
+size_t position_table_bytes(int hkv, int64_t n_q_rows, int64_t total_kv)
+{
+    const int64_t n_qt = (n_q_rows + kTileM - 1) / kTileM, n_kt = (total_kv + kTileN - 1) / kTileN;
+    return (size_t)(2 * n_qt + 2 * (int64_t)hkv * n_kt) * sizeof(int32_t);
+}
+
+cudaError_t launch_wait_selftest(Context *ctx, int max_polls, cudaStream_t s)
+{
+    wait_selftest_kernel<<<1, 32, 0, s>>>(ctx->status, (uint32_t)max_polls);
+    ++ctx->launches;
+    return cudaGetLastError();
+}
+
+cudaError_t launch_prefill_sm100(Context *ctx, const PrefillParams &p, cudaStream_t s)
 {
     static_assert(sizeof(KernelParams) < 3000, "kernel parameter block too large");
     KernelParams kp;
     kp.p = p;
     kp.status = ctx->status;
+    kp.n_kt = (int32_t)((p.total_kv + kTileN - 1) / kTileN);
     int64_t n_qtiles = 0;
     for (int n = 0; n < p.n_seg; ++n) {
         kp.ord_seg[n] = n;
@@ -863,8 +1068,18 @@ cudaError_t launch_prefill_sm100(const Context *ctx, const PrefillParams &p, cud
         }
         attr_set[ctx->device & 63] = true;
     }
+    if (p.general) {
+        // the per-tile position tables first (same stream): the walk and the unmasked fast path read them
+        const int n_arrays = p.kv_head_major ? p.hkv : 1;
+        position_tables_kernel<<<n_arrays + 1, kTabThreads, 0, s>>>(p.q_pos, p.n_q_rows, p.kv_pos, p.total_kv, n_arrays,
+                                                                    kp.n_qtiles, kp.n_kt, p.tab);
+        ++ctx->launches;
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+    }
     prefill_sm100_kernel<<<(unsigned)blocks, kThreads, kSmemBytes, s>>>(mq, mk, mv, kp);
-    ++*launches;
+    ++ctx->launches;
+    ++ctx->tc_launches;
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess && getenv("FEDATTN_DEBUG")) fprintf(stderr, "prefill_sm100_kernel launch: %s\n", cudaGetErrorString(e));
     return e;

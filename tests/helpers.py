@@ -6,6 +6,7 @@ import numpy as np
 import torch
 
 TOL = {"f32": 1e-4, "bf16": 2e-2}     # max-abs bounds: fp32 inputs / bf16 inputs with O(1) outputs
+LSE_TOL = {"f32": 1e-4, "bf16": 1e-3}  # log-sum-exp (fp32 output): fp32 inputs / bf16 inputs
 
 
 def fa():

@@ -1,6 +1,6 @@
 """fedattn_decode_noalloc: the decode entry point for callers that cannot allocate device memory
 (no context, no workspace; its split-KV scratch is a fixed array inside the library).  It must give
-what fedattn_decode gives.  Two calls in a row with different inputs also show that whatever the
+what fedattn_decode gives, and what the fp64 oracle gives.  Two calls in a row with different inputs also show that whatever the
 previous call left in the shared scratch does not leak into the next result.  This file sorts
 last so that a run that stops at the first failure has already run every other test."""
 import numpy as np
@@ -13,7 +13,8 @@ from helpers import TOL, fa, host
 pytestmark = pytest.mark.gpu
 
 
-def _run_pair(m, shape, ctx, mode, q, k, v, stride, lens, max_len):
+def _run_pair(m, shape, ctx, mode, q, k, v, stride, lens, max_len, want):
+    """fedattn_decode_noalloc against fedattn_decode, and against the fp64 oracle's result `want`."""
     o_ref = torch.full_like(q, float("nan")); o_new = torch.full_like(q, float("nan"))
     lse_ref = torch.full(q.shape[:2], float("nan"), device="cuda"); lse_new = torch.full_like(lse_ref, float("nan"))
     m.fedattn_decode(ctx, shape, mode, q, k, v, stride, lens, max_len, o_ref, lse_ref)
@@ -23,9 +24,11 @@ def _run_pair(m, shape, ctx, mode, q, k, v, stride, lens, max_len):
     err = np.abs(host(o_new) - host(o_ref)).max()
     assert np.isfinite(host(o_new)).all() and err <= TOL["bf16"], err
     assert np.abs(host(lse_new) - host(lse_ref)).max() <= 1e-3
+    assert np.abs(host(o_new) - want[0]).max() <= TOL["bf16"]
+    assert np.abs(host(lse_new) - want[1]).max() <= 1e-3
 
 
-def test_noalloc_decode_matches_decode_twice_in_a_row():
+def test_noalloc_decode_matches_decode_twice_in_a_row(oracle):
     m = fa()
     n, cap, hq, hkv, d = 8, 1024, 32, 8, 128
     w = fi.Workload("noalloc", 21, (cap,) * n, hq, hkv, d, "bf16")
@@ -33,14 +36,18 @@ def test_noalloc_decode_matches_decode_twice_in_a_row():
     ctx = m.Context(shape, n * cap, n * cap)
     bf = torch.bfloat16
     for call in range(2):                       # second call: new K/V/q, shorter ragged lengths
-        _, k, v = w.qkv(block=call)
-        q = torch.from_numpy(w.decode_q(call)).to(bf).cuda()
-        k = torch.from_numpy(k).to(bf).cuda(); v = torch.from_numpy(v).to(bf).cuda()
+        _, kn, vn = w.qkv(block=call)
+        qn = w.decode_q(call)
+        q = torch.from_numpy(qn).to(bf).cuda()
+        k = torch.from_numpy(kn).to(bf).cuda(); v = torch.from_numpy(vn).to(bf).cuda()
         lens_l = [cap] * n if call == 0 else [cap - 37 * i for i in range(n)]
         lens = torch.tensor(lens_l, dtype=torch.int32, device="cuda")
-        _run_pair(m, shape, ctx, m.DECODE_LOCAL, q, k, v, cap * hkv * d, lens, cap)
-        tot = torch.tensor([n * cap - 100 * call], dtype=torch.int32, device="cuda")
-        _run_pair(m, shape, ctx, m.DECODE_SYNC, q, k, v, 0, tot, n * cap)
+        want = oracle.decode(qn, kn.reshape(n, cap, hkv, d), vn.reshape(n, cap, hkv, d), lens_l, False)
+        _run_pair(m, shape, ctx, m.DECODE_LOCAL, q, k, v, cap * hkv * d, lens, cap, want)
+        t_len = n * cap - 100 * call
+        tot = torch.tensor([t_len], dtype=torch.int32, device="cuda")
+        want = oracle.decode(qn, kn, vn, [t_len], True)
+        _run_pair(m, shape, ctx, m.DECODE_SYNC, q, k, v, 0, tot, n * cap, want)
 
 
 def test_noalloc_decode_rejects_what_its_scratch_cannot_hold():
