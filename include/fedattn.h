@@ -219,7 +219,8 @@ fedattn_status fedattn_merge(fedattn_ctx *ctx, const fedattn_shape *shape, int64
  *   FEDATTN_DECODE_SYNC   every participant reads rows 0..kv_len[0]-1 of one shared cache
  *                         [T,Hkv,d]; kv_len dev int32 [1]; cache_stride_participant ignored.
  *   q, o dev [N,Hq,d]; lse dev float [N,Hq] or NULL; max_kv_len >= every kv_len (host; sizes the
- *   split-KV grid).  kv_len = 0 gives o = 0, lse = -inf.  Uses the workspace for split-KV partials. */
+ *   split-KV grid).  kv_len = 0 gives o = 0, lse = -inf.  Uses the workspace for split-KV partials.
+ *   Two launches per call (stream, then merge), chained by programmatic dependent launch. */
 typedef enum { FEDATTN_DECODE_LOCAL = 0, FEDATTN_DECODE_SYNC = 1 } fedattn_decode_mode;
 
 fedattn_status fedattn_decode(fedattn_ctx *ctx, const fedattn_shape *shape, int32_t mode,
@@ -234,7 +235,7 @@ fedattn_status fedattn_decode(fedattn_ctx *ctx, const fedattn_shape *shape, int3
  * must not be entered (inside a serving loop with a frozen memory plan, a plugin that receives
  * its tensors and nothing more, a process whose memory is fully pre-partitioned).  This entry
  * point takes no context and allocates nothing, on the host or on the device: the split-KV
- * partials go to a fixed 2.07 MiB array built into the library image, which every GPU that loads
+ * partials go to a fixed 8.25 MiB array built into the library image, which every GPU that loads
  * the library holds until the process exits.
  *
  * Same arguments, layouts and results as fedattn_decode (bf16, head_dim 128 only; anything else
@@ -243,12 +244,10 @@ fedattn_status fedattn_decode(fedattn_ctx *ctx, const fedattn_shape *shape, int3
  * It runs on the CURRENT device.  The first call on each device resolves the array's device
  * address and sets kernel attributes; make that first call outside any stream capture.  The
  * partial slots need not start at zero (every slot that is read is written earlier in the same
- * call) and their contents after a call are unspecified.  The few arrival counters beside them
- * must be zero when a call starts: they are zero when the library is loaded and every completed
- * call leaves them at zero.  All calls on one device share these arrays: two calls that may
- * overlap on the GPU (different streams, no ordering) race on them.  The first call on a device
- * also fills a small host-side table without locking: do not let two host threads make their
- * first call on the same device at the same moment. */
+ * call) and their contents after a call are unspecified.  All calls on one device share the
+ * array: two calls that may overlap on the GPU (different streams, no ordering) race on it.
+ * The first call on a device also fills a small host-side table without locking: do not let two
+ * host threads make their first call on the same device at the same moment. */
 fedattn_status fedattn_decode_noalloc(const fedattn_shape *shape, int32_t mode,
                                       const void *q, const void *k_cache, const void *v_cache,
                                       int64_t cache_stride_participant, const int32_t *kv_len,

@@ -396,7 +396,6 @@ fedattn_status fedattn_decode(fedattn_ctx *ctx, const fedattn_shape *shape, int3
         p.scale = eff_scale(shape); p.sync = mode == FEDATTN_DECODE_SYNC;
         p.cache_stride = cache_stride; p.kv_len = kv_len; p.max_kv_len = max_kv_len;
         p.partial = reinterpret_cast<float *>(ctx->c.scratch); p.partial_bytes = ctx->c.scratch_bytes;
-        p.counters = reinterpret_cast<int32_t *>(ctx->c.workspace + kStatusWords);
         err = launch_decode_bf16(&ctx->c, p, s, &ctx->c.launches);
     } else {
         GenericParams p;

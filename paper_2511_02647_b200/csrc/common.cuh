@@ -9,11 +9,8 @@
 
 namespace fedattn {
 
-// Workspace layout: [0, 256) status words, [256, kStatusBytes) arrival counters of the split-KV decode
-// (zero between calls: the last arriver resets its counter), then the scratch region.
-constexpr size_t kStatusWords = 256;
-constexpr int kDecodeCounters = 4096;
-constexpr size_t kStatusBytes = kStatusWords + kDecodeCounters * sizeof(int32_t);
+// Workspace layout: [0, 256) status words, then the scratch region.
+constexpr size_t kStatusBytes = 256;
 constexpr int kMaxP = FEDATTN_MAX_PARTICIPANTS;
 // Upper bound on spin iterations of any in-kernel wait before it gives up.
 constexpr uint32_t kSpinLimit = 1u << 22;
@@ -123,8 +120,8 @@ struct DecodeParams {
     int32_t max_kv_len;
     float *partial;               // scratch: per-split partial results
     size_t partial_bytes;
-    int32_t *counters;            // kDecodeCounters arrival counters, all zero between calls
     int32_t g_shift;              // log2(hq / hkv) when that is a power of two, else -1 (set by the launcher)
+    int32_t early;                // inputs may be read before the preceding grid is complete (set by the launcher)
 };
 size_t decode_scratch_bytes(int n_part, int hq, int d, int sm_count);
 cudaError_t launch_decode_bf16(const Context *ctx, const DecodeParams &p, cudaStream_t s, int64_t *launches);

@@ -5,14 +5,28 @@
 // (mma.sync m16n8k16), which keeps the 32 flop/byte of the sync step far below the memory time.
 // K/V tiles of 64 keys stream through a 3-stage cp.async pipeline with a 16-byte-chunk XOR
 // swizzle (conflict-free ldmatrix).  Row max / row sum are reduced with warp shuffles inside
-// each 4-lane quad.  Each CTA handles one (cache, KV head, split) and leaves an unnormalised
-// partial (m, l, o) in its shared memory.  The splits of one (cache, KV head) are launched as
-// thread-block clusters of up to 8 CTAs, which merge their partials through distributed shared
-// memory (each CTA of the cluster takes a share of the rows).  If a (cache, KV head) spans several
-// clusters, the cluster results go to global scratch and the CTA that arrives last for its rows
-// merges them, so a decode step is one launch and no CTA ever spins on another.
-#include <cooperative_groups.h>
+// each 4-lane quad.
+//
+// Two launches per decode call, chained by programmatic dependent launch:
+//   decode_stream_kernel  one CTA per (cache, KV head, split); every warp walks its key slice of the
+//                         split's tiles and leaves an unnormalised partial (m, l, o) per query row in
+//                         global scratch.  Nothing is merged here, so a CTA ends with its last tile.
+//   decode_merge_kernel   one CTA per output row: its partials (splits x key slices) are rescaled to a
+//                         common exponent reference, summed, normalised and written.  Its CTAs are
+//                         resident and waiting before the stream kernel ends, so the merge starts the
+//                         moment the last partial is visible.
+// Both kernels release their dependents as soon as they start.  The stream kernel reads its inputs
+// (q, kv_len, K/V) right away and waits for the preceding grid of the stream (griddepcontrol.wait)
+// only before its first write, the partials, which the merge of the previous call may still be
+// reading.  In a run of back-to-back decode calls a stream CTA of call i+1 therefore takes the seat of
+// a stream CTA of call i the moment that one ends, and the late CTAs, the flush and the merge of
+// call i are hidden behind the next call's streaming.  Reading before the wait is sound because the
+// only grids that release dependents early are this file's own, and they write nothing but o, lse
+// and the scratch: the launcher checks the inputs of a call against the outputs of the previous one
+// and falls back to waiting first when they overlap.  No CTA ever waits on another CTA.
 #include <string.h>
+
+#include <mutex>
 
 #include "common.cuh"
 
@@ -27,9 +41,8 @@ constexpr int kTileBytes = kTileKeys * kD * 2;          // 16 KB (K or V)
 constexpr int kStageBytes = 2 * kTileBytes;             // K + V
 constexpr int kPartialStride = kD + 4;                  // m, l, 2 pad, o[128]: o is 16-byte aligned
 constexpr float kRescaleThreshold = 8.0f;               // log2 units
-constexpr int kMaxCluster = 8;                          // CTAs per cluster (portable maximum)
-constexpr int kMaxSlots = 16;                           // clusters per (cache, KV head): partials in global scratch
-constexpr int kCtaPartOffset = 72 * 1024;               // byte offset of the CTA's merged partial in shared memory
+constexpr int kMaxSlots = 64;                           // partials per output row: splits x key slices of a CTA
+constexpr int kMergeGroups = 4;                         // the merge kernel sums a row's partials in this many groups
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -76,74 +89,6 @@ __device__ __forceinline__ uint32_t swz(int row, int chunk) { return (uint32_t)(
 }  // namespace
 
 
-// Merges the n cluster results (slots 0 .. n-1, n <= kMaxSlots) of `rows` stacked query rows row0,
-// row0 + row_step, ... of one (cache, KV head), normalises and writes o / lse.  Called by every thread
-// of the CTA.  Each thread owns 4 output columns of a row and reads every slot's (m, l) itself, so all
-// loads are issued at once and there is no barrier.
-template <int kThreads>
-__device__ __forceinline__ void merge_slots(const DecodeParams &p, int n, int cache, int kvh, int row0, int row_step,
-                                            int rows)
-{
-    const int g = p.hq / p.hkv;
-    for (int i = threadIdx.x; i < rows * (kD / 4); i += kThreads) {
-        const int rr = i / (kD / 4), c4 = i - rr * (kD / 4);
-        const int srow = row0 + rr * row_step;
-        const int part = p.sync ? srow / g : cache;
-        const int head = kvh * g + (p.sync ? srow % g : srow);
-        const size_t orow = (size_t)part * p.hq + head;
-        const float *src = p.partial + orow * n * kPartialStride;
-        float mm = -INFINITY, ll = 0.f;
-        float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int k0 = 0; k0 < n; k0 += 4) {
-            float2 ml[4];
-            float4 v[4];
-#pragma unroll
-            for (int k = 0; k < 4; ++k)
-                if (k0 + k < n) {
-                    ml[k] = __ldcg(reinterpret_cast<const float2 *>(src + (size_t)(k0 + k) * kPartialStride));
-                    v[k] = __ldcg(reinterpret_cast<const float4 *>(src + (size_t)(k0 + k) * kPartialStride + 4 + c4 * 4));
-                }
-            float mn = mm;
-#pragma unroll
-            for (int k = 0; k < 4; ++k)
-                if (k0 + k < n) mn = fmaxf(mn, ml[k].x);
-            const float ms = mn == -INFINITY ? 0.f : mn;
-            const float f0 = ex2(mm - ms);                      // 0 on the first chunk (mm = -inf)
-            ll *= f0; a.x *= f0; a.y *= f0; a.z *= f0; a.w *= f0;
-#pragma unroll
-            for (int k = 0; k < 4; ++k)
-                if (k0 + k < n) {
-                    const float f = ex2(ml[k].x - ms);
-                    ll += ml[k].y * f;
-                    a.x += v[k].x * f; a.y += v[k].y * f; a.z += v[k].z * f; a.w += v[k].w * f;
-                }
-            mm = mn;
-        }
-        const float inv = ll > 0.f ? 1.f / ll : 0.f;
-        __nv_bfloat162 lo = __floats2bfloat162_rn(a.x * inv, a.y * inv), hi = __floats2bfloat162_rn(a.z * inv, a.w * inv);
-        uint2 w;
-        w.x = *reinterpret_cast<uint32_t *>(&lo); w.y = *reinterpret_cast<uint32_t *>(&hi);
-        *reinterpret_cast<uint2 *>(reinterpret_cast<__nv_bfloat16 *>(p.o) + orow * kD + c4 * 4) = w;
-        if (c4 == 0 && p.lse) p.lse[orow] = ll > 0.f ? (mm + log2f(ll)) * 0.6931471805599453f : -INFINITY;
-    }
-}
-
-// true in exactly one CTA: the last of `expected` to call this for the counter (which it resets to zero)
-__device__ __forceinline__ bool arrive_last(int32_t *ctr, int expected, int *s_flag)
-{
-    __threadfence();                                            // this CTA's partials before its arrival
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        const int prev = atomicAdd(ctr, 1);
-        *s_flag = prev == expected - 1;
-        if (*s_flag) *ctr = 0;                                  // ready for the next call
-    }
-    __syncthreads();
-    const bool last = *s_flag != 0;
-    if (last) __threadfence();                                  // the others' partials after their arrivals
-    return last;
-}
-
 #ifdef FEDATTN_DTRACE
 // Debug build only: cycle stamps of the phases of every CTA's thread 0, [cta][event].
 __device__ long long g_dtrace[1024 * 8];
@@ -154,11 +99,13 @@ __device__ long long g_dtrace[1024 * 8];
 
 // grid: x = split, y = KV head, z = cache * n_chunks + chunk   (cache = participant for LOCAL, 0 for SYNC)
 // block: 128 threads = 4 warps over (key slice, M-tile).  kMTiles == 1: 4 key slices of 16 keys of
-// every 64-key tile.  kMTiles == 2: 2 key slices of 32 keys x the 2 M-tiles, one M-tile per warp, so
-// the slice merge at the end moves half as much (K/V fragments are read by two warps instead).
+// every 64-key tile.  kMTiles == 2: 2 key slices of 32 keys x the 2 M-tiles, one M-tile per warp (K/V
+// fragments are read by two warps), which halves the partials per output row.
+// Partial of output row r, slot s = split * kSlices + slice:  partial[(r * n_slots + s) * kPartialStride]
+// = { m (log2 domain, scale included), l, -, -, o[128] }, unnormalised.
 template <int kMTiles>
 __global__ void __launch_bounds__(128, 2)
-decode_split_kernel(const DecodeParams p, int n_splits, int n_chunks)
+decode_stream_kernel(const DecodeParams p, int n_splits, int n_chunks)
 {
     constexpr int kSlices = 4 / kMTiles;                        // key slices per tile
     constexpr int kSteps = 4 / kSlices;                         // 16-key steps per warp and tile
@@ -166,6 +113,10 @@ decode_split_kernel(const DecodeParams p, int n_splits, int n_chunks)
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int slice = warp % kSlices, mt = warp / kSlices;     // this warp's key slice and M-tile
     DTRACE(0);
+    // The inputs are read before the preceding grid of the stream is known to be complete unless the
+    // launcher found that they may be its outputs.  The merge kernel of this call may take its seats.
+    if (!p.early) asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int split = blockIdx.x, kvh = blockIdx.y;
     const int cache = blockIdx.z / n_chunks, chunk = blockIdx.z - cache * n_chunks;
     const int g = p.hq / p.hkv;
@@ -325,139 +276,114 @@ decode_split_kernel(const DecodeParams p, int n_splits, int n_chunks)
         }
     }
     cp_async_wait<0>();
-    __syncthreads();
     DTRACE(3);
 
-    // ---- merge the key slices (warps) into this CTA's partial, kept in shared memory ----
-    // 1. every warp posts the exponent references of its rows; 2. every thread rescales its own
-    // accumulators to the common reference of its rows (in registers) and posts them; 3. the slices
-    // are summed with 16-byte reads.
-    float *red = reinterpret_cast<float *>(smem);               // [slice][16 kMTiles rows][kPartialStride]
-    float *sm_m = reinterpret_cast<float *>(smem + 68 * 1024);  // [slice][16 kMTiles rows]
-    float *sm_l = sm_m + 4 * 16 * kMTiles;
-    float *cta_part = reinterpret_cast<float *>(smem + kCtaPartOffset);   // [16 kMTiles rows][kPartialStride]
+
+    // the scratch may still be read by the merge of the previous call: the preceding grid must be complete
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    // ---- every warp leaves the partial of its key slice: nothing is merged here ----
     constexpr int kRows = 16 * kMTiles;
-    // only the rows that carry a query take part (LOCAL mode stacks g rows into a 16-row tile)
-    const int rows_here = min(kRows, rows_total - chunk * kRows);
-    const int ra = mt * 16 + (lane >> 2), rb = ra + 8;          // this thread's rows inside the CTA
-    if ((lane & 3) == 0) {
-        sm_m[slice * kRows + ra] = m0;
-        sm_m[slice * kRows + rb] = m1;
-    }
-    __syncthreads();
-    {
-        float ma = -INFINITY, mb = -INFINITY;
-#pragma unroll
-        for (int sl = 0; sl < kSlices; ++sl) { ma = fmaxf(ma, sm_m[sl * kRows + ra]); mb = fmaxf(mb, sm_m[sl * kRows + rb]); }
-        const float fa = ex2(m0 - (ma == -INFINITY ? 0.f : ma)), fb = ex2(m1 - (mb == -INFINITY ? 0.f : mb));
-        // quad-reduce l (each lane of a quad summed different keys)
-        float la = l0, lb = l1;
-        la += __shfl_xor_sync(0xffffffffu, la, 1); la += __shfl_xor_sync(0xffffffffu, la, 2);
-        lb += __shfl_xor_sync(0xffffffffu, lb, 1); lb += __shfl_xor_sync(0xffffffffu, lb, 2);
-        if ((lane & 3) == 0) { sm_l[slice * kRows + ra] = la * fa; sm_l[slice * kRows + rb] = lb * fb; }
-        float *w0 = red + ((size_t)slice * kRows + ra) * kPartialStride + 4 + (lane & 3) * 2;
-        float *w1 = w0 + 8 * kPartialStride;
-        if (ra < rows_here) {
-#pragma unroll
-            for (int i = 0; i < 16; ++i)
-                *reinterpret_cast<float2 *>(w0 + i * 8) = make_float2(acc[i][0] * fa, acc[i][1] * fa);
-        }
-        if (rb < rows_here) {
-#pragma unroll
-            for (int i = 0; i < 16; ++i)
-                *reinterpret_cast<float2 *>(w1 + i * 8) = make_float2(acc[i][2] * fb, acc[i][3] * fb);
-        }
-    }
-    __syncthreads();
-    for (int i = tid; i < rows_here * (kD / 4); i += 128) {
-        const int rr = i / (kD / 4), c4 = i - rr * (kD / 4);
-        float4 a = *reinterpret_cast<const float4 *>(red + (size_t)rr * kPartialStride + 4 + c4 * 4);
-#pragma unroll
-        for (int sl = 1; sl < kSlices; ++sl) {
-            const float4 v = *reinterpret_cast<const float4 *>(red + ((size_t)sl * kRows + rr) * kPartialStride + 4 + c4 * 4);
-            a.x += v.x; a.y += v.y; a.z += v.z; a.w += v.w;
-        }
-        float *dst = cta_part + rr * kPartialStride;
-        *reinterpret_cast<float4 *>(dst + 4 + c4 * 4) = a;
-        if (c4 == 0) {
-            float mm = -INFINITY, ll = 0.f;
-#pragma unroll
-            for (int sl = 0; sl < kSlices; ++sl) { mm = fmaxf(mm, sm_m[sl * kRows + rr]); ll += sm_l[sl * kRows + rr]; }
-            dst[0] = mm; dst[1] = ll;
-        }
-    }
-
-    // ---- cluster merge through distributed shared memory: rank k takes rows k, k + cs, ... ----
-    namespace cg = cooperative_groups;
-    cg::cluster_group cluster = cg::this_cluster();
-    const int cs = (int)cluster.num_blocks(), rank = (int)cluster.block_rank();
-    const int ncl = n_splits / cs, ci = split / cs;            // clusters per (cache, KV head); this cluster
-    const int row0 = chunk * kMTiles * 16, rows = min(kMTiles * 16, rows_total - row0);
-    const int my_rows = rows > rank ? (rows - rank + cs - 1) / cs : 0;
+    const int rows_here = min(kRows, rows_total - chunk * kRows);   // LOCAL stacks g rows into a 16-row tile
+    const int n_slots = n_splits * kSlices, slot = split * kSlices + slice;
     auto out_row = [&](int srow) -> size_t {
-        const int part = p.sync ? srow / g : cache;
-        const int head = kvh * g + (p.sync ? srow % g : srow);
-        return (size_t)part * p.hq + head;
+        int part = cache, sub = srow;
+        if (p.sync) {
+            if (p.g_shift >= 0) { part = srow >> p.g_shift; sub = srow & (g - 1); }
+            else { part = srow / g; sub = srow - part * g; }
+        }
+        return (size_t)part * p.hq + kvh * g + sub;
     };
+    // each lane of a quad summed different keys
+    l0 += __shfl_xor_sync(0xffffffffu, l0, 1); l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
+    l1 += __shfl_xor_sync(0xffffffffu, l1, 1); l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
+    const int ra = mt * 16 + (lane >> 2), rb = ra + 8;          // this thread's rows inside the CTA
+    if (ra < rows_here) {
+        float *dst = p.partial + (out_row(chunk * kRows + ra) * n_slots + slot) * kPartialStride;
+        if ((lane & 3) == 0) *reinterpret_cast<float2 *>(dst) = make_float2(m0, l0);
+        dst += 4 + (lane & 3) * 2;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) *reinterpret_cast<float2 *>(dst + i * 8) = make_float2(acc[i][0], acc[i][1]);
+    }
+    if (rb < rows_here) {
+        float *dst = p.partial + (out_row(chunk * kRows + rb) * n_slots + slot) * kPartialStride;
+        if ((lane & 3) == 0) *reinterpret_cast<float2 *>(dst) = make_float2(m1, l1);
+        dst += 4 + (lane & 3) * 2;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) *reinterpret_cast<float2 *>(dst + i * 8) = make_float2(acc[i][2], acc[i][3]);
+    }
     DTRACE(4);
-    cluster.sync();                                             // every CTA's partial is in place
-    for (int i = tid; i < my_rows * (kD / 4); i += 128) {
-        const int k = i / (kD / 4), c4 = i - k * (kD / 4);
-        const int rr = rank + k * cs;
-        float2 ml[kMaxCluster];
-        float4 v[kMaxCluster];
-#pragma unroll
-        for (int q = 0; q < kMaxCluster; ++q)
-            if (q < cs) {
-                const float *peer = cluster.map_shared_rank(cta_part, q) + rr * kPartialStride;
-                ml[q] = *reinterpret_cast<const float2 *>(peer);
-                v[q] = *reinterpret_cast<const float4 *>(peer + 4 + c4 * 4);
-            }
-        float mm = -INFINITY;
-#pragma unroll
-        for (int q = 0; q < kMaxCluster; ++q)
-            if (q < cs) mm = fmaxf(mm, ml[q].x);
-        const float ms = mm == -INFINITY ? 0.f : mm;
-        float ll = 0.f;
-        float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-        for (int q = 0; q < kMaxCluster; ++q)
-            if (q < cs) {
-                const float f = ex2(ml[q].x - ms);
-                ll += ml[q].y * f;
-                a.x += v[q].x * f; a.y += v[q].y * f; a.z += v[q].z * f; a.w += v[q].w * f;
-            }
-        const size_t orow = out_row(row0 + rr);
-        if (ncl == 1) {
-            const float inv = ll > 0.f ? 1.f / ll : 0.f;
-            __nv_bfloat162 lo = __floats2bfloat162_rn(a.x * inv, a.y * inv), hi = __floats2bfloat162_rn(a.z * inv, a.w * inv);
-            uint2 w;
-            w.x = *reinterpret_cast<uint32_t *>(&lo); w.y = *reinterpret_cast<uint32_t *>(&hi);
-            *reinterpret_cast<uint2 *>(reinterpret_cast<__nv_bfloat16 *>(p.o) + orow * kD + c4 * 4) = w;
-            if (c4 == 0 && p.lse) p.lse[orow] = ll > 0.f ? (mm + log2f(ll)) * 0.6931471805599453f : -INFINITY;
-        } else {
-            float *dst = p.partial + (orow * ncl + ci) * kPartialStride;
-            *reinterpret_cast<float4 *>(dst + 4 + c4 * 4) = a;
-            if (c4 == 0) { dst[0] = mm; dst[1] = ll; }
-        }
-    }
-    // This CTA is done reading its peers; it may not exit before they are done reading it.  Arrive now,
-    // wait at the very end: what follows does not touch distributed shared memory.
-    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-    DTRACE(5);
+}
 
-    // ---- several clusters per (cache, KV head): the last to arrive for these rows merges them ----
-    __shared__ int s_flag;
-    if (ncl > 1 && my_rows > 0) {                               // CTA-uniform
-        const int source = blockIdx.z * gridDim.y + kvh;
-        const bool last = arrive_last(p.counters + source * kMaxCluster + rank, ncl, &s_flag);
-        DTRACE(6);
-        if (last) {
-            merge_slots<128>(p, ncl, cache, kvh, row0 + rank, cs, my_rows);
-            DTRACE(7);
-        }
+// A CTA takes output rows (participant, query head) blockIdx.x, blockIdx.x + gridDim.x, ...: thread =
+// (group of slots, 4 output columns).  Every thread folds its group's partials, four loads in flight at
+// a time; the groups meet in shared memory.  The grid is at most one CTA per SM and a CTA is small (128
+// threads, few registers, 2 KB of shared memory), so the whole grid is resident beside the stream CTAs
+// at once: the next call's stream kernel can only be launched when every CTA of this grid has started.
+__global__ void __launch_bounds__(kMergeGroups * (kD / 4), 7)
+decode_merge_kernel(const DecodeParams p, int n_slots, int n_rows)
+{
+    __shared__ float4 s_acc[kMergeGroups][kD / 4];
+    __shared__ float2 s_ml[kMergeGroups];
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");         // the partials of this call
+    const int c4 = threadIdx.x & (kD / 4 - 1), grp = threadIdx.x / (kD / 4);
+    for (size_t orow = blockIdx.x; orow < (size_t)n_rows; orow += gridDim.x) {
+    const int per = (n_slots + kMergeGroups - 1) / kMergeGroups;
+    const int s0 = grp * per, s1 = min(s0 + per, n_slots);
+    const float *src = p.partial + orow * n_slots * kPartialStride;
+    float mm = -INFINITY, ll = 0.f;
+    float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int k0 = s0; k0 < s1; k0 += 4) {
+        float2 ml[4];
+        float4 v[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+            if (k0 + k < s1) {
+                ml[k] = __ldcg(reinterpret_cast<const float2 *>(src + (size_t)(k0 + k) * kPartialStride));
+                v[k] = __ldcg(reinterpret_cast<const float4 *>(src + (size_t)(k0 + k) * kPartialStride + 4 + c4 * 4));
+            }
+        float mn = mm;
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+            if (k0 + k < s1) mn = fmaxf(mn, ml[k].x);
+        const float ms = mn == -INFINITY ? 0.f : mn;
+        const float f0 = ex2(mm - ms);                          // 0 on the first batch (mm = -inf)
+        ll *= f0; a.x *= f0; a.y *= f0; a.z *= f0; a.w *= f0;
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+            if (k0 + k < s1) {
+                const float f = ex2(ml[k].x - ms);              // 0 for an empty partial (m = -inf)
+                ll += ml[k].y * f;
+                a.x += v[k].x * f; a.y += v[k].y * f; a.z += v[k].z * f; a.w += v[k].w * f;
+            }
+        mm = mn;
     }
-    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+    s_acc[grp][c4] = a;
+    if (c4 == 0) s_ml[grp] = make_float2(mm, ll);
+    __syncthreads();
+    if (grp == 0) {
+        float m_all = -INFINITY;
+#pragma unroll
+        for (int q = 0; q < kMergeGroups; ++q) m_all = fmaxf(m_all, s_ml[q].x);
+        const float mr = m_all == -INFINITY ? 0.f : m_all;
+        float l_all = 0.f;
+        float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int q = 0; q < kMergeGroups; ++q) {
+            const float f = ex2(s_ml[q].x - mr);
+            const float4 t = s_acc[q][c4];
+            l_all += s_ml[q].y * f;
+            o.x += t.x * f; o.y += t.y * f; o.z += t.z * f; o.w += t.w * f;
+        }
+        const float inv = l_all > 0.f ? 1.f / l_all : 0.f;
+        __nv_bfloat162 lo = __floats2bfloat162_rn(o.x * inv, o.y * inv), hi = __floats2bfloat162_rn(o.z * inv, o.w * inv);
+        uint2 w;
+        w.x = *reinterpret_cast<uint32_t *>(&lo); w.y = *reinterpret_cast<uint32_t *>(&hi);
+        *reinterpret_cast<uint2 *>(reinterpret_cast<__nv_bfloat16 *>(p.o) + orow * kD + c4 * 4) = w;
+        if (c4 == 0 && p.lse) p.lse[orow] = l_all > 0.f ? (m_all + log2f(l_all)) * 0.6931471805599453f : -INFINITY;
+    }
+    __syncthreads();                                            // the group buffers are reused by the next row
+    }
 }
 
 #ifdef FEDATTN_DTRACE
@@ -473,50 +399,101 @@ size_t decode_scratch_bytes(int n_part, int hq, int d, int /*sm_count*/)
     return (size_t)n_part * hq * kMaxSlots * kPartialStride * sizeof(float);
 }
 
-// Grid rule shared by both entry points.  Splits are chosen so that the whole grid is resident at
-// once (two CTAs per SM): a grid slightly larger than that would run a nearly empty second wave.
-// The splits of one (cache, KV head) form clusters of cs = 1, 2, 4 or 8 CTAs along grid.x.
-static cudaError_t launch_decode_split(const DecodeParams &p_in, int sm_count, int max_slots, cudaStream_t s,
+// Grid rule shared by both entry points.  Splits are chosen so that the whole stream grid is resident
+// at once (two CTAs per SM): a grid slightly larger than that would run a nearly empty second wave.
+// Output buffers of the decode calls per device since the last call that waited first.  Grids that
+// release their dependents early can pile up (each only needs its predecessor to have STARTED), so a
+// stream kernel that reads before it waits may run while the merge of any of those calls is still
+// writing.  A call whose inputs overlap one of the recorded buffers, or that would not fit into the
+// record, waits first; its grids then start only when everything before them is complete, which
+// empties the record.
+struct Range {
+    const char *p;
+    size_t bytes;
+};
+struct OutputRecord {
+    Range r[16];
+    int n = 0;
+};
+static OutputRecord g_outputs[64];
+static std::mutex g_outputs_mutex;
+
+static bool overlaps(const void *a, size_t a_bytes, const Range &b)
+{
+    const char *x = static_cast<const char *>(a);
+    return a && b.p && a_bytes && b.bytes && x < b.p + b.bytes && b.p < x + a_bytes;
+}
+
+static cudaError_t launch_decode_split(const DecodeParams &p_in, int device, int sm_count, cudaStream_t s,
                                        int64_t *launches)
 {
     DecodeParams p = p_in;
+    {
+        const size_t row_bytes = (size_t)p.hkv * kD * 2, qo_bytes = (size_t)p.n_part * p.hq * kD * 2;
+        const size_t cache_bytes = p.sync ? (size_t)p.max_kv_len * row_bytes
+                                          : ((size_t)(p.n_part - 1) * p.cache_stride * 2 + (size_t)p.max_kv_len * row_bytes);
+        const size_t len_bytes = (p.sync ? 1 : p.n_part) * sizeof(int32_t), lse_bytes = (size_t)p.n_part * p.hq * sizeof(float);
+        const void *in[4] = {p.q, p.k, p.v, p.kv_len};
+        const size_t in_bytes[4] = {qo_bytes, cache_bytes, cache_bytes, len_bytes};
+        const Range out[2] = {{static_cast<const char *>(p.o), qo_bytes},
+                              {reinterpret_cast<const char *>(p.lse), p.lse ? lse_bytes : 0}};
+        std::lock_guard<std::mutex> lock(g_outputs_mutex);
+        OutputRecord &rec = g_outputs[device & 63];
+        bool wait_first = false;
+        for (int i = 0; i < 4 && !wait_first; ++i)
+            for (int j = 0; j < rec.n && !wait_first; ++j) wait_first = overlaps(in[i], in_bytes[i], rec.r[j]);
+        int n_new = 0;
+        bool is_new[2] = {false, false};
+        for (int o = 0; o < 2; ++o) {
+            if (!out[o].bytes) continue;
+            bool known = false;
+            for (int j = 0; j < rec.n; ++j) known |= rec.r[j].p == out[o].p && rec.r[j].bytes >= out[o].bytes;
+            is_new[o] = !known;
+            n_new += !known;
+        }
+        if (rec.n + n_new > 16) wait_first = true;
+        if (wait_first) rec.n = 0;
+        for (int o = 0; o < 2; ++o)
+            if (out[o].bytes && (wait_first || is_new[o])) rec.r[rec.n++] = out[o];
+        p.early = wait_first ? 0 : 1;
+    }
     const int g = p.hq / p.hkv;
     p.g_shift = -1;
     for (int sh = 0; sh < 16; ++sh)
         if ((1 << sh) == g) p.g_shift = sh;
     const int rows_total = p.sync ? p.n_part * g : g;
     const int m_tiles = rows_total > 16 ? 2 : 1;
+    const int slices = 4 / m_tiles;                             // key slices (warps per M-tile) of a CTA
     const int n_chunks = (rows_total + 16 * m_tiles - 1) / (16 * m_tiles);
     const int caches = p.sync ? 1 : p.n_part;
     const int sources = caches * p.hkv * n_chunks;
     const int tiles = (p.max_kv_len + kTileKeys - 1) / kTileKeys;
     int n_splits = 2 * sm_count / sources;                     // rounded down: one wave
     if (n_splits > tiles / 2) n_splits = tiles / 2;            // at least two tiles per split
+    if (n_splits > kMaxSlots / slices) n_splits = kMaxSlots / slices;
     if (n_splits < 1) n_splits = 1;
-    int cs = 1;
-    while (cs * 2 <= kMaxCluster && cs * 2 <= n_splits) cs *= 2;
-    int ncl = n_splits / cs;
-    if (ncl > max_slots) ncl = max_slots;
-    if (ncl > kMaxSlots) ncl = kMaxSlots;
-    // several clusters per source meet through the arrival counters (kMaxCluster per source); with more
-    // sources than counters every source keeps to one cluster, which needs none
-    if (ncl > 1 && (int64_t)sources * kMaxCluster > kDecodeCounters) ncl = 1;
-    n_splits = ncl * cs;
-    if (ncl > 1 && (size_t)p.n_part * p.hq * ncl * kPartialStride * sizeof(float) > p.partial_bytes)
-        return cudaErrorInvalidValue;
+    const int n_slots = n_splits * slices;
+    if ((size_t)p.n_part * p.hq * n_slots * kPartialStride * sizeof(float) > p.partial_bytes) return cudaErrorInvalidValue;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof(cfg));
     cfg.gridDim = dim3(n_splits, p.hkv, caches * n_chunks);
     cfg.blockDim = dim3(128, 1, 1);
-    cfg.dynamicSmemBytes = kStages * kStageBytes;              // 96 KB (also covers the merge buffers)
+    cfg.dynamicSmemBytes = kStages * kStageBytes;              // 96 KB
     cfg.stream = s;
-    cudaLaunchAttribute attr;
-    attr.id = cudaLaunchAttributeClusterDimension;
-    attr.val.clusterDim.x = cs; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    cudaError_t e = m_tiles == 1 ? cudaLaunchKernelEx(&cfg, decode_split_kernel<1>, p, n_splits, n_chunks)
-                                 : cudaLaunchKernelEx(&cfg, decode_split_kernel<2>, p, n_splits, n_chunks);
+    cudaError_t e = m_tiles == 1 ? cudaLaunchKernelEx(&cfg, decode_stream_kernel<1>, p, n_splits, n_chunks)
+                                 : cudaLaunchKernelEx(&cfg, decode_stream_kernel<2>, p, n_splits, n_chunks);
+    if (launches) ++*launches;
+    if (e != cudaSuccess) return e;
+    const int n_rows = p.n_part * p.hq, rows_per_cta = (n_rows + sm_count - 1) / sm_count;
+    cfg.gridDim = dim3((n_rows + rows_per_cta - 1) / rows_per_cta, 1, 1);
+    cfg.blockDim = dim3(kMergeGroups * (kD / 4), 1, 1);
+    cfg.dynamicSmemBytes = 0;
+    e = cudaLaunchKernelEx(&cfg, decode_merge_kernel, p, n_slots, n_rows);
     if (launches) ++*launches;
     return e != cudaSuccess ? e : cudaGetLastError();
 }
@@ -524,9 +501,9 @@ static cudaError_t launch_decode_split(const DecodeParams &p_in, int sm_count, i
 static cudaError_t set_decode_smem_attr()
 {
     const int smem = kStages * kStageBytes;
-    cudaError_t e = cudaFuncSetAttribute(decode_split_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    cudaError_t e = cudaFuncSetAttribute(decode_stream_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(decode_split_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        e = cudaFuncSetAttribute(decode_stream_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     return e;
 }
 
@@ -538,7 +515,7 @@ cudaError_t launch_decode_bf16(const Context *ctx, const DecodeParams &p, cudaSt
         if (e != cudaSuccess) return e;
         attr_set[ctx->device & 63] = true;
     }
-    return launch_decode_split(p, ctx->sm_count, kMaxSlots, s, launches);
+    return launch_decode_split(p, ctx->device, ctx->sm_count, s, launches);
 }
 
 }  // namespace fedattn
@@ -548,23 +525,19 @@ cudaError_t launch_decode_bf16(const Context *ctx, const DecodeParams &p, cudaSt
 // allocator must not be entered (a latency-critical serving loop, a plugin that is handed its
 // buffers and nothing else), or code that cannot create the workspace-owning context because it
 // is not allowed to call cudaMalloc.  For them the split-KV partials live in a fixed array that is
-// part of the library image: every GPU that loads the library holds these 2.07 MiB until exit.
+// part of the library image: every GPU that loads the library holds these 8.25 MiB until exit.
 namespace fedattn {
 namespace {
 
 constexpr int kStaticMaxRows = 256;     // n_participants * n_q_heads
-constexpr int kStaticMaxSlots = 16;       // cluster results per (cache, KV head)
-constexpr size_t kStaticScratchFloats = (size_t)kStaticMaxRows * kStaticMaxSlots * kPartialStride;
+constexpr size_t kStaticScratchFloats = (size_t)kStaticMaxRows * kMaxSlots * kPartialStride;
 
 static __device__ __align__(256) float g_decode_scratch[kStaticScratchFloats];
-// arrival counters of the split merge; zero at load, and every call leaves them zero again
-static __device__ __align__(256) int32_t g_decode_counters[kDecodeCounters];
 
 // Device address of g_decode_scratch per device.  In host code the array's name is only a handle
 // for the runtime, so the address handed to the kernels comes from cudaGetSymbolAddress, taken
 // once per device with that device current.
 float *g_decode_scratch_ptr[64] = {};
-int32_t *g_decode_counters_ptr[64] = {};
 int g_decode_sm_count[64] = {};
 
 }  // namespace
@@ -599,10 +572,7 @@ extern "C" fedattn_status fedattn_decode_noalloc(const fedattn_shape *shape, int
         if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1)
             return FEDATTN_ERR_CUDA;
         if (set_decode_smem_attr() != cudaSuccess) return FEDATTN_ERR_CUDA;
-        int32_t *cptr = nullptr;
-        if (cudaGetSymbolAddress((void **)&cptr, g_decode_counters) != cudaSuccess || !cptr) return FEDATTN_ERR_CUDA;
         g_decode_sm_count[dev] = sms;
-        g_decode_counters_ptr[dev] = cptr;
         g_decode_scratch_ptr[dev] = ptr;
     }
 
@@ -615,11 +585,9 @@ extern "C" fedattn_status fedattn_decode_noalloc(const fedattn_shape *shape, int
     p.cache_stride = cache_stride_participant; p.kv_len = kv_len; p.max_kv_len = max_kv_len;
     p.partial = g_decode_scratch_ptr[dev];
     p.partial_bytes = kStaticScratchFloats * sizeof(float);
-    p.counters = g_decode_counters_ptr[dev];
 
-    // same grid rule as the workspace-backed call, with the split count capped to the built-in scratch
-    if (launch_decode_split(p, g_decode_sm_count[dev], kStaticMaxSlots, static_cast<cudaStream_t>(stream), nullptr) !=
-        cudaSuccess)
+    // same kernels and grid rule as the workspace-backed call
+    if (launch_decode_split(p, dev, g_decode_sm_count[dev], static_cast<cudaStream_t>(stream), nullptr) != cudaSuccess)
         return FEDATTN_ERR_CUDA;
     return FEDATTN_OK;
 }

@@ -46,6 +46,7 @@ constexpr int kD = 128;              // head dim
 // the exchange costs more.)
 constexpr int kSplit = 2;
 constexpr int kCols = kTileN / kSplit;
+static_assert(kCols == 64, "the visibility mask of a thread's columns is one 64-bit word");
 constexpr int kSoftmaxThreads = 128 * kSplit;
 constexpr int kThreads = kSoftmaxThreads + 128;  // then a warpgroup holding the TMA producer warp and the MMA issuer warp
 // Registers move from that warpgroup to the softmax warpgroups once the roles split (setmaxnreg):
@@ -642,17 +643,13 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         auto wg_sync = [&]() { asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "n"(32 * kSplit) : "memory"); };
         const bool o_aligned32 = (reinterpret_cast<uintptr_t>(p.o) & 31) == 0;
 
-        // One visit = the softmax of one S tile of one sub-tile.  Mask kinds: 0 none (every key of the tile
-        // is visible to every row); 1 prefix (this thread's columns c < a0 are visible); 2 two ranges
-        // (c < a0, or a1 <= c < a2); 3 explicit positions (column c is key a1 + c, visible iff it exists and
-        // its position is <= a0 = the row's position).  Masked columns become -inf and every exponential of
-        // a masked tile goes through ex2.approx, which maps -inf to 0; in unmasked tiles a fixed subset of
-        // the columns takes the polynomial so that the ex2 unit, which is as slow as the tensor pipe for this
-        // tile shape, is not the bottleneck.
-        auto visit = [&](auto mask_tag, int t, int j, int gt, int a0, int a1, int a2, const int32_t *kvp, float &m_used,
-                         float &l) {
-            constexpr int kMask = decltype(mask_tag)::value;
-            constexpr bool kPartial = kMask != 0;
+        // One visit = the softmax of one S tile of one sub-tile.  kPartial: some row of the tile has masked
+        // columns; bit c of `vis` says whether this thread's column c is visible.  Masked columns become
+        // -inf and every exponential goes through ex2.approx, which maps -inf to 0; in unmasked tiles a fixed
+        // subset of the columns takes the polynomial so that the ex2 unit, which is as slow as the tensor
+        // pipe for this tile shape, is not the bottleneck.
+        auto visit = [&](auto partial_tag, int t, int j, int gt, uint64_t vis, float &m_used, float &l) {
+            constexpr bool kPartial = decltype(partial_tag)::value;
             const uint32_t tS = tmem_base + lane_base + kColS + t * 128 + kCols * hf;   // fp32 S, this part
             const uint32_t tP = tS;                                                      // bf16 P, this part
             const uint32_t tO = tmem_base + lane_base + kColO + t * 128 + kCols * hf;
@@ -663,22 +660,11 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
 #pragma unroll
             for (int c = 0; c < kCols; c += 32) FEDATTN_TMEM_LD32(tS + c, (s + c));
             tmem_wait_ld();
-            if (kMask == 1) {
+            if (kPartial) {
+                const uint32_t vis_lo = (uint32_t)vis, vis_hi = (uint32_t)(vis >> 32);
 #pragma unroll
                 for (int c = 0; c < kCols; ++c)
-                    if (c >= a0) s[c] = 0xff800000u;            // -inf; columns < a0 are visible
-            } else if (kMask == 2) {
-#pragma unroll
-                for (int c = 0; c < kCols; ++c)
-                    if (c >= a0 && !(c >= a1 && c < a2)) s[c] = 0xff800000u;
-            } else if (kMask == 3) {
-                const int T = (int)p.total_kv;
-#pragma unroll
-                for (int c = 0; c < kCols; ++c) {
-                    const int key = a1 + c;                     // the same address in every lane: one broadcast load
-                    const int kpos = kvp ? __ldg(kvp + min(key, T - 1)) : key;
-                    if (key >= T || kpos > a0) s[c] = 0xff800000u;
-                }
+                    if (!(((c < 32 ? vis_lo : vis_hi) >> (c & 31)) & 1u)) s[c] = 0xff800000u;      // -inf
             }
             // partial row maximum: 8 independent chains, then a tree
             float mx[8];
@@ -798,19 +784,32 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                 const int t = n_sub == 2 ? (v & 1) : 0;
                 const int j = n_sub == 2 ? (v >> 1) : v;
                 const int gt = (t ? gsub1 : gsub0) + j;
+                // columns of this thread that lie below n (n may be <= 0 or >= kCols)
+                auto below = [](int n) -> uint64_t { return n <= 0 ? 0ull : (n >= 64 ? ~0ull : (1ull << n) - 1ull); };
                 if (two_range) {
                     const int k0 = tile_of(it, j) * kTileN;     // first key of the tile
-                    if (k0 + kTileN <= it.a || (k0 >= it.b && k0 + kTileN <= T))
-                        visit(std::integral_constant<int, 0>{}, t, j, gt, 0, 0, 0, nullptr, m_a, l_a);
-                    else
-                        visit(std::integral_constant<int, 2>{}, t, j, gt, c_r - k0, it.b - k0 - kCols * hf, T - k0 - kCols * hf,
-                              nullptr, m_a, l_a);
+                    if (k0 + kTileN <= it.a || (k0 >= it.b && k0 + kTileN <= T)) {
+                        visit(std::false_type{}, t, j, gt, 0, m_a, l_a);
+                    } else {                                    // keys [0, a) and [b, T)
+                        const int cb = k0 + kCols * hf;         // key of this thread's column 0
+                        visit(std::true_type{}, t, j, gt, below(it.a - cb) | (below(T - cb) & ~below(it.b - cb)), m_a, l_a);
+                    }
                 } else if (j < n_full) {
-                    visit(std::integral_constant<int, 0>{}, t, j, gt, 0, 0, 0, nullptr, m_a, l_a);
+                    visit(std::false_type{}, t, j, gt, 0, m_a, l_a);
                 } else if (p.general) {
-                    visit(std::integral_constant<int, 3>{}, t, j, gt, p_row, j * kTileN + kCols * hf, 0, it.kvp, m_a, l_a);
+                    // column c is key cb + c: visible iff it exists and its position is not above the row's.
+                    // The address is the same in every lane: broadcast loads.
+                    const int cb = j * kTileN + kCols * hf;
+                    uint64_t vis = 0;
+#pragma unroll 8
+                    for (int c = 0; c < kCols; ++c) {
+                        const int key = cb + c;
+                        const int kpos = it.kvp ? __ldg(it.kvp + min(key, T - 1)) : key;
+                        if (key < T && kpos <= p_row) vis |= 1ull << c;
+                    }
+                    visit(std::true_type{}, t, j, gt, vis, m_a, l_a);
                 } else {
-                    visit(std::integral_constant<int, 1>{}, t, j, gt, c_r - j * kTileN, 0, 0, nullptr, m_a, l_a);
+                    visit(std::true_type{}, t, j, gt, below(c_r - j * kTileN), m_a, l_a);
                 }
                 if (n_sub == 2) {
                     float x = m_a; m_a = m_b; m_b = x;
