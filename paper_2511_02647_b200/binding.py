@@ -169,57 +169,140 @@ class Context:
             pass
 
 
-def fedattn_local(ctx: Context, shape: Shape, q, k, v, cu_seqlens_host: Sequence[int], o, lse=None,
-                  stream=None):
+# Every entry point comes in two forms: ``fedattn_x(...)`` marshals its arguments and calls the library;
+# ``prepare_x(...)`` marshals once and returns a zero-argument callable that repeats the same call (same
+# buffers, same stream), for loops in which the per-call marshalling of tensors and pointer arrays would
+# cost more host time than the kernel takes on the device.  Both do argument marshalling only.
+class PreparedCall:
+    """A library call with its arguments already converted; calling it enqueues the work again."""
+
+    def __init__(self, fn, args, where: str, keep):
+        self._fn, self._args, self._where, self._keep = fn, args, where, keep
+
+    def __call__(self, stream=None):
+        # every entry point takes the stream last; `stream` (a raw cudaStream_t) replaces the prepared one
+        code = self._fn(*self._args) if stream is None else self._fn(*self._args[:-1], stream)
+        if code != 0:
+            raise FedAttnError(code, self._where)
+
+
+def _args_local(ctx, shape, q, k, v, cu_seqlens_host, o, lse, stream):
     cu = _i32_array(cu_seqlens_host)
     if len(cu) != shape.n_participants + 1:
         raise ValueError("cu_seqlens must have N+1 entries")
-    _check(_lib.fedattn_local(ctx.handle, C.byref(shape), _ptr(q), _ptr(k), _ptr(v), cu, _ptr(o), _ptr(lse),
-                              _stream(stream)), "fedattn_local")
+    return (ctx.handle, C.byref(shape), _ptr(q), _ptr(k), _ptr(v), cu, _ptr(o), _ptr(lse), _stream(stream))
 
 
-def fedattn_aggregate_kv(ctx: Context, shape: Shape, mode: int, k_parts, v_parts, seqlens_host,
-                         k_sel_host=None, sel_idx_in=None, k_agg=None, v_agg=None, kv_pos=None, cu_kv=None,
-                         sel_idx_out=None, stream=None):
+def fedattn_local(ctx: Context, shape: Shape, q, k, v, cu_seqlens_host: Sequence[int], o, lse=None,
+                  stream=None):
+    _check(_lib.fedattn_local(*_args_local(ctx, shape, q, k, v, cu_seqlens_host, o, lse, stream)), "fedattn_local")
+
+
+def prepare_local(ctx: Context, shape: Shape, q, k, v, cu_seqlens_host: Sequence[int], o, lse=None, stream=None):
+    return PreparedCall(_lib.fedattn_local, _args_local(ctx, shape, q, k, v, cu_seqlens_host, o, lse, stream),
+                        "fedattn_local", (ctx, shape, q, k, v, o, lse))
+
+
+def _args_aggregate_kv(ctx, shape, mode, k_parts, v_parts, seqlens_host, k_sel_host, sel_idx_in, k_agg, v_agg, kv_pos,
+                       cu_kv, sel_idx_out, stream):
     n = shape.n_participants
     if len(k_parts) != n or len(v_parts) != n or len(seqlens_host) != n:
         raise ValueError("need one K part, V part and length per participant")
     kp = (C.c_void_p * n)(*[_ptr(t) for t in k_parts])
     vp = (C.c_void_p * n)(*[_ptr(t) for t in v_parts])
     ks = None if k_sel_host is None else _i32_array(k_sel_host)
-    _check(_lib.fedattn_aggregate_kv(ctx.handle, C.byref(shape), int(mode), kp, vp, _i32_array(seqlens_host), ks,
-                                     _ptr(sel_idx_in), _ptr(k_agg), _ptr(v_agg), _ptr(kv_pos), _ptr(cu_kv),
-                                     _ptr(sel_idx_out), _stream(stream)), "fedattn_aggregate_kv")
+    return (ctx.handle, C.byref(shape), int(mode), kp, vp, _i32_array(seqlens_host), ks, _ptr(sel_idx_in), _ptr(k_agg),
+            _ptr(v_agg), _ptr(kv_pos), _ptr(cu_kv), _ptr(sel_idx_out), _stream(stream))
+
+
+def fedattn_aggregate_kv(ctx: Context, shape: Shape, mode: int, k_parts, v_parts, seqlens_host,
+                         k_sel_host=None, sel_idx_in=None, k_agg=None, v_agg=None, kv_pos=None, cu_kv=None,
+                         sel_idx_out=None, stream=None):
+    _check(_lib.fedattn_aggregate_kv(*_args_aggregate_kv(ctx, shape, mode, k_parts, v_parts, seqlens_host, k_sel_host,
+                                                         sel_idx_in, k_agg, v_agg, kv_pos, cu_kv, sel_idx_out, stream)),
+           "fedattn_aggregate_kv")
+
+
+def prepare_aggregate_kv(ctx: Context, shape: Shape, mode: int, k_parts, v_parts, seqlens_host, k_sel_host=None,
+                         sel_idx_in=None, k_agg=None, v_agg=None, kv_pos=None, cu_kv=None, sel_idx_out=None, stream=None):
+    return PreparedCall(_lib.fedattn_aggregate_kv,
+                        _args_aggregate_kv(ctx, shape, mode, k_parts, v_parts, seqlens_host, k_sel_host, sel_idx_in, k_agg,
+                                           v_agg, kv_pos, cu_kv, sel_idx_out, stream),
+                        "fedattn_aggregate_kv", (ctx, shape, list(k_parts), list(v_parts), sel_idx_in, k_agg, v_agg, kv_pos,
+                                                 cu_kv, sel_idx_out))
+
+
+def _args_sync(ctx, shape, q, q_pos, k_agg, v_agg, kv_pos, total_kv, kv_head_major, o, lse, stream):
+    return (ctx.handle, C.byref(shape), _ptr(q), int(q.shape[0]), _ptr(q_pos), _ptr(k_agg), _ptr(v_agg), _ptr(kv_pos),
+            int(total_kv), int(bool(kv_head_major)), _ptr(o), _ptr(lse), _stream(stream))
 
 
 def fedattn_sync(ctx: Context, shape: Shape, q, q_pos, k_agg, v_agg, kv_pos, total_kv: int,
                  kv_head_major: bool, o, lse=None, stream=None):
-    _check(_lib.fedattn_sync(ctx.handle, C.byref(shape), _ptr(q), int(q.shape[0]), _ptr(q_pos), _ptr(k_agg),
-                             _ptr(v_agg), _ptr(kv_pos), int(total_kv), int(bool(kv_head_major)), _ptr(o),
-                             _ptr(lse), _stream(stream)), "fedattn_sync")
+    _check(_lib.fedattn_sync(*_args_sync(ctx, shape, q, q_pos, k_agg, v_agg, kv_pos, total_kv, kv_head_major, o, lse,
+                                         stream)), "fedattn_sync")
+
+
+def prepare_sync(ctx: Context, shape: Shape, q, q_pos, k_agg, v_agg, kv_pos, total_kv: int, kv_head_major: bool, o,
+                 lse=None, stream=None):
+    return PreparedCall(_lib.fedattn_sync,
+                        _args_sync(ctx, shape, q, q_pos, k_agg, v_agg, kv_pos, total_kv, kv_head_major, o, lse, stream),
+                        "fedattn_sync", (ctx, shape, q, q_pos, k_agg, v_agg, kv_pos, o, lse))
+
+
+def _args_sync_remote(ctx, shape, q, cu_seqlens_host, k_agg, v_agg, kv_pos, total_kv, kv_head_major, o, lse, stream):
+    cu = _i32_array(cu_seqlens_host)
+    if len(cu) != shape.n_participants + 1:
+        raise ValueError("cu_seqlens must have N+1 entries")
+    return (ctx.handle, C.byref(shape), _ptr(q), cu, _ptr(k_agg), _ptr(v_agg), _ptr(kv_pos), int(total_kv),
+            int(bool(kv_head_major)), _ptr(o), _ptr(lse), _stream(stream))
 
 
 def fedattn_sync_remote(ctx: Context, shape: Shape, q, cu_seqlens_host: Sequence[int], k_agg, v_agg, kv_pos,
                         total_kv: int, kv_head_major: bool, o, lse, stream=None):
-    cu = _i32_array(cu_seqlens_host)
-    if len(cu) != shape.n_participants + 1:
-        raise ValueError("cu_seqlens must have N+1 entries")
-    _check(_lib.fedattn_sync_remote(ctx.handle, C.byref(shape), _ptr(q), cu, _ptr(k_agg), _ptr(v_agg), _ptr(kv_pos),
-                                    int(total_kv), int(bool(kv_head_major)), _ptr(o), _ptr(lse), _stream(stream)),
-           "fedattn_sync_remote")
+    _check(_lib.fedattn_sync_remote(*_args_sync_remote(ctx, shape, q, cu_seqlens_host, k_agg, v_agg, kv_pos, total_kv,
+                                                       kv_head_major, o, lse, stream)), "fedattn_sync_remote")
+
+
+def prepare_sync_remote(ctx: Context, shape: Shape, q, cu_seqlens_host: Sequence[int], k_agg, v_agg, kv_pos, total_kv: int,
+                        kv_head_major: bool, o, lse, stream=None):
+    return PreparedCall(_lib.fedattn_sync_remote,
+                        _args_sync_remote(ctx, shape, q, cu_seqlens_host, k_agg, v_agg, kv_pos, total_kv, kv_head_major, o,
+                                          lse, stream),
+                        "fedattn_sync_remote", (ctx, shape, q, k_agg, v_agg, kv_pos, o, lse))
+
+
+def _args_merge(ctx, shape, n_rows, o_a, lse_a, o_b, lse_b, o, lse, stream):
+    return (ctx.handle, C.byref(shape), int(n_rows), _ptr(o_a), _ptr(lse_a), _ptr(o_b), _ptr(lse_b), _ptr(o), _ptr(lse),
+            _stream(stream))
 
 
 def fedattn_merge(ctx: Context, shape: Shape, n_rows: int, o_a, lse_a, o_b, lse_b, o, lse=None, stream=None):
-    _check(_lib.fedattn_merge(ctx.handle, C.byref(shape), int(n_rows), _ptr(o_a), _ptr(lse_a), _ptr(o_b), _ptr(lse_b),
-                              _ptr(o), _ptr(lse), _stream(stream)), "fedattn_merge")
+    _check(_lib.fedattn_merge(*_args_merge(ctx, shape, n_rows, o_a, lse_a, o_b, lse_b, o, lse, stream)), "fedattn_merge")
 
+
+def prepare_merge(ctx: Context, shape: Shape, n_rows: int, o_a, lse_a, o_b, lse_b, o, lse=None, stream=None):
+    return PreparedCall(_lib.fedattn_merge, _args_merge(ctx, shape, n_rows, o_a, lse_a, o_b, lse_b, o, lse, stream),
+                        "fedattn_merge", (ctx, shape, o_a, lse_a, o_b, lse_b, o, lse))
+
+
+def _args_decode(ctx, shape, mode, q, k_cache, v_cache, cache_stride_participant, kv_len, max_kv_len, o, lse, stream):
+    return (ctx.handle, C.byref(shape), int(mode), _ptr(q), _ptr(k_cache), _ptr(v_cache), int(cache_stride_participant),
+            _ptr(kv_len), int(max_kv_len), _ptr(o), _ptr(lse), _stream(stream))
 
 
 def fedattn_decode(ctx: Context, shape: Shape, mode: int, q, k_cache, v_cache, cache_stride_participant: int,
                    kv_len, max_kv_len: int, o, lse=None, stream=None):
-    _check(_lib.fedattn_decode(ctx.handle, C.byref(shape), int(mode), _ptr(q), _ptr(k_cache), _ptr(v_cache),
-                               int(cache_stride_participant), _ptr(kv_len), int(max_kv_len), _ptr(o), _ptr(lse),
-                               _stream(stream)), "fedattn_decode")
+    _check(_lib.fedattn_decode(*_args_decode(ctx, shape, mode, q, k_cache, v_cache, cache_stride_participant, kv_len,
+                                             max_kv_len, o, lse, stream)), "fedattn_decode")
+
+
+def prepare_decode(ctx: Context, shape: Shape, mode: int, q, k_cache, v_cache, cache_stride_participant: int, kv_len,
+                   max_kv_len: int, o, lse=None, stream=None):
+    return PreparedCall(_lib.fedattn_decode,
+                        _args_decode(ctx, shape, mode, q, k_cache, v_cache, cache_stride_participant, kv_len, max_kv_len, o,
+                                     lse, stream),
+                        "fedattn_decode", (ctx, shape, q, k_cache, v_cache, kv_len, o, lse))
 
 
 def fedattn_decode_noalloc(shape: Shape, mode: int, q, k_cache, v_cache, cache_stride_participant: int,

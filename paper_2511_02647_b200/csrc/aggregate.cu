@@ -119,12 +119,14 @@ __device__ __forceinline__ double sq_acc_bf16x2(double s, uint32_t w)
 constexpr int kSelThreads = 256;
 constexpr int kSelMaxLen = 4096;
 constexpr int kMaxSlices = 8;              // portable cluster size
+constexpr int kCtasPerSm = 3;              // resident CTAs the staging rings are sized for
 
 template <int kDtype>
 __global__ void __launch_bounds__(kSelThreads)
 topk_fused_kernel(const PartsParams pp, int hkv, int vpr /* 16-byte vectors per (row, head) */,
                   int n_stages /* buffers in every warp's staging ring, 2..4 */,
                   int max_len /* longest participant: sizes the key arrays */,
+                  int early /* the inputs may be read before the preceding grid of the stream is complete */,
                   uint4 *k_agg, uint4 *v_agg, int32_t *kv_pos, int32_t *cu_kv, int32_t *sel_idx_out)
 {
     // dynamic shared memory: keys [max_len] u64 | kept rows [max_len] u16 | staging [8 warps][n_stages][32 rows][128 B]
@@ -142,10 +144,20 @@ topk_fused_kernel(const PartsParams pp, int hkv, int vpr /* 16-byte vectors per 
     cg::cluster_group cluster = cg::this_cluster();
     const int h = blockIdx.x, n = blockIdx.y, slice = blockIdx.z, n_slices = gridDim.z;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    if (h == 0 && n == 0 && slice == 0 && cu_kv && tid <= pp.n) cu_kv[tid] = pp.cu_kv[tid];
+    // Launched with programmatic stream serialization: the dependents may take their seats at once, and
+    // this kernel waits for the preceding grid only before its first write (the outputs of an earlier
+    // call may still be read or written by it) unless its inputs might be that grid's outputs.
+    if (!early) asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int len = pp.off[n + 1] - pp.off[n];
     const int k = pp.cu_kv[n + 1] - pp.cu_kv[n];
-    if (k == 0 || len == 0) return;                           // the same for every slice of the cluster
+    if (k == 0 || len == 0) {                                 // the same for every slice of the cluster
+        if (h == 0 && n == 0 && slice == 0 && cu_kv && tid <= pp.n) {
+            asm volatile("griddepcontrol.wait;" ::: "memory");
+            cu_kv[tid] = pp.cu_kv[tid];
+        }
+        return;
+    }
     const int64_t T = pp.cu_kv[pp.n];
 
     // ---- 1. scores of this slice's tokens ----
@@ -384,7 +396,10 @@ topk_fused_kernel(const PartsParams pp, int hkv, int vpr /* 16-byte vectors per 
     }
     __syncthreads();
 
-    // gather this slice: rows my_rows[0 .. o_hi - o_lo) of participant n, head h
+    // gather this slice: rows my_rows[0 .. o_hi - o_lo) of participant n, head h.  First write of this
+    // kernel: the preceding grid of the stream must be complete.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (h == 0 && n == 0 && slice == 0 && cu_kv && tid <= pp.n) cu_kv[tid] = pp.cu_kv[tid];
     const int n_out = o_hi - o_lo;
     const int64_t out_row0 = (int64_t)h * T + pp.cu_kv[n] + o_lo;
     const uint4 *ksrc = reinterpret_cast<const uint4 *>(pp.k[n]), *vsrc = reinterpret_cast<const uint4 *>(pp.v[n]);
@@ -426,17 +441,32 @@ cudaError_t launch_topk_fused(const PartsParams &pp, int hkv, int d, int dtype, 
 {
     if (pp.cu_kv[pp.n] == 0 && !cu_kv) return cudaSuccess;
     const int elt = dtype == FEDATTN_BF16 ? 2 : 4;
+    int early;
+    {
+        const size_t row_bytes = (size_t)hkv * d * elt;
+        const size_t T = (size_t)pp.cu_kv[pp.n];
+        MemRange in[2 * kMaxP];
+        for (int i = 0; i < pp.n; ++i) {
+            const size_t bytes = (size_t)(pp.off[i + 1] - pp.off[i]) * row_bytes;
+            in[2 * i] = {pp.k[i], bytes};
+            in[2 * i + 1] = {pp.v[i], bytes};
+        }
+        const MemRange out[5] = {{k_agg, T * row_bytes}, {v_agg, T * row_bytes}, {kv_pos, kv_pos ? T * hkv * 4 : 0},
+                                 {cu_kv, cu_kv ? (size_t)(pp.n + 1) * 4 : 0}, {sel_idx_out, sel_idx_out ? T * hkv * 4 : 0}};
+        early = early_read_allowed(device, in, 2 * pp.n, out, 5) ? 1 : 0;
+    }
     const int vpr = d * elt / 16;
     int max_len = 0;
     for (int i = 0; i < pp.n; ++i) max_len = max(max_len, pp.off[i + 1] - pp.off[i]);
     if (max_len > kSelMaxLen) return cudaErrorInvalidValue;
     // Shared memory per CTA: keys (8 B) and kept rows (2 B) per token of the longest participant, then
-    // the staging buffers.  As many buffers (2..4) as still let two CTAs share an SM: what is in flight
-    // from HBM is all but one of them.
+    // the staging buffers.  As many buffers (2..4) as still let kCtasPerSm CTAs share an SM: what is in
+    // flight from HBM is all but one of them.  More resident CTAs matter more than deeper rings: CTAs in
+    // different phases (scores, selection, gather), also of consecutive calls, keep HBM busy.
     const int stage_bytes = (kSelThreads / 32) * 32 * 128;    // one buffer per warp: 32 rows x 128 bytes
     const int fixed = (max_len * 10 + 15) & ~15;
-    const int two_per_sm = (228 * 1024) / 2 - 1024 /*reserved per CTA*/ - 2048 /*static*/;
-    int n_stages = (two_per_sm - fixed) / stage_bytes;
+    const int per_cta = (228 * 1024) / kCtasPerSm - 1024 /*reserved per CTA*/ - 2048 /*static*/;
+    int n_stages = (per_cta - fixed) / stage_bytes;
     n_stages = n_stages < 2 ? 2 : (n_stages > 4 ? 4 : n_stages);
     const int smem = fixed + n_stages * stage_bytes;
     static bool attr_set[64] = {};                            // the attribute is per device
@@ -458,15 +488,17 @@ cudaError_t launch_topk_fused(const PartsParams &pp, int hkv, int d, int dtype, 
     cfg.blockDim = dim3(kSelThreads, 1, 1);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = s;
-    cudaLaunchAttribute attr;
-    attr.id = cudaLaunchAttributeClusterDimension;
-    attr.val.clusterDim.x = 1; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = slices;
-    cfg.attrs = &attr;
-    cfg.numAttrs = 1;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 1; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = slices;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
     cudaError_t e = dtype == FEDATTN_BF16
-                        ? cudaLaunchKernelEx(&cfg, topk_fused_kernel<FEDATTN_BF16>, pp, hkv, vpr, n_stages, max_len,
+                        ? cudaLaunchKernelEx(&cfg, topk_fused_kernel<FEDATTN_BF16>, pp, hkv, vpr, n_stages, max_len, early,
                                              (uint4 *)k_agg, (uint4 *)v_agg, kv_pos, cu_kv, sel_idx_out)
-                        : cudaLaunchKernelEx(&cfg, topk_fused_kernel<FEDATTN_F32>, pp, hkv, vpr, n_stages, max_len,
+                        : cudaLaunchKernelEx(&cfg, topk_fused_kernel<FEDATTN_F32>, pp, hkv, vpr, n_stages, max_len, early,
                                              (uint4 *)k_agg, (uint4 *)v_agg, kv_pos, cu_kv, sel_idx_out);
     ++*launches;
     return e != cudaSuccess ? e : cudaGetLastError();

@@ -28,6 +28,16 @@ struct Context {
     void *encode_tiled;    // cuTensorMapEncodeTiled entry point (driver), or nullptr
 };
 
+// ---- early-start bookkeeping (programmatic dependent launch) ------------------------------------
+struct MemRange {
+    const void *p;
+    size_t bytes;
+};
+// Records `out` as buffers that grids of this call may still be writing when later grids start, and
+// returns whether this call may read `in` before the preceding grid of the stream is complete (false:
+// it must wait first).  n_out <= 16.
+bool early_read_allowed(int device, const MemRange *in, int n_in, const MemRange *out, int n_out);
+
 // ---- generic SIMT attention (fp32 or bf16 storage, any head_dim <= 128) --------------------
 enum GenericMode { kLocal = 0, kSync = 1, kDecodeLocal = 2, kDecodeSync = 3 };
 

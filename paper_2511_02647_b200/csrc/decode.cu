@@ -21,12 +21,11 @@
 // reading.  In a run of back-to-back decode calls a stream CTA of call i+1 therefore takes the seat of
 // a stream CTA of call i the moment that one ends, and the late CTAs, the flush and the merge of
 // call i are hidden behind the next call's streaming.  Reading before the wait is sound because the
-// only grids that release dependents early are this file's own, and they write nothing but o, lse
-// and the scratch: the launcher checks the inputs of a call against the outputs of the previous one
-// and falls back to waiting first when they overlap.  No CTA ever waits on another CTA.
+// only grids that release dependents early are this library's own, and they write nothing but their
+// outputs and the scratch: the launcher checks the inputs of a call against the outputs of the recent
+// calls of that kind and falls back to waiting first when they overlap (early_start.cu).  No CTA ever
+// waits on another CTA.
 #include <string.h>
-
-#include <mutex>
 
 #include "common.cuh"
 
@@ -401,61 +400,19 @@ size_t decode_scratch_bytes(int n_part, int hq, int d, int /*sm_count*/)
 
 // Grid rule shared by both entry points.  Splits are chosen so that the whole stream grid is resident
 // at once (two CTAs per SM): a grid slightly larger than that would run a nearly empty second wave.
-// Output buffers of the decode calls per device since the last call that waited first.  Grids that
-// release their dependents early can pile up (each only needs its predecessor to have STARTED), so a
-// stream kernel that reads before it waits may run while the merge of any of those calls is still
-// writing.  A call whose inputs overlap one of the recorded buffers, or that would not fit into the
-// record, waits first; its grids then start only when everything before them is complete, which
-// empties the record.
-struct Range {
-    const char *p;
-    size_t bytes;
-};
-struct OutputRecord {
-    Range r[16];
-    int n = 0;
-};
-static OutputRecord g_outputs[64];
-static std::mutex g_outputs_mutex;
-
-static bool overlaps(const void *a, size_t a_bytes, const Range &b)
-{
-    const char *x = static_cast<const char *>(a);
-    return a && b.p && a_bytes && b.bytes && x < b.p + b.bytes && b.p < x + a_bytes;
-}
-
 static cudaError_t launch_decode_split(const DecodeParams &p_in, int device, int sm_count, cudaStream_t s,
                                        int64_t *launches)
 {
     DecodeParams p = p_in;
     {
+        // may the stream kernel read its inputs before the preceding grid of the stream is complete?
         const size_t row_bytes = (size_t)p.hkv * kD * 2, qo_bytes = (size_t)p.n_part * p.hq * kD * 2;
         const size_t cache_bytes = p.sync ? (size_t)p.max_kv_len * row_bytes
                                           : ((size_t)(p.n_part - 1) * p.cache_stride * 2 + (size_t)p.max_kv_len * row_bytes);
-        const size_t len_bytes = (p.sync ? 1 : p.n_part) * sizeof(int32_t), lse_bytes = (size_t)p.n_part * p.hq * sizeof(float);
-        const void *in[4] = {p.q, p.k, p.v, p.kv_len};
-        const size_t in_bytes[4] = {qo_bytes, cache_bytes, cache_bytes, len_bytes};
-        const Range out[2] = {{static_cast<const char *>(p.o), qo_bytes},
-                              {reinterpret_cast<const char *>(p.lse), p.lse ? lse_bytes : 0}};
-        std::lock_guard<std::mutex> lock(g_outputs_mutex);
-        OutputRecord &rec = g_outputs[device & 63];
-        bool wait_first = false;
-        for (int i = 0; i < 4 && !wait_first; ++i)
-            for (int j = 0; j < rec.n && !wait_first; ++j) wait_first = overlaps(in[i], in_bytes[i], rec.r[j]);
-        int n_new = 0;
-        bool is_new[2] = {false, false};
-        for (int o = 0; o < 2; ++o) {
-            if (!out[o].bytes) continue;
-            bool known = false;
-            for (int j = 0; j < rec.n; ++j) known |= rec.r[j].p == out[o].p && rec.r[j].bytes >= out[o].bytes;
-            is_new[o] = !known;
-            n_new += !known;
-        }
-        if (rec.n + n_new > 16) wait_first = true;
-        if (wait_first) rec.n = 0;
-        for (int o = 0; o < 2; ++o)
-            if (out[o].bytes && (wait_first || is_new[o])) rec.r[rec.n++] = out[o];
-        p.early = wait_first ? 0 : 1;
+        const MemRange in[4] = {{p.q, qo_bytes}, {p.k, cache_bytes}, {p.v, cache_bytes},
+                                {p.kv_len, (p.sync ? 1 : p.n_part) * sizeof(int32_t)}};
+        const MemRange out[2] = {{p.o, qo_bytes}, {p.lse, p.lse ? (size_t)p.n_part * p.hq * sizeof(float) : 0}};
+        p.early = early_read_allowed(device, in, 4, out, 2) ? 1 : 0;
     }
     const int g = p.hq / p.hkv;
     p.g_shift = -1;

@@ -442,6 +442,9 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     uint64_t *p_full = bars + 16;                        // [sub-tile][column part]
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 24);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(bars + 25);
+    // what the producer tells the MMA issuer about an item, published before the item's Q load is issued
+    // and read after q_full: {KV tiles, sub-tiles}; -1 tiles = no more items.  Two slots, like the phases.
+    volatile int *item_info = reinterpret_cast<volatile int *>(bars + 26);
     float *x_max = reinterpret_cast<float *>(bars + 32);            // [2 buffers][kSplit column parts][128 rows]
     float *x_sum = x_max + 2 * kSplit * kTileM;                     // [2 sub-tiles][kSplit column parts][128 rows]
 
@@ -494,6 +497,8 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                 const Item it = decode_item(kp, item);
                 if (it.n_tiles == 0) continue;
                 if (qn > 0) mbar_wait(q_empty, (qn - 1) & 1, abort_flag, kp.status);   // previous item's S MMAs done
+                item_info[(qn & 1) * 2] = it.n_tiles;
+                item_info[(qn & 1) * 2 + 1] = it.valid1 ? 2 : 1;
                 mbar_expect_tx(q_full, it.valid1 ? 2 * kTileBytes : kTileBytes);
                 tma_load_3d(sQ, &map_q, q_full, 0, it.head0, it.q_row0);
                 tma_load_3d(sQ + kHalfBytes, &map_q, q_full, 64, it.head0, it.q_row0);
@@ -518,6 +523,10 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                 git += it.n_tiles;
                 ++qn;
             }
+            // end marker for the MMA issuer, in the slot and phase the next item would have used
+            if (qn > 0) mbar_wait(q_empty, (qn - 1) & 1, abort_flag, kp.status);
+            item_info[(qn & 1) * 2] = -1;
+            mbar_arrive(q_full);
             if (*abort_flag) {
                 // give the copies still in flight a bounded chance to land before the CTA retires
                 for (int gt = max(0, git - 2); gt < git; ++gt) {
@@ -553,14 +562,12 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         // git / qn count the KV tiles / items of sub-tile 0 (and of the K/V ring); git1 / qn1
         // count only the items in which the pair's second head exists.
         int git = 0, qn = 0, git1 = 0, qn1 = 0;
-        for (int k = 0; k < n_rounds; ++k) {
-            const int item = item_of(k);
-            if (item >= n_items) continue;
-            const Item it = decode_item(kp, item);
-            const int n = it.n_tiles;
-            if (n == 0) continue;
-            const int n_sub = it.valid1 ? 2 : 1;
-            mbar_wait(q_full, qn & 1, abort_flag, kp.status);
+        for (;;) {
+            // the producer decodes the work items; this warp only learns their shape
+            if (!mbar_wait(q_full, qn & 1, abort_flag, kp.status)) break;
+            const int n = item_info[(qn & 1) * 2];
+            if (n < 0) break;
+            const int n_sub = item_info[(qn & 1) * 2 + 1];
             mbar_wait(k_full + (git & 1), (git >> 1) & 1, abort_flag, kp.status);
             tc_fence_after();
             for (int t = 0; t < n_sub; ++t) {
@@ -607,7 +614,7 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             }
             git += n;
             ++qn;
-            if (it.valid1) { git1 += n; ++qn1; }
+            if (n_sub == 2) { git1 += n; ++qn1; }
         }
     } else if (warp >= 4 * kSplit) {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kOtherRegs));      // the two idle warps of that warpgroup
