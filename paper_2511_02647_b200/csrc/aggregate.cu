@@ -119,7 +119,7 @@ __device__ __forceinline__ double sq_acc_bf16x2(double s, uint32_t w)
 constexpr int kSelThreads = 256;
 constexpr int kSelMaxLen = 4096;
 constexpr int kMaxSlices = 8;              // portable cluster size
-constexpr int kCtasPerSm = 3;              // resident CTAs the staging rings are sized for
+constexpr int kCtasPerSm = 2;              // resident CTAs the staging rings are sized for
 
 template <int kDtype>
 __global__ void __launch_bounds__(kSelThreads)
@@ -481,7 +481,7 @@ cudaError_t launch_topk_fused(const PartsParams &pp, int hkv, int d, int dtype, 
     // slices per (head, participant): a power of two <= 8 (one cluster), about two CTAs per SM in total
     const int pairs = hkv * pp.n;
     int slices = 1;
-    while (slices * 2 <= kMaxSlices && pairs * slices * 2 <= 2 * sm_count) slices *= 2;
+    while (slices * 2 <= kMaxSlices && pairs * slices * 2 <= sm_count) slices *= 2;
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof(cfg));
     cfg.gridDim = dim3(hkv, pp.n, slices);

@@ -336,6 +336,28 @@ __device__ __forceinline__ int count_le(const int32_t *pos, int n, int x)
     return lo;
 }
 
+// The same count, found by a converged warp together: every step probes 32 evenly spaced entries at
+// once (one round trip to memory per step instead of one per halving), so 4096 entries take 3 steps.
+// Every lane returns the count.
+__device__ __forceinline__ int count_le_warp(const int32_t *pos, int n, int x, int lane)
+{
+    int lo = 0, hi = n;                                         // the count lies in [lo, hi]
+    while (hi > lo) {
+        const int width = hi - lo;
+        if (width <= 32) {
+            const bool le = lane < width && __ldg(pos + lo + lane) <= x;
+            return lo + __popc(__ballot_sync(0xffffffffu, le));  // the entries <= x are a prefix
+        }
+        const int stride = (width + 31) >> 5;
+        const int probe = min(lo + (lane + 1) * stride - 1, hi - 1);
+        const int k = __popc(__ballot_sync(0xffffffffu, __ldg(pos + probe) <= x));
+        if (k == 32) return hi;                                 // even the last entry is <= x
+        hi = min(lo + (k + 1) * stride - 1, hi - 1);            // entry `hi` is > x: the count is at most hi
+        lo = lo + k * stride;
+    }
+    return lo;
+}
+
 }  // namespace
 
 // One unit of work: a 128-row query tile x one pair of query heads that share a KV head.
@@ -349,8 +371,10 @@ struct Item {
 };
 __device__ __forceinline__ int tile_of(const Item &it, int j) { return j < it.n_a ? j : it.t_b0 + (j - it.n_a); }
 
-// allowed-prefix length c(row): keys kv_begin .. kv_begin + c - 1 are visible to query row r of the tile
-__device__ __forceinline__ int prefix_len(const PrefillParams &p, const Item &it, int r)
+// allowed-prefix length c(row): keys kv_begin .. kv_begin + c - 1 are visible to query row r of the tile.
+// Called by a converged warp with the same r in every lane (the searches are warp-cooperative).
+template <bool kSpecial>
+__device__ __forceinline__ int prefix_len(const PrefillParams &p, const Item &it, int r, int lane)
 {
     const int pos = it.q_row0 + r;
     const int T = (int)p.total_kv;
@@ -358,16 +382,19 @@ __device__ __forceinline__ int prefix_len(const PrefillParams &p, const Item &it
         const int seg_len = p.cu[it.seg + 1] - p.cu[it.seg];
         return p.causal ? min(pos - p.cu[it.seg] + 1, seg_len) : seg_len;
     }
-    if (p.remote_only) {                               // what lies before the row's own segment
+    if (kSpecial && p.remote_only) {                   // what lies before the row's own segment
         const int before = p.cu[it.seg];
-        return it.kvp ? count_le(it.kvp, T, before - 1) : min(before, T);
+        return it.kvp ? count_le_warp(it.kvp, T, before - 1, lane) : min(before, T);
     }
     if (!p.causal) return T;
     if (!it.kvp) return min(pos + 1, T);
-    return count_le(it.kvp, T, pos);
+    return count_le_warp(it.kvp, T, pos, lane);
 }
 
-__device__ __forceinline__ Item decode_item(const KernelParams &kp, int item)
+// Called by a converged warp (all lanes get the same item).  kSpecial: the kernel instance that also
+// serves explicit positions and remote-only attention; the plain instance carries none of their state.
+template <bool kSpecial>
+__device__ __forceinline__ Item decode_item(const KernelParams &kp, int item, int lane)
 {
     const PrefillParams &p = kp.p;
     Item it;
@@ -399,23 +426,27 @@ __device__ __forceinline__ Item decode_item(const KernelParams &kp, int item)
     it.kvp = p.kv_pos ? p.kv_pos + (p.kv_head_major ? (int64_t)it.kvh * p.total_kv : 0) : nullptr;
     it.kv_begin = p.sync ? 0 : p.cu[seg];
     it.t_b0 = 0; it.a = 0; it.b = 0;
-    if (p.general) {
+    if (kSpecial && p.general) {
         // tiles up to the last one that holds a key position <= the tile's largest query position
         const PosTables pt = pos_tables(p.tab, kp.n_qtiles, p.kv_head_major ? p.hkv : 1, kp.n_kt);
         const int32_t *suf = pt.suf_min + (p.kv_head_major ? (size_t)it.kvh * kp.n_kt : 0);
-        it.n_tiles = count_le(suf, kp.n_kt, __ldg(pt.q_max + (it.q_row0 >> 7)));
+        it.n_tiles = count_le_warp(suf, kp.n_kt, __ldg(pt.q_max + (it.q_row0 >> 7)), lane);
         it.n_a = it.n_tiles;
-    } else if (p.sync && p.remote_only && !p.causal) {
-        // keys [0, a) lie before the row's segment, keys [b, T) after it
+    } else if (kSpecial && p.sync && p.remote_only) {
+        // keys [0, a) lie before the rows' segment; when bidirectional, keys [b, T) after it count too
         const int T = (int)p.total_kv, n_t = (T + kTileN - 1) / kTileN;
-        it.a = prefix_len(p, it, 0);
-        const int after = p.cu[seg + 1];
-        it.b = it.kvp ? count_le(it.kvp, T, after - 1) : min(after, T);
+        it.a = prefix_len<kSpecial>(p, it, 0, lane);
         it.n_a = (it.a + kTileN - 1) / kTileN;
-        it.t_b0 = it.b >= T ? n_t : max(it.b / kTileN, it.n_a);
-        it.n_tiles = it.n_a + (n_t - it.t_b0);
+        it.n_tiles = it.n_a;
+        it.b = T;
+        if (!p.causal) {
+            const int after = p.cu[seg + 1];
+            it.b = it.kvp ? count_le_warp(it.kvp, T, after - 1, lane) : min(after, T);
+            it.t_b0 = it.b >= T ? n_t : max(it.b / kTileN, it.n_a);
+            it.n_tiles = it.n_a + (n_t - it.t_b0);
+        }
     } else {
-        it.n_tiles = (prefix_len(p, it, it.n_valid - 1) + kTileN - 1) / kTileN;
+        it.n_tiles = (prefix_len<kSpecial>(p, it, it.n_valid - 1, lane) + kTileN - 1) / kTileN;
         it.n_a = it.n_tiles;
     }
     return it;
@@ -425,6 +456,7 @@ __device__ __forceinline__ Item decode_item(const KernelParams &kp, int item)
 // Barrier phases run on: per-CTA counters of KV tiles (git) and of non-empty items (qn) give stages
 // and parities, so the producer prefetches the next item's K/V and Q while the current item's last
 // tiles and its epilogue are still in flight.
+template <bool kSpecial>
 __global__ void __launch_bounds__(kThreads, 1)
 prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                      const __grid_constant__ CUtensorMap map_v, const __grid_constant__ KernelParams kp)
@@ -486,16 +518,20 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     if (warp == kProducerWarp) {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kOtherRegs));
         // ================= TMA producer =================
+        // The whole warp decodes the work items (their searches are warp-cooperative); lane 0 waits and
+        // issues the copies.
         if (lane == 0) {
             asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&map_q) : "memory");
             asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&map_k) : "memory");
             asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&map_v) : "memory");
-            int git = 0, qn = 0;
-            for (int k = 0; k < n_rounds; ++k) {
-                const int item = item_of(k);
-                if (item >= n_items) continue;
-                const Item it = decode_item(kp, item);
-                if (it.n_tiles == 0) continue;
+        }
+        int git = 0, qn = 0;
+        for (int k = 0; k < n_rounds; ++k) {
+            const int item = item_of(k);
+            if (item >= n_items) continue;
+            const Item it = decode_item<kSpecial>(kp, item, lane);
+            if (it.n_tiles == 0) continue;
+            if (lane == 0) {
                 if (qn > 0) mbar_wait(q_empty, (qn - 1) & 1, abort_flag, kp.status);   // previous item's S MMAs done
                 item_info[(qn & 1) * 2] = it.n_tiles;
                 item_info[(qn & 1) * 2 + 1] = it.valid1 ? 2 : 1;
@@ -508,7 +544,7 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                 }
                 for (int j = 0; j < it.n_tiles; ++j) {
                     const int gt = git + j, st = gt & 1, use = gt >> 1;
-                    const int row = it.kv_begin + tile_of(it, j) * kTileN;
+                    const int row = it.kv_begin + (kSpecial ? tile_of(it, j) : j) * kTileN;
                     const int c1 = p.kv_head_major ? row : it.kvh, c2 = p.kv_head_major ? it.kvh : row;
                     if (gt >= 2) mbar_wait(k_empty + st, (use - 1) & 1, abort_flag, kp.status);
                     TRACE(j, 7);
@@ -520,9 +556,12 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                     tma_load_3d(sV + st * kTileBytes, &map_v, v_full + st, 0, c1, c2);
                     tma_load_3d(sV + st * kTileBytes + kHalfBytes, &map_v, v_full + st, 64, c1, c2);
                 }
-                git += it.n_tiles;
-                ++qn;
             }
+            __syncwarp();
+            git += it.n_tiles;
+            ++qn;
+        }
+        if (lane == 0) {
             // end marker for the MMA issuer, in the slot and phase the next item would have used
             if (qn > 0) mbar_wait(q_empty, (qn - 1) & 1, abort_flag, kp.status);
             item_info[(qn & 1) * 2] = -1;
@@ -563,7 +602,8 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         // count only the items in which the pair's second head exists.
         int git = 0, qn = 0, git1 = 0, qn1 = 0;
         for (;;) {
-            // the producer decodes the work items; this warp only learns their shape
+            // the producer decodes the work items; this warp only learns their shape (decoding them here as
+            // well does not fit into this role's 64 registers)
             if (!mbar_wait(q_full, qn & 1, abort_flag, kp.status)) break;
             const int n = item_info[(qn & 1) * 2];
             if (n < 0) break;
@@ -749,7 +789,7 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         for (k = 0; k < n_rounds; ++k) {
             const int item = item_of(k);
             if (item >= n_items) continue;
-            const Item it = decode_item(kp, item);
+            const Item it = decode_item<kSpecial>(kp, item, lane);
             const int n_tiles = it.n_tiles;
             const int n_sub = it.valid1 ? 2 : 1;
             const bool valid = r < it.n_valid;
@@ -766,18 +806,35 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                 }
                 continue;
             }
-            const bool two_range = p.sync && p.remote_only && !p.causal;
+            const bool two_range = kSpecial && p.sync && p.remote_only && !p.causal;
+            const bool general = kSpecial && p.general;
             int c_row = 0, n_full = 0, p_row = 0;
-            if (p.general) {
+            if (general) {
                 // every (query, key) pair on its own positions; the tiles whose keys all lie at or below the
                 // tile's smallest query position (a prefix of the walk, see PosTables) need no test
                 const PosTables pt = pos_tables(p.tab, kp.n_qtiles, p.kv_head_major ? p.hkv : 1, kp.n_kt);
                 const int32_t *pre = pt.pre_max + (p.kv_head_major ? (size_t)it.kvh * kp.n_kt : 0);
-                n_full = count_le(pre, kp.n_kt, __ldg(pt.q_min + (it.q_row0 >> 7)));
+                n_full = count_le_warp(pre, kp.n_kt, __ldg(pt.q_min + (it.q_row0 >> 7)), lane);
                 const int row = it.q_row0 + min(r, it.n_valid - 1);
                 p_row = p.q_pos ? __ldg(p.q_pos + row) : row;
             } else {
-                c_row = prefix_len(p, it, r);
+                if (kSpecial && p.sync && p.remote_only) {
+                    c_row = it.a;                               // the same for every row of the segment
+                } else if (p.sync && p.causal && it.kvp) {
+                    // Sparse aggregate, row position = row index.  One cooperative search gives the keys
+                    // visible to all of the warp's 32 consecutive rows; the next 32 keys are the only ones
+                    // that can tell these rows apart (more only if positions repeat: then each lane searches).
+                    const int T = (int)p.total_kv, p0 = it.q_row0 + (r & ~31);
+                    const int cw = count_le_warp(it.kvp, T, p0 - 1, lane);
+                    const int wv = cw + lane < T ? __ldg(it.kvp + cw + lane) : INT32_MAX;
+                    int cnt = 0;
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) cnt += __shfl_sync(0xffffffffu, wv, j) <= p0 + lane;
+                    c_row = cw + cnt;
+                    if (__shfl_sync(0xffffffffu, wv, 31) <= p0 + 31) c_row = count_le(it.kvp, T, p0 + lane);
+                } else {
+                    c_row = prefix_len<kSpecial>(p, it, r, lane);   // arithmetic only
+                }
                 // prefix lengths do not decrease with the row, so KV tiles below the prefix of the warp's first
                 // row are unmasked for the whole warp (the choice of code path only has to be warp-uniform)
                 n_full = __shfl_sync(0xffffffffu, c_row, 0) / kTileN;
@@ -803,7 +860,7 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                     }
                 } else if (j < n_full) {
                     visit(std::false_type{}, t, j, gt, 0, m_a, l_a);
-                } else if (p.general) {
+                } else if (general) {
                     // column c is key cb + c: visible iff it exists and its position is not above the row's.
                     // The address is the same in every lane: broadcast loads.
                     const int cb = j * kTileN + kCols * hf;
@@ -1067,7 +1124,9 @@ cudaError_t launch_prefill_sm100(Context *ctx, const PrefillParams &p, cudaStrea
         return cudaErrorInvalidValue;
     static bool attr_set[64] = {};
     if (!attr_set[ctx->device & 63]) {
-        cudaError_t e = cudaFuncSetAttribute(prefill_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        cudaError_t e = cudaFuncSetAttribute(prefill_sm100_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(prefill_sm100_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
         if (e != cudaSuccess) {
             if (getenv("FEDATTN_DEBUG")) fprintf(stderr, "prefill_sm100_kernel attribute: %s\n", cudaGetErrorString(e));
             return e;
@@ -1083,7 +1142,10 @@ cudaError_t launch_prefill_sm100(Context *ctx, const PrefillParams &p, cudaStrea
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
     }
-    prefill_sm100_kernel<<<(unsigned)blocks, kThreads, kSmemBytes, s>>>(mq, mk, mv, kp);
+    // the plain instance serves local attention and sync attention under the prefix mask; explicit positions
+    // and remote-only attention run the instance that carries their extra state
+    if (p.general || p.remote_only) prefill_sm100_kernel<true><<<(unsigned)blocks, kThreads, kSmemBytes, s>>>(mq, mk, mv, kp);
+    else prefill_sm100_kernel<false><<<(unsigned)blocks, kThreads, kSmemBytes, s>>>(mq, mk, mv, kp);
     ++ctx->launches;
     ++ctx->tc_launches;
     cudaError_t e = cudaGetLastError();

@@ -238,6 +238,38 @@ def test_topk_zero_and_subnormal_terms(oracle, d):
         assert np.array_equal(host(agg["k_agg"]), ka) and np.array_equal(host(agg["v_agg"]), va)
 
 
+@pytest.mark.parametrize("d", [128, 64])
+def test_topk_scores_around_the_exactness_bound(oracle, d):
+    """The bf16 score kernel sums a row in tree order when it can prove that no addition of the defined
+    chain rounds (row sum below 2^53 times the smallest term's unit), and walks the chain otherwise.
+    Rows built around that bound: groups of rows that share their large elements and differ only in a
+    tiny element (exponents on both sides of the bound, full and minimal mantissa) and in where it
+    sits in the row, so that inside a group the order is decided by the last bits of the score."""
+    rng = np.random.default_rng(31)
+    hkv, groups, per_group = 2, 90, 8
+    L = groups * per_group
+    base = fi.round_to_bf16(rng.standard_normal((groups, 1, hkv, d)).astype(np.float32) * np.float32(2.0))
+    k = np.repeat(base, per_group, axis=1).reshape(L, hkv, d).copy()
+    tiny_exp = [-18, -17, -16, -15, -14, -13]                        # the bound sits near 2^-16 .. 2^-15 for sums of a few hundred
+    for g in range(groups):
+        for j in range(per_group):
+            row = g * per_group + j
+            e = tiny_exp[(g + j) % len(tiny_exp)]
+            mant = np.float32(1.9921875) if (g // 2 + j) % 2 else np.float32(1.0)     # 8-bit mantissa 0xff or 0x80
+            col = [0, d // 2, d - 1, 3][j % 4]
+            k[row, :, col] = mant * np.float32(2.0) ** e * (1 if j % 2 else -1)
+    k = fi.round_to_bf16(k)
+    v = fi.round_to_bf16(rng.standard_normal((L, hkv, d)).astype(np.float32))
+    kp, vp = [k[:L // 2], k[L // 2:]], [v[:L // 2], v[L // 2:]]
+    r = Runner(2, hkv, hkv, d, "bf16", L)
+    for ksel in ([L // 4, L // 4], [101, 257], [7, 355], [L // 2 - 3, 1]):
+        agg = r.aggregate(fa().AGG_TOPK_KNORM, kp, vp, ksel)
+        ka, va, pos, cu, sel = oracle.aggregate_topk(kp, vp, ksel)
+        assert agg["status"] == 0
+        assert np.array_equal(agg["sel_idx"].cpu().numpy(), sel), ksel
+        assert np.array_equal(host(agg["k_agg"]), ka) and np.array_equal(host(agg["v_agg"]), va)
+
+
 @pytest.mark.parametrize("dtype,hq,hkv,d", [("bf16", 8, 2, 128), ("bf16", 32, 8, 128), ("f32", 4, 2, 64)])
 def test_token_level_selection_and_sync_over_it(oracle, dtype, hq, hkv, d):
     """Token-level selection: one score per token over all KV heads (a chain of Hkv * d terms), indices
