@@ -59,9 +59,11 @@ N_SETS = 3            # rotating input sets: ~600 MB touched per cycle, larger t
 SPARSE_RATIO_NUM, SPARSE_RATIO_DEN = 1, 4
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
 # profiles/ (None: the kernel has changed since its counters were taken)
-PREFILL_SYNC_DRAM_BYTES = None      # prefill_sm100_kernel, the cfg2 sync launch
-DECODE_DRAM_BYTES = None            # decode_stream_kernel + decode_merge_kernel, one cfg5 call
-TOPK_DRAM_BYTES = None              # topk_fused_kernel, one cfg4 sparse aggregation
+PREFILL_DRAM_BYTES = 374_249_000        # prefill_sm100_kernel, the three cfg2 launches the roofline covers: local 137.1 MB,
+                                        # sync 134.9 MB, sparse sync 102.2 MB (read + written)
+DECODE_DRAM_BYTES = 140_620_000         # one cfg5 call: decode_stream_kernel 138.45 MB + decode_merge_kernel 2.17 MB
+                                        # (the merge reads its partials from DRAM only under the profiler's cache flush)
+TOPK_DRAM_BYTES = 42_225_000            # topk_fused_kernel, one cfg4 sparse aggregation (42.0 MB read + 0.2 MB written)
 NOMINAL_TENSOR, NOMINAL_HBM = 2250.0, 8000.0     # B200 spec: dense bf16 TFLOP/s, HBM3e GB/s
 MIN_REGION_S = 0.2                  # every microsecond-scale leg is timed over a region at least this long
 
@@ -365,7 +367,7 @@ def run_ours(args):
                          "frac": round(achieved / pk["tensor"], 4), "peak_kind": "burst bf16, " + pk["kind"],
                          "frac_of_sustained": round(achieved / pk["tensor_sustained"], 4) if pk["tensor_sustained"] else None,
                          "frac_of_nominal_2250": round(achieved / NOMINAL_TENSOR, 4),
-                         "traffic": PREFILL_SYNC_DRAM_BYTES},
+                         "traffic": PREFILL_DRAM_BYTES},
             "calls": calls,
             "step_tflop": round(step_flops / 1e12, 5),
         }
@@ -524,6 +526,7 @@ EVENTS = "CUDA events on the launching stream around back-to-back calls, region 
 
 def leg_cfg5(args, quick=False):
     """Decode: N=8 caches x 4096 tokens; a step = 3 local calls + 1 sync call (sync every H=4)."""
+    quick = quick or args.quick
     torch, fa, dev = _setup()
     w = fi.cfg5()
     N, Hq, Hkv, d, L = w.n_participants, w.n_q_heads, w.n_kv_heads, w.head_dim, w.total_tokens
@@ -567,12 +570,13 @@ def leg_cfg5(args, quick=False):
     W = max(args.warmup, 3)
     floor = 0.0 if quick else MIN_REGION_S
     sampler = ClockSampler(0); sampler.start(); time.sleep(0.25)
-    ms_local = _timed(torch, stream, lambda i: call(i, False), 400, W, floor)
-    ms_sync = _timed(torch, stream, lambda i: call(i, True), 400, W, floor)
+    n_it = 8 if quick else 400
+    ms_local = _timed(torch, stream, lambda i: call(i, False), n_it, W, floor)
+    ms_sync = _timed(torch, stream, lambda i: call(i, True), n_it, W, floor)
     l0 = ctx.launch_count()
     step(0)
     launches = ctx.launch_count() - l0
-    ms_step = _timed(torch, stream, step, 100, W, floor)
+    ms_step = _timed(torch, stream, step, 4 if quick else 100, W, floor)
     time.sleep(0.25); clocks = sampler.stop()
     assert ctx.poll() == 0
 
@@ -580,17 +584,17 @@ def leg_cfg5(args, quick=False):
         qs[i % n_q].copy_(hq[i % n_q], non_blocking=True)
         step(i)
         ho.copy_(o, non_blocking=True)
-    ms_e2e = _timed(torch, stream, e2e_step, 50, 2)
+    ms_e2e = _timed(torch, stream, e2e_step, 2 if quick else 50, 2)
 
-    g_local = _graph_timed(torch, lambda i, st: call(i, False, st), 2 * n_sets)
-    g_sync = _graph_timed(torch, lambda i, st: call(i, True, st), 2 * n_sets)
+    g_local = None if quick else _graph_timed(torch, lambda i, st: call(i, False, st), 2 * n_sets)
+    g_sync = None if quick else _graph_timed(torch, lambda i, st: call(i, True, st), 2 * n_sets)
     kv_bytes = 2 * L * Hkv * d * 2 + 2 * N * Hq * d * 2        # per call: every K/V row once + q + o
     pk = peaks()
     calls = {"decode_local": _hbm_call(pk, kv_bytes, ms_local, g_local), "decode_sync": _hbm_call(pk, kv_bytes, ms_sync, g_sync),
              "decode_step_3local_1sync": _hbm_call(pk, 4 * kv_bytes, ms_step)}
     calls["decode_step_3local_1sync"]["launches"] = launches
     roof = _hbm_roofline(pk, "decode_stream_kernel + decode_merge_kernel (two launches per decode call; 3 local + 1 sync)",
-                         4 * kv_bytes, ms_step, DECODE_DRAM_BYTES, EVENTS)
+                         4 * kv_bytes, ms_step, 4 * DECODE_DRAM_BYTES, EVENTS)
     return {"calls": calls, "rooflines": {"decode": roof}, "launches": launches, "ms_step": ms_step, "clocks": clocks,
             "metric": "fedattn_decode_gbs", "unit": "GB/s", "value": 4 * kv_bytes / (ms_step * 1e-3) / 1e9,
             "config": {"workload": w.name, "participants": N, "cache_tokens": seqlens[0], "q_heads": Hq, "kv_heads": Hkv, "head_dim": d,
@@ -604,6 +608,7 @@ def leg_cfg5(args, quick=False):
 def leg_cfg4(args, quick=False):
     """Sparse aggregation (top 256 of 1024 keys per participant and KV head) + sync over the selected KV,
     and the exchange block that keeps the own segment complete (top-k and seeded random selection)."""
+    quick = quick or args.quick
     torch, fa, dev = _setup()
     w = fi.cfg4()
     N, Hq, Hkv, d, L = w.n_participants, w.n_q_heads, w.n_kv_heads, w.head_dim, w.total_tokens
@@ -675,18 +680,19 @@ def leg_cfg4(args, quick=False):
     f_sync = 4.0 * d * (Hq // Hkv) * pairs
     f_exch = 4.0 * d * Hq * (sum(n * (n + 1) // 2 for n in seqlens) + sum(seqlens[n] * sum(ksel[:n]) for n in range(N)))
     sampler = ClockSampler(0); sampler.start(); time.sleep(0.25)
-    ms_agg = _timed(torch, stream, agg, 200, W, floor)
-    ms_tok = _timed(torch, stream, agg_tok, 200, W, floor)
+    n_it = 8 if quick else 200
+    ms_agg = _timed(torch, stream, agg, n_it, W, floor)
+    ms_tok = _timed(torch, stream, agg_tok, n_it, W, floor)
     ms_sync = _timed(torch, stream, sync, K, W)
     ms_exch = _timed(torch, stream, exchange, K, W)
     l0 = ctx.launch_count()
     step(0)
     launches = ctx.launch_count() - l0
     ms_step = _timed(torch, stream, step, K, W)
-    g_agg = _graph_timed(torch, agg, 2 * n_sets)
-    g_tok = _graph_timed(torch, agg_tok, 2 * n_sets)
+    g_agg = None if quick else _graph_timed(torch, agg, 2 * n_sets)
+    g_tok = None if quick else _graph_timed(torch, agg_tok, 2 * n_sets)
     # the random draw last: it overwrites the sparse aggregate of every set
-    ms_rand = _timed(torch, stream, agg_rand, 200, W, floor)
+    ms_rand = _timed(torch, stream, agg_rand, n_it, W, floor)
     ms_exch_rand = _timed(torch, stream, exchange_random, K, W)
     time.sleep(0.25); clocks = sampler.stop()
     assert ctx.poll() == 0
@@ -1021,6 +1027,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--workload", default="all", choices=["all", "cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
+    ap.add_argument("--quick", action="store_true",
+                    help="few iterations per leg and no graph replays (keeps a profiler capture short)")
     ap.add_argument("--sets", type=int, default=N_SETS,
                     help="rotating input sets (1 keeps device memory small for a profiler capture)")
     args = ap.parse_args()
