@@ -634,8 +634,9 @@ def leg_cfg4(args, quick=False):
     ho = torch.empty((L, Hq, d), dtype=bf).pin_memory()
     # a seeded random selection at the same ratio: the draw is an input (int32 [Hkv, T] local indices)
     sel_rand = torch.from_numpy(fi.random_selection(w.seed, seqlens, ksel, Hkv)).to(dev)
-    k_tok = torch.empty((T, Hkv, d), dtype=bf, device=dev); v_tok = torch.empty_like(k_tok)
-    pos_tok = torch.empty((T,), dtype=torch.int32, device=dev); sel_tok = torch.empty_like(pos_tok)
+    for b in sets:                                       # token-level outputs, one set per input set like the rest
+        b["k_tok"] = torch.empty((T, Hkv, d), dtype=bf, device=dev); b["v_tok"] = torch.empty_like(b["k_tok"])
+        b["pos_tok"] = torch.empty((T,), dtype=torch.int32, device=dev); b["sel_tok"] = torch.empty_like(b["pos_tok"])
     o_b = torch.empty_like(sets[0]["q"])
     lse_a = torch.empty((L, Hq), dtype=torch.float32, device=dev); lse_b = torch.empty_like(lse_a)
 
@@ -643,8 +644,8 @@ def leg_cfg4(args, quick=False):
         return dict(
             agg=fa.prepare_aggregate_kv(ctx, shape, fa.AGG_TOPK_KNORM, b["kp"], b["vp"], seqlens, ksel, None, b["k_sp"], b["v_sp"],
                                         b["pos"], None, b["sel"]),
-            agg_tok=fa.prepare_aggregate_kv(ctx, shape, fa.AGG_TOPK_TOKEN, b["kp"], b["vp"], seqlens, ksel, None, k_tok, v_tok,
-                                            pos_tok, None, sel_tok),
+            agg_tok=fa.prepare_aggregate_kv(ctx, shape, fa.AGG_TOPK_TOKEN, b["kp"], b["vp"], seqlens, ksel, None, b["k_tok"],
+                                            b["v_tok"], b["pos_tok"], None, b["sel_tok"]),
             agg_rand=fa.prepare_aggregate_kv(ctx, shape, fa.AGG_INDEXED, b["kp"], b["vp"], seqlens, ksel, sel_rand, b["k_sp"],
                                              b["v_sp"], b["pos"], None, None),
             sync=fa.prepare_sync(ctx, shape, b["q"], None, b["k_sp"], b["v_sp"], b["pos"], T, True, b["o"]),

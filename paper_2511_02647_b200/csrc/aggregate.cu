@@ -127,6 +127,9 @@ topk_fused_kernel(const PartsParams pp, int hkv, int vpr /* 16-byte vectors per 
                   int n_stages /* buffers in every warp's staging ring, 2..4 */,
                   int max_len /* longest participant: sizes the key arrays */,
                   int early /* the inputs may be read before the preceding grid of the stream is complete */,
+                  long long my_seq /* this call's sequence number in its context */,
+                  long long need_seq /* the latest call that writes one of this call's outputs (0: none) */,
+                  long long *done_seq /* the context's word: largest sequence number known to be complete */,
                   uint4 *k_agg, uint4 *v_agg, int32_t *kv_pos, int32_t *cu_kv, int32_t *sel_idx_out)
 {
     // dynamic shared memory: keys [max_len] u64 | kept rows [max_len] u16 | staging [8 warps][n_stages][32 rows][128 B]
@@ -144,18 +147,34 @@ topk_fused_kernel(const PartsParams pp, int hkv, int vpr /* 16-byte vectors per 
     cg::cluster_group cluster = cg::this_cluster();
     const int h = blockIdx.x, n = blockIdx.y, slice = blockIdx.z, n_slices = gridDim.z;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    // Launched with programmatic stream serialization: the dependents may take their seats at once, and
-    // this kernel waits for the preceding grid only before its first write (the outputs of an earlier
-    // call may still be read or written by it) unless its inputs might be that grid's outputs.
+    // Launched with programmatic stream serialization: the dependents may take their seats at once.
+    // Inputs are read before the preceding grid of the stream is known to be complete unless they might be
+    // its outputs (early == 0).  Outputs are written at once when every earlier call that writes the same
+    // buffers is known to be over (*done_seq >= need_seq), else after griddepcontrol.wait.  One CTA of the
+    // grid always waits for the preceding grid before it exits: a grid must not complete before its
+    // predecessor, or what follows in the stream could overtake earlier work; that CTA then records that
+    // every call before this one is complete.
     if (!early) asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    const bool closer = h == 0 && n == 0 && slice == 0;
+    auto close_call = [&]() {
+        if (closer) {
+            asm volatile("griddepcontrol.wait;" ::: "memory");
+            if (tid == 0) atomicMax(reinterpret_cast<unsigned long long *>(done_seq), (unsigned long long)(my_seq - 1));
+        }
+    };
+    auto may_write = [&]() {                                  // CTA-uniform
+        if (need_seq > 0 && *reinterpret_cast<volatile long long *>(done_seq) < need_seq)
+            asm volatile("griddepcontrol.wait;" ::: "memory");
+    };
     const int len = pp.off[n + 1] - pp.off[n];
     const int k = pp.cu_kv[n + 1] - pp.cu_kv[n];
     if (k == 0 || len == 0) {                                 // the same for every slice of the cluster
-        if (h == 0 && n == 0 && slice == 0 && cu_kv && tid <= pp.n) {
-            asm volatile("griddepcontrol.wait;" ::: "memory");
+        if (closer && cu_kv && tid <= pp.n) {
+            may_write();
             cu_kv[tid] = pp.cu_kv[tid];
         }
+        close_call();
         return;
     }
     const int64_t T = pp.cu_kv[pp.n];
@@ -396,15 +415,15 @@ topk_fused_kernel(const PartsParams pp, int hkv, int vpr /* 16-byte vectors per 
     }
     __syncthreads();
 
-    // gather this slice: rows my_rows[0 .. o_hi - o_lo) of participant n, head h.  First write of this
-    // kernel: the preceding grid of the stream must be complete.
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    if (h == 0 && n == 0 && slice == 0 && cu_kv && tid <= pp.n) cu_kv[tid] = pp.cu_kv[tid];
+    // gather this slice: rows my_rows[0 .. o_hi - o_lo) of participant n, head h.  First write of this kernel.
+    may_write();
+    if (closer && cu_kv && tid <= pp.n) cu_kv[tid] = pp.cu_kv[tid];
     const int n_out = o_hi - o_lo;
     const int64_t out_row0 = (int64_t)h * T + pp.cu_kv[n] + o_lo;
     const uint4 *ksrc = reinterpret_cast<const uint4 *>(pp.k[n]), *vsrc = reinterpret_cast<const uint4 *>(pp.v[n]);
-    // four vectors of K and of V in flight per thread before the first store
-    constexpr int kGatherUnroll = 4;
+    // eight vectors of K and of V in flight per thread before the first store (a CTA gathers its rows in a few
+    // round trips to memory: the gather is bound by that latency, not by bandwidth)
+    constexpr int kGatherUnroll = 8;
     for (int i0 = tid; i0 < n_out * vpr; i0 += kSelThreads * kGatherUnroll) {
         uint4 kk[kGatherUnroll], vv[kGatherUnroll];
 #pragma unroll
@@ -433,15 +452,20 @@ topk_fused_kernel(const PartsParams pp, int hkv, int vpr /* 16-byte vectors per 
         if (sel_idx_out) sel_idx_out[out_row0 + r] = my_rows[r];
     }
     asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+    close_call();
 }
 
 cudaError_t launch_topk_fused(const PartsParams &pp, int hkv, int d, int dtype, void *k_agg, void *v_agg,
-                              int32_t *kv_pos, int32_t *cu_kv, int32_t *sel_idx_out, int device, int sm_count,
-                              cudaStream_t s, int64_t *launches)
+                              int32_t *kv_pos, int32_t *cu_kv, int32_t *sel_idx_out, Context *ctx, cudaStream_t s)
 {
+    const int device = ctx->device, sm_count = ctx->sm_count;
+    int64_t *launches = &ctx->launches;
     if (pp.cu_kv[pp.n] == 0 && !cu_kv) return cudaSuccess;
     const int elt = dtype == FEDATTN_BF16 ? 2 : 4;
     int early;
+    long long *done_seq = reinterpret_cast<long long *>(ctx->workspace + kDoneSeqOffset);
+    const long long my_seq = ++ctx->agg_seq;
+    int64_t need_seq = 0;
     {
         const size_t row_bytes = (size_t)hkv * d * elt;
         const size_t T = (size_t)pp.cu_kv[pp.n];
@@ -453,7 +477,7 @@ cudaError_t launch_topk_fused(const PartsParams &pp, int hkv, int d, int dtype, 
         }
         const MemRange out[5] = {{k_agg, T * row_bytes}, {v_agg, T * row_bytes}, {kv_pos, kv_pos ? T * hkv * 4 : 0},
                                  {cu_kv, cu_kv ? (size_t)(pp.n + 1) * 4 : 0}, {sel_idx_out, sel_idx_out ? T * hkv * 4 : 0}};
-        early = early_read_allowed(device, in, 2 * pp.n, out, 5) ? 1 : 0;
+        early = early_read_allowed(device, in, 2 * pp.n, out, 5, done_seq, my_seq, &need_seq) ? 1 : 0;
     }
     const int vpr = d * elt / 16;
     int max_len = 0;
@@ -496,10 +520,10 @@ cudaError_t launch_topk_fused(const PartsParams &pp, int hkv, int d, int dtype, 
     cfg.attrs = attr;
     cfg.numAttrs = 2;
     cudaError_t e = dtype == FEDATTN_BF16
-                        ? cudaLaunchKernelEx(&cfg, topk_fused_kernel<FEDATTN_BF16>, pp, hkv, vpr, n_stages, max_len, early,
-                                             (uint4 *)k_agg, (uint4 *)v_agg, kv_pos, cu_kv, sel_idx_out)
-                        : cudaLaunchKernelEx(&cfg, topk_fused_kernel<FEDATTN_F32>, pp, hkv, vpr, n_stages, max_len, early,
-                                             (uint4 *)k_agg, (uint4 *)v_agg, kv_pos, cu_kv, sel_idx_out);
+                        ? cudaLaunchKernelEx(&cfg, topk_fused_kernel<FEDATTN_BF16>, pp, hkv, vpr, n_stages, max_len, early, my_seq,
+                                             (long long)need_seq, done_seq, (uint4 *)k_agg, (uint4 *)v_agg, kv_pos, cu_kv, sel_idx_out)
+                        : cudaLaunchKernelEx(&cfg, topk_fused_kernel<FEDATTN_F32>, pp, hkv, vpr, n_stages, max_len, early, my_seq,
+                                             (long long)need_seq, done_seq, (uint4 *)k_agg, (uint4 *)v_agg, kv_pos, cu_kv, sel_idx_out);
     ++*launches;
     return e != cudaSuccess ? e : cudaGetLastError();
 }

@@ -103,6 +103,7 @@ fedattn_status fedattn_create(fedattn_ctx **out, int device, void *workspace, si
     c.scratch_bytes = workspace_bytes - kStatusBytes;
     c.launches = 0;
     c.tc_launches = 0;
+    c.agg_seq = 0;
     c.encode_tiled = nullptr;
     if (prop.major == 10) {
         void *fn = nullptr;
@@ -236,14 +237,12 @@ fedattn_status fedattn_aggregate_kv(fedattn_ctx *ctx, const fedattn_shape *shape
         return err == cudaSuccess ? FEDATTN_OK : FEDATTN_ERR_CUDA;
     }
     if (mode == FEDATTN_AGG_TOPK_KNORM) {
-        err = launch_topk_fused(pp, hkv, d, shape->dtype, k_agg, v_agg, kv_pos, cu_kv, sel_idx_out, ctx->c.device,
-                                ctx->c.sm_count, s, &ctx->c.launches);
+        err = launch_topk_fused(pp, hkv, d, shape->dtype, k_agg, v_agg, kv_pos, cu_kv, sel_idx_out, &ctx->c, s);
         return err == cudaSuccess ? FEDATTN_OK : FEDATTN_ERR_CUDA;
     }
     if (mode == FEDATTN_AGG_TOPK_TOKEN) {
         // the per-head kernel on the token row viewed as one head of Hkv * d channels: token-major output
-        err = launch_topk_fused(pp, 1, hkv * d, shape->dtype, k_agg, v_agg, kv_pos, cu_kv, sel_idx_out, ctx->c.device,
-                                ctx->c.sm_count, s, &ctx->c.launches);
+        err = launch_topk_fused(pp, 1, hkv * d, shape->dtype, k_agg, v_agg, kv_pos, cu_kv, sel_idx_out, &ctx->c, s);
         return err == cudaSuccess ? FEDATTN_OK : FEDATTN_ERR_CUDA;
     }
     const int32_t *sel = sel_idx_in;

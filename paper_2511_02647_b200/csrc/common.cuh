@@ -9,8 +9,10 @@
 
 namespace fedattn {
 
-// Workspace layout: [0, 256) status words, then the scratch region.
+// Workspace layout: [0, 256) status area (word 0: the status word; bytes 64..71: the sequence number of the
+// latest sparse aggregation known to be complete), then the scratch region.
 constexpr size_t kStatusBytes = 256;
+constexpr size_t kDoneSeqOffset = 64;
 constexpr int kMaxP = FEDATTN_MAX_PARTICIPANTS;
 // Upper bound on spin iterations of any in-kernel wait before it gives up.
 constexpr uint32_t kSpinLimit = 1u << 22;
@@ -25,6 +27,7 @@ struct Context {
     size_t scratch_bytes;
     int64_t launches;
     int64_t tc_launches;   // launches of the tcgen05 attention kernel among them
+    int64_t agg_seq;       // sequence number of the latest sparse aggregation call
     void *encode_tiled;    // cuTensorMapEncodeTiled entry point (driver), or nullptr
 };
 
@@ -36,7 +39,11 @@ struct MemRange {
 // Records `out` as buffers that grids of this call may still be writing when later grids start, and
 // returns whether this call may read `in` before the preceding grid of the stream is complete (false:
 // it must wait first).  n_out <= 16.
-bool early_read_allowed(int device, const MemRange *in, int n_in, const MemRange *out, int n_out);
+// owner / seq: the context's sequence counter for this call (null / 0: none).  need_seq (nullable) receives the
+// largest sequence number of the owner's recorded calls that write one of `out` (0: none; INT64_MAX: a writer
+// that cannot be named, wait before writing).
+bool early_read_allowed(int device, const MemRange *in, int n_in, const MemRange *out, int n_out,
+                        const void *owner = nullptr, int64_t seq = 0, int64_t *need_seq = nullptr);
 
 // ---- generic SIMT attention (fp32 or bf16 storage, any head_dim <= 128) --------------------
 enum GenericMode { kLocal = 0, kSync = 1, kDecodeLocal = 2, kDecodeSync = 3 };
@@ -79,8 +86,7 @@ cudaError_t launch_concat(const PartsParams &pp, int hkv, int d, int elt_bytes, 
                           int32_t *kv_pos, int32_t *cu_kv, cudaStream_t s, int sm_count, int64_t *launches);
 
 cudaError_t launch_topk_fused(const PartsParams &pp, int hkv, int d, int dtype, void *k_agg, void *v_agg,
-                              int32_t *kv_pos, int32_t *cu_kv, int32_t *sel_idx_out, int device, int sm_count,
-                              cudaStream_t s, int64_t *launches);
+                              int32_t *kv_pos, int32_t *cu_kv, int32_t *sel_idx_out, Context *ctx, cudaStream_t s);
 cudaError_t launch_gather(const PartsParams &pp, int hkv, int d, int elt_bytes, const int32_t *sel_idx,
                           void *k_agg, void *v_agg, int32_t *kv_pos, int32_t *cu_kv, int32_t *sel_idx_out,
                           int32_t *status, int sm_count, cudaStream_t s, int64_t *launches);

@@ -9,6 +9,14 @@
 // call that waited first.  A call whose inputs overlap a recorded buffer, or whose outputs would not
 // fit into the record, waits first; its grids then start only when everything before them is
 // complete, which empties the record.
+//
+// Writes are ordered the same way.  A kernel that would write a buffer that a recorded call also writes
+// has to know that call is over.  Calls of one context carry sequence numbers, and the context keeps a
+// device word `done` = the largest sequence number whose call is known to be complete (written by a
+// later call's kernel after ITS griddepcontrol.wait returned).  The launcher hands the kernel the number
+// it needs (`need_seq`); the kernel writes at once when done >= need_seq and waits for the preceding
+// grid otherwise.  Buffers written by anything that has no sequence number in that context make the
+// kernel wait (need_seq = INT64_MAX).
 #include <mutex>
 
 #include "common.cuh"
@@ -18,8 +26,13 @@ namespace fedattn {
 namespace {
 
 constexpr int kRecord = 64;
+struct Entry {
+    MemRange r;
+    const void *owner;      // whose sequence numbers `seq` counts in (a context's status area), or null
+    int64_t seq;            // the owner's latest call that writes this buffer
+};
 struct OutputRecord {
-    MemRange r[kRecord];
+    Entry e[kRecord];
     int n = 0;
 };
 OutputRecord g_outputs[64];        // per device
@@ -33,30 +46,40 @@ bool overlaps(const MemRange &a, const MemRange &b)
 
 }  // namespace
 
-bool early_read_allowed(int device, const MemRange *in, int n_in, const MemRange *out, int n_out)
+bool early_read_allowed(int device, const MemRange *in, int n_in, const MemRange *out, int n_out, const void *owner,
+                        int64_t seq, int64_t *need_seq)
 {
     std::lock_guard<std::mutex> lock(g_outputs_mutex);
     OutputRecord &rec = g_outputs[device & 63];
     bool wait_first = false;
     for (int i = 0; i < n_in && !wait_first; ++i)
-        for (int j = 0; j < rec.n && !wait_first; ++j) wait_first = overlaps(in[i], rec.r[j]);
-    // outputs not yet covered by a recorded buffer
-    bool is_new[16];
+        for (int j = 0; j < rec.n && !wait_first; ++j) wait_first = overlaps(in[i], rec.e[j].r);
+    // Which recorded calls wrote into this call's outputs?  Calls of the same owner are named by their
+    // sequence number (the kernel can tell on the device whether they are over); anything else cannot be
+    // named and makes the call wait before its first write.
+    int64_t need = 0;
+    bool same[16];
     int n_new = 0;
     if (n_out > 16) wait_first = true;
     for (int o = 0; o < n_out && o < 16; ++o) {
-        is_new[o] = false;
+        same[o] = false;
         if (!out[o].p || !out[o].bytes) continue;
-        bool known = false;
-        for (int j = 0; j < rec.n && !known; ++j)
-            known = rec.r[j].p == out[o].p && rec.r[j].bytes >= out[o].bytes;
-        is_new[o] = !known;
-        n_new += !known;
+        for (int j = 0; j < rec.n; ++j) {
+            if (!overlaps(out[o], rec.e[j].r)) continue;
+            if (owner && rec.e[j].owner == owner) need = need > rec.e[j].seq ? need : rec.e[j].seq;
+            else need = INT64_MAX;
+            if (rec.e[j].r.p == out[o].p && rec.e[j].r.bytes >= out[o].bytes && rec.e[j].owner == owner) {
+                same[o] = true;
+                rec.e[j].seq = seq;                               // the buffer's latest writer is this call
+            }
+        }
+        n_new += !same[o];
     }
     if (rec.n + n_new > kRecord) wait_first = true;
-    if (wait_first) rec.n = 0;
+    if (wait_first) { rec.n = 0; need = 0; }                      // this call waits first: nothing before it is left
     for (int o = 0; o < n_out && o < 16 && rec.n < kRecord; ++o)
-        if (out[o].p && out[o].bytes && (wait_first || is_new[o])) rec.r[rec.n++] = out[o];
+        if (out[o].p && out[o].bytes && (wait_first || !same[o])) rec.e[rec.n++] = Entry{out[o], owner, seq};
+    if (need_seq) *need_seq = need;
     return !wait_first;
 }
 
