@@ -11,21 +11,21 @@
 //     S_t = Q_t K_j^T          (tcgen05.mma, A/B from shared memory, D in TMEM)
 //     P_t = exp2(S_t*c - m)    (softmax threads, TMEM -> registers -> TMEM, P aliases S)
 //     O_t += P_t V_j           (tcgen05.mma, A = P from TMEM, B = V from shared memory)
-// The tensor pipe alternates between the sub-tiles (PV_0 S_0 | PV_1 S_1 | ...), the softmax threads
-// serve them alternately as well, so while the softmax of one sub-tile runs the tensor pipe works
-// for the other.  O stays in TMEM for the whole tile walk and is rescaled only when a row's running
-// maximum grows by more than 2^8 (the final normalisation uses the same reference, so the result
-// is exact up to rounding).
+// The tensor pipe alternates between the sub-tiles (PV_0 S_0 | PV_1 S_1 | ...); each sub-tile has a
+// softmax warpgroup of its own, so while one warpgroup is in the serial part of its visit the other
+// computes and the tensor pipe works for whichever sub-tile is ready.  O stays in TMEM for the whole
+// tile walk and is rescaled only when a row's running maximum grows by more than 2^8 (the final
+// normalisation uses the same reference, so the result is exact up to rounding).
 //
-// Warp roles: warps 0-7 softmax/epilogue.  Both warpgroups work on the same S tile, split by
-// columns: thread = (query row = TMEM lane, column half); the halves of a row exchange their
-// maxima through shared memory once per tile.  Warp 8 TMA producer (+ TMEM allocation), warp 9
-// MMA issuer (the whole warp walks the loop, one elected lane issues); warps 10-11 only fill that
-// warpgroup, which hands most of its registers to the softmax warpgroups (setmaxnreg works on whole
-// warpgroups).  3/8 of the exponentials
-// of unmasked tiles are evaluated by a polynomial on the FMA pipe, because for this tile shape the
-// ex2 unit is exactly as slow as the tensor pipe.  Every wait is bounded; on expiry the CTA sets
-// the status word, stops waiting and runs to its normal end (TMEM is always released).
+// Warp roles: warps 0-3 softmax/epilogue of sub-tile 0, warps 4-7 of sub-tile 1: thread = query row =
+// TMEM lane, all 128 key columns of the S tile and the whole row of O, walked in 32-column chunks
+// (once for the row maximum, once for the exponentials); nothing is exchanged between threads.  Warp 8
+// TMA producer (+ TMEM allocation), warp 9 MMA issuer (the whole warp walks the loop, one elected lane
+// issues); warp 10 checks the order of the key positions, warp 11 only fills that warpgroup, which
+// hands most of its registers to the softmax warpgroups (setmaxnreg works on whole warpgroups).
+// 2/8 of the exponentials of unmasked tiles are evaluated by a polynomial on the FMA pipe, because for
+// this tile shape the ex2 unit alone is as slow as the tensor pipe.  Every wait is bounded; on expiry
+// the CTA sets the status word, stops waiting and runs to its normal end (TMEM is always released).
 #include <cuda.h>
 
 #include <stdio.h>
@@ -41,12 +41,11 @@ namespace {
 constexpr int kTileM = 128;          // query rows per CTA
 constexpr int kTileN = 128;          // keys per KV tile
 constexpr int kD = 128;              // head dim
-// softmax warpgroups; each owns kCols key columns of every S tile.  (Four warpgroups of 32 columns
-// were measured 20 % slower than two of 64: the exponentials are throughput-bound either way and
-// the exchange costs more.)
+// two softmax warpgroups, one per sub-tile.  (Both on the same S tile, split by columns with the row
+// maxima exchanged through shared memory, was 2-4 % slower on dense sync; four warpgroups of 32 columns
+// 20 %.)  P is handed to the MMA warp in kSplit halves of kCols keys, so that PV starts on the first.
 constexpr int kSplit = 2;
 constexpr int kCols = kTileN / kSplit;
-static_assert(kCols == 64, "the visibility mask of a thread's columns is one 64-bit word");
 constexpr int kSoftmaxThreads = 128 * kSplit;
 constexpr int kThreads = kSoftmaxThreads + 128;  // then a warpgroup holding the TMA producer warp and the MMA issuer warp
 // Registers move from that warpgroup to the softmax warpgroups once the roles split (setmaxnreg):
@@ -60,12 +59,11 @@ constexpr int kProducerWarp = 4 * kSplit, kMmaWarp = 4 * kSplit + 1;
 static_assert(kSplit == 2 || kSplit == 4, "column split");
 constexpr uint32_t kTileBytes = kTileM * kD * 2;      // 32 KB: one Q, K or V tile
 constexpr uint32_t kHalfBytes = kTileBytes / 2;       // one 64-column TMA box
-constexpr uint32_t kSmemBytes = 6 * kTileBytes + 1024 /*alignment slack*/ + 256 /*barriers*/ +
-                                4 * kSplit * kTileM * 4 /*row max / row sum exchange*/;
+constexpr uint32_t kSmemBytes = 6 * kTileBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kColS = 0, kColO = 256;   // S (and P, aliased) of sub-tile t at kColS + 128 t; O at kColO + 128 t
-// P (bf16 pairs) of keys kCols q .. kCols q + kCols - 1 sits at S column kCols q, i.e. inside the S
-// columns that the same softmax warpgroup reads
+// P (bf16 pairs) of keys kCols q .. kCols q + kCols - 1 sits at S column kCols q: every 32-key chunk of P
+// lands in S columns that its thread has already read
 constexpr uint32_t kWaitLimit = 1u << 20;
 constexpr float kRescaleThreshold = 8.0f;
 
@@ -278,9 +276,10 @@ __device__ __forceinline__ float max3(float a, float b, float c)
 // 2^n by adding n to the exponent field.  The magic constant 1.5 * 2^23 makes the low mantissa
 // bits of x + magic hold n.  x is clamped at -125 so that the exponent arithmetic cannot wrap:
 // anything smaller contributes 2^-125 instead of an even smaller value.  Needs x <= 100.
-// bit (c & 7) set: column pair c takes the polynomial instead of ex2.approx.  3 of 8 pairs: measured
-// best of 0, 2, 3, 4, 5 of 8 (the polynomial loads the ALU pipe as much as ex2 loads its own unit).
-constexpr uint32_t kPolyMask = 0x49;
+// bit (c & 7) set: column pair c takes the polynomial instead of ex2.approx.  2 of 8 pairs: 1, 2 and 3 of 8
+// are within 1 % of each other (which is best depends on the board), none costs 2-3 %, 4 and 5 of 8 cost
+// 2 and 5 % (the polynomial loads the ALU pipe as much as ex2 loads its own unit).
+constexpr uint32_t kPolyMask = 0x11;
 __device__ __forceinline__ void exp2_poly_x2(uint64_t x2, float &p0, float &p1)
 {
     float x0, x1;
@@ -477,8 +476,6 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     // what the producer tells the MMA issuer about an item, published before the item's Q load is issued
     // and read after q_full: {KV tiles, sub-tiles}; -1 tiles = no more items.  Two slots, like the phases.
     volatile int *item_info = reinterpret_cast<volatile int *>(bars + 26);
-    float *x_max = reinterpret_cast<float *>(bars + 32);            // [2 buffers][kSplit column parts][128 rows]
-    float *x_sum = x_max + 2 * kSplit * kTileM;                     // [2 sub-tiles][kSplit column parts][128 rows]
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int n_items = kp.n_items;
@@ -494,7 +491,7 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         mbar_init(q_full, 1); mbar_init(q_empty, 1);
         for (int i = 0; i < 2; ++i) {
             mbar_init(k_full + i, 1); mbar_init(k_empty + i, 1); mbar_init(v_full + i, 1); mbar_init(v_empty + i, 1);
-            mbar_init(s_full + i, 1); mbar_init(o_done + i, 1); mbar_init(o_free + i, kSoftmaxThreads / 32);
+            mbar_init(s_full + i, 1); mbar_init(o_done + i, 1); mbar_init(o_free + i, 4);
             for (int q = 0; q < kSplit; ++q) mbar_init(p_full + kSplit * i + q, 4);
         }
         *abort_flag = (*reinterpret_cast<volatile int32_t *>(kp.status) == FEDATTN_ERR_TIMEOUT) ? 1 : 0;
@@ -672,66 +669,57 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     } else {
         asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kSoftmaxRegs));
         // ================= softmax + epilogue =================
-        // All softmax warpgroups work on the same S tile: thread = (query row r = TMEM lane, column part hf).
-        // Warpgroup hf owns keys kCols hf .. kCols hf + kCols - 1 of every S tile and the same head-dim
-        // columns of O.  The two sub-tiles (heads) are served alternately, so while the
-        // softmax of one sub-tile runs the tensor pipe works on the other.  Row maxima are exchanged
-        // through shared memory once per tile, row sums once per item.
-        const int hf = warp >> 2;                               // column part 0 .. kSplit - 1
+        // Warpgroup t serves sub-tile t (query head head0 + t) on its own: thread = query row r = TMEM lane,
+        // all 128 key columns of the S tile, the whole row of O.  The two warpgroups never meet: no row
+        // maximum or row sum has to be exchanged, and while one is in the serial part of its visit (wait,
+        // TMEM load, maximum) the other computes.  A row is walked twice in 32-column chunks, once for the
+        // maximum and once for the exponentials, so that a thread never holds more than two chunks.
+        const int t = warp >> 2;                                // sub-tile of this warpgroup
         const int r = tid & 127;                                // query row = TMEM lane
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+        const uint32_t tS = tmem_base + lane_base + kColS + t * 128;   // fp32 S; bf16 P of keys 64q.. at column 64q
+        const uint32_t tO = tmem_base + lane_base + kColO + t * 128;
         const float sl2 = p.scale * 1.4426950408889634f;
         const uint64_t sl2_2 = pack_f32x2(sl2, sl2);
-        int gsub0 = 0, gsub1 = 0;                               // KV tiles each sub-tile has been through
-        int xb = 0;                                             // exchange buffer parity
-        int k = 0;                                              // round of the static schedule
-        // the threads that share query rows are the warps w, w + 4, ...: one named barrier per row quarter
-        const int bar_id = 1 + (warp & 3);
-        auto wg_sync = [&]() { asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "n"(32 * kSplit) : "memory"); };
+        int gsub = 0;                                           // KV tiles this sub-tile has been through
         const bool o_aligned32 = (reinterpret_cast<uintptr_t>(p.o) & 31) == 0;
+        auto below32 = [](int n) -> uint32_t { return n <= 0 ? 0u : (n >= 32 ? 0xffffffffu : (1u << n) - 1u); };
 
-        // One visit = the softmax of one S tile of one sub-tile.  kPartial: some row of the tile has masked
-        // columns; bit c of `vis` says whether this thread's column c is visible.  Masked columns become
-        // -inf and every exponential goes through ex2.approx, which maps -inf to 0; in unmasked tiles a fixed
-        // subset of the columns takes the polynomial so that the ex2 unit, which is as slow as the tensor
-        // pipe for this tile shape, is not the bottleneck.
-        auto visit = [&](auto partial_tag, int t, int j, int gt, uint64_t vis, float &m_used, float &l) {
+        // One visit = the softmax of one S tile.  kPartial: some row of the tile has masked columns; bit i of
+        // vm[c] says whether column 32 c + i is visible to this thread's row.  Masked columns become -inf and
+        // every exponential goes through ex2.approx, which maps -inf to 0; in unmasked tiles a fixed subset of
+        // the columns takes the polynomial so that the ex2 unit is not the bottleneck.
+        auto visit = [&](auto partial_tag, int j, int gt, const uint32_t (&vm)[4], float &m_used, float &l) {
             constexpr bool kPartial = decltype(partial_tag)::value;
-            const uint32_t tS = tmem_base + lane_base + kColS + t * 128 + kCols * hf;   // fp32 S, this part
-            const uint32_t tP = tS;                                                      // bf16 P, this part
-            const uint32_t tO = tmem_base + lane_base + kColO + t * 128 + kCols * hf;
             mbar_wait(s_full + t, gt & 1, abort_flag, kp.status);
             if (tid == 0) TRACE(j, t ? 5 : 0);
             tc_fence_after();
-            uint32_t s[kCols];
-#pragma unroll
-            for (int c = 0; c < kCols; c += 32) FEDATTN_TMEM_LD32(tS + c, (s + c));
-            tmem_wait_ld();
-            if (kPartial) {
-                const uint32_t vis_lo = (uint32_t)vis, vis_hi = (uint32_t)(vis >> 32);
-#pragma unroll
-                for (int c = 0; c < kCols; ++c)
-                    if (!(((c < 32 ? vis_lo : vis_hi) >> (c & 31)) & 1u)) s[c] = 0xff800000u;      // -inf
-            }
-            // partial row maximum: 8 independent chains, then a tree
+            uint32_t sa[32], sb[32];
+            // ---- pass 1: the row maximum ----
             float mx[8];
 #pragma unroll
-            for (int i = 0; i < 8; ++i) mx[i] = fmaxf(__uint_as_float(s[2 * i]), __uint_as_float(s[2 * i + 1]));
+            for (int i = 0; i < 8; ++i) mx[i] = -INFINITY;
+            FEDATTN_TMEM_LD32(tS, sa);
 #pragma unroll
-            for (int c = 16; c < kCols; c += 16)
+            for (int c = 0; c < 4; ++c) {
+                uint32_t *cur = (c & 1) ? sb : sa, *nxt = (c & 1) ? sa : sb;
+                tmem_wait_ld();
+                if (c < 3) FEDATTN_TMEM_LD32(tS + 32 * (c + 1), nxt);
+                if (kPartial) {
 #pragma unroll
-                for (int i = 0; i < 8; ++i)
-                    mx[i] = max3(mx[i], __uint_as_float(s[c + 2 * i]), __uint_as_float(s[c + 2 * i + 1]));
-            const float pm = fmaxf(max3(mx[0], mx[1], mx[2]), fmaxf(max3(mx[3], mx[4], mx[5]), fmaxf(mx[6], mx[7])));
-            // row maximum over all parts: post this thread's partial maximum, meet the threads that hold the
-            // other parts of the row (one softmax-wide barrier per visit), read theirs
-            x_max[(xb * kSplit + hf) * kTileM + r] = pm;
-            wg_sync();
-            float rm = pm;
+                    for (int i = 0; i < 32; ++i)
+                        if (!((vm[c] >> i) & 1u)) cur[i] = 0xff800000u;          // -inf
+                }
 #pragma unroll
-            for (int q = 1; q < kSplit; ++q) rm = fmaxf(rm, x_max[(xb * kSplit + ((hf + q) & (kSplit - 1))) * kTileM + r]);
-            xb ^= 1;
+                for (int i = 0; i < 8; ++i) {
+                    mx[i] = max3(mx[i], __uint_as_float(cur[2 * i]), __uint_as_float(cur[2 * i + 1]));
+                    mx[i] = max3(mx[i], __uint_as_float(cur[16 + 2 * i]), __uint_as_float(cur[16 + 2 * i + 1]));
+                }
+            }
+            const float rm = fmaxf(max3(mx[0], mx[1], mx[2]), fmaxf(max3(mx[3], mx[4], mx[5]), fmaxf(mx[6], mx[7])));
             const float t_max = rm * sl2;
+            // the second walk starts while the reference is settled
+            FEDATTN_TMEM_LD32(tS, sa);
             if (j == 0) {
                 m_used = (t_max == -INFINITY) ? 0.f : t_max;
             } else {
@@ -742,8 +730,9 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                     const float alpha = need ? ex2(m_used - t_max) : 1.f;
                     mbar_wait(o_done + t, (gt - 1) & 1, abort_flag, kp.status);   // O holds tiles 0..j-1
                     tc_fence_after();
+                    tmem_wait_ld();                                               // sa is in flight: one wait serves both
 #pragma unroll 1
-                    for (int oc = 0; oc < kCols / 32; ++oc) {
+                    for (int oc = 0; oc < 4; ++oc) {
                         uint32_t o[32];
                         FEDATTN_TMEM_LD32(tO + oc * 32, o);
                         tmem_wait_ld();
@@ -754,55 +743,64 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                     if (need) { l *= alpha; m_used = t_max; }
                 }
             }
+            // ---- pass 2: exponentials, row sum, P ----
             const uint64_t negm2 = pack_f32x2(-m_used, -m_used);
             uint64_t sum2[4] = {0, 0, 0, 0};
 #pragma unroll
-            for (int cc = 0; cc < kCols / 32; ++cc) {
+            for (int c = 0; c < 4; ++c) {
+                uint32_t *cur = (c & 1) ? sb : sa, *nxt = (c & 1) ? sa : sb;
+                tmem_wait_ld();
+                if (c < 3) FEDATTN_TMEM_LD32(tS + 32 * (c + 1), nxt);
+                if (kPartial) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i)
+                        if (!((vm[c] >> i) & 1u)) cur[i] = 0xff800000u;
+                }
                 uint32_t pk[16];
 #pragma unroll
-                for (int c = 0; c < 16; ++c) {
-                    const uint64_t x2 = fma_f32x2(pack_f32x2(__uint_as_float(s[cc * 32 + 2 * c]),
-                                                             __uint_as_float(s[cc * 32 + 2 * c + 1])), sl2_2, negm2);
+                for (int i = 0; i < 16; ++i) {
+                    const uint64_t x2 = fma_f32x2(pack_f32x2(__uint_as_float(cur[2 * i]), __uint_as_float(cur[2 * i + 1])), sl2_2, negm2);
                     float p0, p1;
-                    if (!kPartial && ((kPolyMask >> (c & 7)) & 1)) {
+                    if (!kPartial && ((kPolyMask >> (i & 7)) & 1)) {
                         exp2_poly_x2(x2, p0, p1);
                     } else {
                         float x0, x1;
                         unpack_f32x2(x2, x0, x1);
                         p0 = ex2(x0); p1 = ex2(x1);
                     }
-                    sum2[c & 3] = add_f32x2(sum2[c & 3], pack_f32x2(p0, p1));
-                    pk[c] = pack_bf16(p0, p1);
+                    sum2[i & 3] = add_f32x2(sum2[i & 3], pack_f32x2(p0, p1));
+                    pk[i] = pack_bf16(p0, p1);
                 }
-                FEDATTN_TMEM_ST16(tP + cc * 16, pk);
+                // keys 32 c .. 32 c + 31 as bf16 pairs: columns 64 (c / 2) + 16 (c % 2) .., all inside S columns
+                // that this thread has already read
+                FEDATTN_TMEM_ST16(tS + 64 * (c >> 1) + 16 * (c & 1), pk);
+                if (c & 1) {                                    // a 64-key half of P is complete: PV may start on it
+                    tmem_wait_st();
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(p_full + kSplit * t + (c >> 1));      // one arrival per warp
+                }
             }
             float r0, r1;
             unpack_f32x2(add_f32x2(add_f32x2(sum2[0], sum2[1]), add_f32x2(sum2[2], sum2[3])), r0, r1);
             l += r0 + r1;
-            tmem_wait_st();
-            tc_fence_before();
             if (tid == 0) TRACE(j, t ? 6 : 1);
-            __syncwarp();
-            if (lane == 0) mbar_arrive(p_full + kSplit * t + hf);      // one arrival per warp
         };
 
-        for (k = 0; k < n_rounds; ++k) {
+        for (int k = 0; k < n_rounds; ++k) {
             const int item = item_of(k);
             if (item >= n_items) continue;
             const Item it = decode_item<kSpecial>(kp, item, lane);
+            if (t == 1 && !it.valid1) continue;                 // the pair's second head does not exist
             const int n_tiles = it.n_tiles;
-            const int n_sub = it.valid1 ? 2 : 1;
             const bool valid = r < it.n_valid;
-            __nv_bfloat16 *orow0 = reinterpret_cast<__nv_bfloat16 *>(p.o) +
-                                   ((int64_t)(it.q_row0 + r) * p.hq + it.head0) * kD + kCols * hf;
-            float *lse0 = p.lse ? p.lse + (int64_t)(it.q_row0 + r) * p.hq + it.head0 : nullptr;
+            __nv_bfloat16 *orow = reinterpret_cast<__nv_bfloat16 *>(p.o) + ((int64_t)(it.q_row0 + r) * p.hq + it.head0 + t) * kD;
+            float *lse_p = p.lse ? p.lse + (int64_t)(it.q_row0 + r) * p.hq + it.head0 + t : nullptr;
             if (n_tiles == 0) {                                 // nothing visible to any row of the tile
                 if (valid) {
-                    for (int t = 0; t < n_sub; ++t) {
 #pragma unroll
-                        for (int c = 0; c < kCols; c += 8) *reinterpret_cast<uint4 *>(orow0 + t * kD + c) = make_uint4(0, 0, 0, 0);
-                        if (lse0 && hf == 0) lse0[t] = -INFINITY;
-                    }
+                    for (int c = 0; c < kD; c += 8) *reinterpret_cast<uint4 *>(orow + c) = make_uint4(0, 0, 0, 0);
+                    if (lse_p) *lse_p = -INFINITY;
                 }
                 continue;
             }
@@ -829,7 +827,7 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                     const int wv = cw + lane < T ? __ldg(it.kvp + cw + lane) : INT32_MAX;
                     int cnt = 0;
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) cnt += __shfl_sync(0xffffffffu, wv, j) <= p0 + lane;
+                    for (int jj = 0; jj < 32; ++jj) cnt += __shfl_sync(0xffffffffu, wv, jj) <= p0 + lane;
                     c_row = cw + cnt;
                     if (__shfl_sync(0xffffffffu, wv, 31) <= p0 + 31) c_row = count_le(it.kvp, T, p0 + lane);
                 } else {
@@ -839,94 +837,86 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                 // row are unmasked for the whole warp (the choice of code path only has to be warp-uniform)
                 n_full = __shfl_sync(0xffffffffu, c_row, 0) / kTileN;
             }
-            const int c_r = c_row - kCols * hf;                 // visible keys, counted from this thread's first column
             const int T = (int)p.total_kv;
-            // state of the sub-tile being visited (a) and of the other one (b); swapped after every visit
-            float m_a = 0.f, l_a = 0.f, m_b = 0.f, l_b = 0.f;
-            const int n_visits = n_tiles * n_sub;
-            for (int v = 0; v < n_visits; ++v) {
-                const int t = n_sub == 2 ? (v & 1) : 0;
-                const int j = n_sub == 2 ? (v >> 1) : v;
-                const int gt = (t ? gsub1 : gsub0) + j;
-                // columns of this thread that lie below n (n may be <= 0 or >= kCols)
-                auto below = [](int n) -> uint64_t { return n <= 0 ? 0ull : (n >= 64 ? ~0ull : (1ull << n) - 1ull); };
-                if (two_range) {
+            float m_run = 0.f, l_run = 0.f;
+            for (int j = 0; j < n_tiles; ++j) {
+                const int gt = gsub + j;
+                // which columns of this tile the thread's row sees: everything (warp-uniform), or a mask per chunk
+                bool full;
+                uint32_t vm[4] = {0, 0, 0, 0};
+                if (two_range) {                                // keys [0, a) and [b, T)
                     const int k0 = tile_of(it, j) * kTileN;     // first key of the tile
-                    if (k0 + kTileN <= it.a || (k0 >= it.b && k0 + kTileN <= T)) {
-                        visit(std::false_type{}, t, j, gt, 0, m_a, l_a);
-                    } else {                                    // keys [0, a) and [b, T)
-                        const int cb = k0 + kCols * hf;         // key of this thread's column 0
-                        visit(std::true_type{}, t, j, gt, below(it.a - cb) | (below(T - cb) & ~below(it.b - cb)), m_a, l_a);
+                    full = k0 + kTileN <= it.a || (k0 >= it.b && k0 + kTileN <= T);
+                    if (!full) {
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) {
+                            const int cb = k0 + 32 * c;
+                            vm[c] = below32(it.a - cb) | (below32(T - cb) & ~below32(it.b - cb));
+                        }
                     }
-                } else if (j < n_full) {
-                    visit(std::false_type{}, t, j, gt, 0, m_a, l_a);
-                } else if (general) {
-                    // column c is key cb + c: visible iff it exists and its position is not above the row's.
-                    // The address is the same in every lane: broadcast loads.
-                    const int cb = j * kTileN + kCols * hf;
-                    uint64_t vis = 0;
-#pragma unroll 8
-                    for (int c = 0; c < kCols; ++c) {
-                        const int key = cb + c;
-                        const int kpos = it.kvp ? __ldg(it.kvp + min(key, T - 1)) : key;
-                        if (key < T && kpos <= p_row) vis |= 1ull << c;
-                    }
-                    visit(std::true_type{}, t, j, gt, vis, m_a, l_a);
                 } else {
-                    visit(std::true_type{}, t, j, gt, below(c_r - j * kTileN), m_a, l_a);
+                    full = j < n_full;
+                    if (!full && general) {
+                        // column i of chunk c is key cb + i: visible iff it exists and its position is not above
+                        // the row's.  The address is the same in every lane: broadcast loads.
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) {
+                            const int cb = j * kTileN + 32 * c;
+                            uint32_t m = 0;
+#pragma unroll 4
+                            for (int i = 0; i < 32; ++i) {
+                                const int key = cb + i;
+                                const int kpos = it.kvp ? __ldg(it.kvp + min(key, T - 1)) : key;
+                                if (key < T && kpos <= p_row) m |= 1u << i;
+                            }
+                            vm[c] = m;
+                        }
+                    } else if (!full) {
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) vm[c] = below32(c_row - j * kTileN - 32 * c);
+                    }
                 }
-                if (n_sub == 2) {
-                    float x = m_a; m_a = m_b; m_b = x;
-                    x = l_a; l_a = l_b; l_b = x;
-                }
+                if (full) visit(std::false_type{}, j, gt, vm, m_run, l_run);
+                else visit(std::true_type{}, j, gt, vm, m_run, l_run);
             }
-            // after an even number of swaps (a) is sub-tile 0 again
 
-            // ---- epilogue: drain this thread's half of O from TMEM (frees it for the next item), exchange
-            //      the row sums, then O / l -> bf16 -> global
-#pragma unroll 1
-            for (int t = 0; t < n_sub; ++t) {
-                const float m_t = t ? m_b : m_a, l_t = t ? l_b : l_a;
-                const uint32_t tO = tmem_base + lane_base + kColO + t * 128 + kCols * hf;
-                mbar_wait(o_done + t, ((t ? gsub1 : gsub0) + n_tiles - 1) & 1, abort_flag, kp.status);
-                tc_fence_after();
-                uint32_t o[kCols];
+            // ---- epilogue: drain this row of O from TMEM (frees it for the next item), O / l -> bf16 -> global
+            mbar_wait(o_done + t, (gsub + n_tiles - 1) & 1, abort_flag, kp.status);
+            tc_fence_after();
+            const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
+            uint32_t oa[32], ob[32];
+            FEDATTN_TMEM_LD32(tO, oa);
 #pragma unroll
-                for (int c = 0; c < kCols; c += 32) FEDATTN_TMEM_LD32(tO + c, (o + c));
+            for (int c = 0; c < 4; ++c) {
+                uint32_t *cur = (c & 1) ? ob : oa, *nxt = (c & 1) ? oa : ob;
                 tmem_wait_ld();
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(o_free + t);             // one arrival per warp
-                x_sum[(t * kSplit + hf) * kTileM + r] = l_t;
-                wg_sync();
-                float lt = 0.f;                                 // same summation order in every part of the row
-#pragma unroll
-                for (int q = 0; q < kSplit; ++q) lt += x_sum[(t * kSplit + q) * kTileM + r];
+                if (c < 3) {
+                    FEDATTN_TMEM_LD32(tO + 32 * (c + 1), nxt);
+                } else {
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(o_free + t);     // one arrival per warp: O_t may be overwritten
+                }
                 if (valid) {
-                    const float inv = lt > 0.f ? 1.f / lt : 0.f;
-                    __nv_bfloat16 *orow = orow0 + t * kD;
-                    // a thread's 32 bytes are one full sector: 256-bit stores halve the store transactions
 #pragma unroll
-                    for (int c = 0; c < kCols; c += 16) {
+                    for (int h2 = 0; h2 < 2; ++h2) {
                         uint32_t w[8];
 #pragma unroll
                         for (int i = 0; i < 8; ++i)
-                            w[i] = pack_bf16(__uint_as_float(o[c + 2 * i]) * inv, __uint_as_float(o[c + 2 * i + 1]) * inv);
+                            w[i] = pack_bf16(__uint_as_float(cur[16 * h2 + 2 * i]) * inv, __uint_as_float(cur[16 * h2 + 2 * i + 1]) * inv);
+                        __nv_bfloat16 *dst = orow + 32 * c + 16 * h2;
                         if (o_aligned32) {
-                            asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(orow + c), "r"(w[0]), "r"(w[1]),
+                            asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(dst), "r"(w[0]), "r"(w[1]),
                                          "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7]) : "memory");
                         } else {
-                            *reinterpret_cast<uint4 *>(orow + c) = make_uint4(w[0], w[1], w[2], w[3]);
-                            *reinterpret_cast<uint4 *>(orow + c + 8) = make_uint4(w[4], w[5], w[6], w[7]);
+                            *reinterpret_cast<uint4 *>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
+                            *reinterpret_cast<uint4 *>(dst + 8) = make_uint4(w[4], w[5], w[6], w[7]);
                         }
                     }
-                    if (lse0 && hf == 0) lse0[t] = lt > 0.f ? (m_t + log2f(lt)) * 0.6931471805599453f : -INFINITY;
                 }
             }
-            gsub0 += n_tiles;
-            if (n_sub == 2) gsub1 += n_tiles;
-            // x_sum of this item is read before the next item's epilogue writes it again: the next item's
-            // first wg_sync (row-max exchange or row-sum exchange) lies in between
+            if (valid && lse_p) *lse_p = l_run > 0.f ? (m_run + log2f(l_run)) * 0.6931471805599453f : -INFINITY;
+            gsub += n_tiles;
         }
     }
 
