@@ -160,7 +160,7 @@ topk_fused_kernel(const PartsParams pp, int hkv, int vpr /* 16-byte vectors per 
     auto close_call = [&]() {
         if (closer) {
             asm volatile("griddepcontrol.wait;" ::: "memory");
-            if (tid == 0) atomicMax(reinterpret_cast<unsigned long long *>(done_seq), (unsigned long long)(my_seq - 1));
+            if (tid == 0 && my_seq > 0) atomicMax(reinterpret_cast<unsigned long long *>(done_seq), (unsigned long long)(my_seq - 1));
         }
     };
     auto may_write = [&]() {                                  // CTA-uniform
@@ -464,7 +464,7 @@ cudaError_t launch_topk_fused(const PartsParams &pp, int hkv, int d, int dtype, 
     const int elt = dtype == FEDATTN_BF16 ? 2 : 4;
     int early;
     long long *done_seq = reinterpret_cast<long long *>(ctx->workspace + kDoneSeqOffset);
-    const long long my_seq = ++ctx->agg_seq;
+    long long my_seq = 0;
     int64_t need_seq = 0;
     {
         const size_t row_bytes = (size_t)hkv * d * elt;
@@ -477,7 +477,10 @@ cudaError_t launch_topk_fused(const PartsParams &pp, int hkv, int d, int dtype, 
         }
         const MemRange out[5] = {{k_agg, T * row_bytes}, {v_agg, T * row_bytes}, {kv_pos, kv_pos ? T * hkv * 4 : 0},
                                  {cu_kv, cu_kv ? (size_t)(pp.n + 1) * 4 : 0}, {sel_idx_out, sel_idx_out ? T * hkv * 4 : 0}};
-        early = early_read_allowed(device, in, 2 * pp.n, out, 5, done_seq, my_seq, &need_seq) ? 1 : 0;
+        const EarlyStart es = early_start(device, s, in, 2 * pp.n, out, 5, true, done_seq, &ctx->agg_seq, &ctx->agg_key);
+        early = es.early ? 1 : 0;
+        my_seq = es.seq;
+        need_seq = es.need_seq;
     }
     const int vpr = d * elt / 16;
     int max_len = 0;

@@ -104,6 +104,7 @@ fedattn_status fedattn_create(fedattn_ctx **out, int device, void *workspace, si
     c.launches = 0;
     c.tc_launches = 0;
     c.agg_seq = 0;
+    c.agg_key = ~0ull;
     c.encode_tiled = nullptr;
     if (prop.major == 10) {
         void *fn = nullptr;
@@ -120,7 +121,11 @@ fedattn_status fedattn_create(fedattn_ctx **out, int device, void *workspace, si
     return FEDATTN_OK;
 }
 
-void fedattn_destroy(fedattn_ctx *ctx) { delete ctx; }
+void fedattn_destroy(fedattn_ctx *ctx)
+{
+    if (ctx) early_start_forget(ctx->c.device, ctx->c.workspace + kDoneSeqOffset);
+    delete ctx;
+}
 
 int64_t fedattn_launch_count(const fedattn_ctx *ctx) { return ctx ? ctx->c.launches : 0; }
 

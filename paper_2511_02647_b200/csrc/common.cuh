@@ -28,6 +28,7 @@ struct Context {
     int64_t launches;
     int64_t tc_launches;   // launches of the tcgen05 attention kernel among them
     int64_t agg_seq;       // sequence number of the latest sparse aggregation call
+    uint64_t agg_key;      // key of the stream that call ran on (early-start bookkeeping)
     void *encode_tiled;    // cuTensorMapEncodeTiled entry point (driver), or nullptr
 };
 
@@ -36,14 +37,23 @@ struct MemRange {
     const void *p;
     size_t bytes;
 };
-// Records `out` as buffers that grids of this call may still be writing when later grids start, and
-// returns whether this call may read `in` before the preceding grid of the stream is complete (false:
-// it must wait first).  n_out <= 16.
-// owner / seq: the context's sequence counter for this call (null / 0: none).  need_seq (nullable) receives the
-// largest sequence number of the owner's recorded calls that write one of `out` (0: none; INT64_MAX: a writer
-// that cannot be named, wait before writing).
-bool early_read_allowed(int device, const MemRange *in, int n_in, const MemRange *out, int n_out,
-                        const void *owner = nullptr, int64_t seq = 0, int64_t *need_seq = nullptr);
+struct EarlyStart {
+    bool early;          // the inputs may be read before the preceding grid of the stream is complete
+    int64_t seq;         // this call's sequence number in its context (0: none, publish nothing)
+    int64_t need_seq;    // the context's latest recorded call that reads or writes one of `out` (0: none;
+                         // INT64_MAX: one that cannot be named, wait before the first write)
+};
+// Records `in` (read) and `out` (written) as buffers that grids of this call may still be using when
+// later grids of `stream` start, and decides how the call may start.  writes_before_wait: the call's
+// kernel writes `out` before its griddepcontrol.wait when need_seq allows it (otherwise overlaps of
+// `out` with recorded buffers do not matter).  owner / seq_counter / owner_key: the context's done
+// word, its sequence counter and the key of the stream its numbered calls last ran on (all null for
+// calls without sequence numbers).
+EarlyStart early_start(int device, cudaStream_t stream, const MemRange *in, int n_in, const MemRange *out, int n_out,
+                       bool writes_before_wait = false, const void *owner = nullptr, int64_t *seq_counter = nullptr,
+                       uint64_t *owner_key = nullptr);
+// The owner's sequence numbers are about to lose their meaning (its context is being destroyed).
+void early_start_forget(int device, const void *owner);
 
 // ---- generic SIMT attention (fp32 or bf16 storage, any head_dim <= 128) --------------------
 enum GenericMode { kLocal = 0, kSync = 1, kDecodeLocal = 2, kDecodeSync = 3 };

@@ -412,7 +412,7 @@ static cudaError_t launch_decode_split(const DecodeParams &p_in, int device, int
         const MemRange in[4] = {{p.q, qo_bytes}, {p.k, cache_bytes}, {p.v, cache_bytes},
                                 {p.kv_len, (p.sync ? 1 : p.n_part) * sizeof(int32_t)}};
         const MemRange out[2] = {{p.o, qo_bytes}, {p.lse, p.lse ? (size_t)p.n_part * p.hq * sizeof(float) : 0}};
-        p.early = early_read_allowed(device, in, 4, out, 2) ? 1 : 0;
+        p.early = early_start(device, s, in, 4, out, 2).early ? 1 : 0;
     }
     const int g = p.hq / p.hkv;
     p.g_shift = -1;

@@ -1,0 +1,141 @@
+"""Stream order of calls that start early (programmatic dependent launch): chains of aggregation and
+decode calls over shared buffers, issued back to back without a host synchronisation, must give what
+the same calls give one at a time.  Expected values come from the fp64 CPU oracle."""
+import numpy as np
+import pytest
+import torch
+
+import fedattn_inputs as fi
+from helpers import LSE_TOL, TOL, check_close, dev, fa, host, make_shape
+
+pytestmark = pytest.mark.gpu
+
+N, L, KSEL, HQ, HKV, D = 8, 1024, 512, 8, 2, 128
+
+
+def _case(seed):
+    w = fi.Workload("order", seed, (L,) * N, HQ, HKV, D, "bf16")
+    _, k, v = w.qkv()
+    lens = [L] * N
+    kp, vp = np.split(k, np.cumsum(lens)[:-1]), np.split(v, np.cumsum(lens)[:-1])
+    return w.decode_q(0), kp, vp
+
+
+class _Chain:
+    """Two input sets A and B aggregated (token-level top-k) into ONE set of output buffers, each
+    aggregation followed by a sync decode that reads those buffers."""
+
+    def __init__(self, oracle):
+        m = fa()
+        self.m = m
+        self.shape = make_shape(N, HQ, HKV, D, "bf16")
+        self.ctx = m.Context(self.shape, N * L, N * L)
+        T = N * KSEL
+        self.T = T
+        bf = torch.bfloat16
+        self.k_agg = torch.zeros((T, HKV, D), dtype=bf, device="cuda")
+        self.v_agg = torch.zeros_like(self.k_agg)
+        self.kv_pos = torch.zeros((T,), dtype=torch.int32, device="cuda")
+        self.cu_kv = torch.zeros((N + 1,), dtype=torch.int32, device="cuda")
+        self.sel = torch.zeros((T,), dtype=torch.int32, device="cuda")
+        self.lens = torch.tensor([T], dtype=torch.int32, device="cuda")
+        self.sets, self.want = [], []
+        for seed in (71, 72):
+            q, kp, vp = _case(seed)
+            ka, va, _, _, _ = oracle.aggregate_topk_token(kp, vp, [KSEL] * N)
+            self.want.append(oracle.decode(q, ka, va, [T], True))
+            self.sets.append((dev(q, "bf16"), [dev(x, "bf16") for x in kp], [dev(x, "bf16") for x in vp]))
+
+    def aggregate(self, i, stream=None):
+        _, kd, vd = self.sets[i]
+        self.m.fedattn_aggregate_kv(self.ctx, self.shape, self.m.AGG_TOPK_TOKEN, kd, vd, [L] * N, [KSEL] * N, None,
+                                    self.k_agg, self.v_agg, self.kv_pos, self.cu_kv, self.sel, stream=stream)
+
+    def decode(self, i, o, lse, stream=None):
+        self.m.fedattn_decode(self.ctx, self.shape, self.m.DECODE_SYNC, self.sets[i][0], self.k_agg, self.v_agg, 0,
+                              self.lens, self.T, o, lse, stream=stream)
+
+    def check(self, i, o, lse, what):
+        check_close(host(o), self.want[i][0], TOL["bf16"], what + " o")
+        check_close(host(lse), self.want[i][1], LSE_TOL["bf16"], what + " lse")
+
+
+def test_aggregation_into_buffers_a_running_decode_still_reads(oracle):
+    """aggregate(A) -> decode -> aggregate(B) -> decode -> ... over one set of output buffers: the second
+    aggregation must not overwrite rows the first decode has yet to read, the decode must not read rows
+    the aggregation has yet to write."""
+    c = _Chain(oracle)
+    reps = 24
+    o = torch.full((reps, 2, N, HQ, D), float("nan"), dtype=torch.bfloat16, device="cuda")
+    lse = torch.full((reps, 2, N, HQ), float("nan"), device="cuda")
+    for r in range(reps):
+        for i in (0, 1):
+            c.aggregate(i)
+            c.decode(i, o[r, i], lse[r, i])
+    torch.cuda.synchronize()
+    assert c.ctx.poll() == 0
+    for r in range(reps):
+        for i in (0, 1):
+            c.check(i, o[r, i], lse[r, i], "rep %d set %d" % (r, i))
+
+
+def test_repeated_aggregation_into_the_same_buffers_then_one_reader(oracle):
+    """aggregate(A), aggregate(B), aggregate(A), ... back to back into the same buffers (each may write
+    as soon as the one before it is over), then one decode: it sees the last one's rows."""
+    c = _Chain(oracle)
+    o = torch.full((4, N, HQ, D), float("nan"), dtype=torch.bfloat16, device="cuda")
+    lse = torch.full((4, N, HQ), float("nan"), device="cuda")
+    for t, n_calls in enumerate((1, 2, 7, 16)):
+        for j in range(n_calls):
+            c.aggregate(j & 1)
+        c.decode((n_calls - 1) & 1, o[t], lse[t])
+    torch.cuda.synchronize()
+    assert c.ctx.poll() == 0
+    for t, n_calls in enumerate((1, 2, 7, 16)):
+        c.check((n_calls - 1) & 1, o[t], lse[t], "%d aggregations" % n_calls)
+
+
+def test_chain_on_two_streams_with_events_and_in_a_replayed_graph(oracle):
+    """The same chain with the context moving between two streams (ordered by events), and captured once
+    into a CUDA graph that is replayed: every replay orders its calls like the first."""
+    c = _Chain(oracle)
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    o = torch.full((6, 2, N, HQ, D), float("nan"), dtype=torch.bfloat16, device="cuda")
+    lse = torch.full((6, 2, N, HQ), float("nan"), device="cuda")
+    torch.cuda.synchronize()
+    prev = None
+    for r in range(6):
+        for i in (0, 1):
+            s = (s1, s2)[(r + i) & 1]
+            if prev is not None:
+                s.wait_event(prev)
+            c.aggregate(i, stream=s.cuda_stream)
+            c.decode(i, o[r, i], lse[r, i], stream=s.cuda_stream)
+            prev = torch.cuda.Event()
+            prev.record(s)
+    torch.cuda.synchronize()
+    assert c.ctx.poll() == 0
+    for r in range(6):
+        for i in (0, 1):
+            c.check(i, o[r, i], lse[r, i], "two streams rep %d set %d" % (r, i))
+
+    og = torch.full((2, N, HQ, D), float("nan"), dtype=torch.bfloat16, device="cuda")
+    lg = torch.full((2, N, HQ), float("nan"), device="cuda")
+    g = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        g.capture_begin()
+        for i in (0, 1, 0, 1):
+            c.aggregate(i, stream=side.cuda_stream)
+            c.decode(i, og[i], lg[i], stream=side.cuda_stream)
+        g.capture_end()
+    torch.cuda.current_stream().wait_stream(side)
+    for _ in range(5):
+        og.fill_(float("nan"))
+        g.replay()
+        c.aggregate(0)                       # an eager call between replays, into the same buffers
+    torch.cuda.synchronize()
+    assert c.ctx.poll() == 0
+    for i in (0, 1):
+        c.check(i, og[i], lg[i], "graph replay set %d" % i)
