@@ -32,6 +32,15 @@
  *     lse is always float.  Softmax and accumulation are fp32.
  *   - One context serves one stream at a time: calls that share a context and may overlap on
  *     the GPU race on its workspace.
+ *   - Results are those of stream order: every call behaves as if it ran after all earlier work
+ *     of its stream and before all later work.  fedattn_decode and the sparse modes of
+ *     fedattn_aggregate_kv are launched with programmatic stream serialization and may touch
+ *     their buffers before the preceding kernel of the stream has ended; the library tracks the
+ *     buffers of such calls and holds a call back whenever that could be observed.  What the
+ *     caller has to keep: a kernel of the caller's own that is launched with the programmatic
+ *     attribute into the same stream executes griddepcontrol.wait before it ends (kernels
+ *     launched the ordinary way need nothing), and buffers shared with work on OTHER streams are
+ *     ordered by events or stream synchronisation, as always.
  */
 #ifndef FEDATTN_H_
 #define FEDATTN_H_
