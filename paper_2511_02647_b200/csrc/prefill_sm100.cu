@@ -18,8 +18,8 @@
 // normalisation uses the same reference, so the result is exact up to rounding).
 //
 // Warp roles: warps 0-3 softmax/epilogue of sub-tile 0, warps 4-7 of sub-tile 1: thread = query row =
-// TMEM lane, all 128 key columns of the S tile and the whole row of O, walked in 32-column chunks
-// (once for the row maximum, once for the exponentials); nothing is exchanged between threads.  Warp 8
+// TMEM lane, all 128 key columns of the S tile (read from TMEM once, held in registers for the row
+// maximum and then the exponentials) and the whole row of O; nothing is exchanged between threads.  Warp 8
 // TMA producer (+ TMEM allocation), warp 9 MMA issuer (the whole warp walks the loop, one elected lane
 // issues); warp 10 checks the order of the key positions, warp 11 only fills that warpgroup, which
 // hands most of its registers to the softmax warpgroups (setmaxnreg works on whole warpgroups).
@@ -279,7 +279,10 @@ __device__ __forceinline__ float max3(float a, float b, float c)
 // bit (c & 7) set: column pair c takes the polynomial instead of ex2.approx.  2 of 8 pairs: 1, 2 and 3 of 8
 // are within 1 % of each other (which is best depends on the board), none costs 2-3 %, 4 and 5 of 8 cost
 // 2 and 5 % (the polynomial loads the ALU pipe as much as ex2 loads its own unit).
-constexpr uint32_t kPolyMask = 0x11;
+#ifndef FEDATTN_POLY_MASK
+#define FEDATTN_POLY_MASK 0x11
+#endif
+constexpr uint32_t kPolyMask = FEDATTN_POLY_MASK;
 __device__ __forceinline__ void exp2_poly_x2(uint64_t x2, float &p0, float &p1)
 {
     float x0, x1;
@@ -672,8 +675,8 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         // Warpgroup t serves sub-tile t (query head head0 + t) on its own: thread = query row r = TMEM lane,
         // all 128 key columns of the S tile, the whole row of O.  The two warpgroups never meet: no row
         // maximum or row sum has to be exchanged, and while one is in the serial part of its visit (wait,
-        // TMEM load, maximum) the other computes.  A row is walked twice in 32-column chunks, once for the
-        // maximum and once for the exponentials, so that a thread never holds more than two chunks.
+        // TMEM load, maximum) the other computes.  A thread reads its row of S from TMEM once and keeps all
+        // 128 values in registers for both walks (maximum, then exponentials).
         const int t = warp >> 2;                                // sub-tile of this warpgroup
         const int r = tid & 127;                                // query row = TMEM lane
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
@@ -694,17 +697,20 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             mbar_wait(s_full + t, gt & 1, abort_flag, kp.status);
             if (tid == 0) TRACE(j, t ? 5 : 0);
             tc_fence_after();
-            uint32_t sa[32], sb[32];
-            // ---- pass 1: the row maximum ----
+            // the whole row of S in registers: read from TMEM once, used for the maximum and the exponentials
+            uint32_t s0[32], s1[32], s2[32], s3[32];
             float mx[8];
 #pragma unroll
             for (int i = 0; i < 8; ++i) mx[i] = -INFINITY;
-            FEDATTN_TMEM_LD32(tS, sa);
+            FEDATTN_TMEM_LD32(tS, s0);
+            FEDATTN_TMEM_LD32(tS + 32, s1);
+            tmem_wait_ld();
+            FEDATTN_TMEM_LD32(tS + 64, s2);
+            FEDATTN_TMEM_LD32(tS + 96, s3);
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
-                uint32_t *cur = (c & 1) ? sb : sa, *nxt = (c & 1) ? sa : sb;
-                tmem_wait_ld();
-                if (c < 3) FEDATTN_TMEM_LD32(tS + 32 * (c + 1), nxt);
+                uint32_t *cur = c == 0 ? s0 : (c == 1 ? s1 : (c == 2 ? s2 : s3));
+                if (c == 2) tmem_wait_ld();
                 if (kPartial) {
 #pragma unroll
                     for (int i = 0; i < 32; ++i)
@@ -718,8 +724,6 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             }
             const float rm = fmaxf(max3(mx[0], mx[1], mx[2]), fmaxf(max3(mx[3], mx[4], mx[5]), fmaxf(mx[6], mx[7])));
             const float t_max = rm * sl2;
-            // the second walk starts while the reference is settled
-            FEDATTN_TMEM_LD32(tS, sa);
             if (j == 0) {
                 m_used = (t_max == -INFINITY) ? 0.f : t_max;
             } else {
@@ -730,7 +734,6 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                     const float alpha = need ? ex2(m_used - t_max) : 1.f;
                     mbar_wait(o_done + t, (gt - 1) & 1, abort_flag, kp.status);   // O holds tiles 0..j-1
                     tc_fence_after();
-                    tmem_wait_ld();                                               // sa is in flight: one wait serves both
 #pragma unroll 1
                     for (int oc = 0; oc < 4; ++oc) {
                         uint32_t o[32];
@@ -748,14 +751,7 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             uint64_t sum2[4] = {0, 0, 0, 0};
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
-                uint32_t *cur = (c & 1) ? sb : sa, *nxt = (c & 1) ? sa : sb;
-                tmem_wait_ld();
-                if (c < 3) FEDATTN_TMEM_LD32(tS + 32 * (c + 1), nxt);
-                if (kPartial) {
-#pragma unroll
-                    for (int i = 0; i < 32; ++i)
-                        if (!((vm[c] >> i) & 1u)) cur[i] = 0xff800000u;
-                }
+                uint32_t *cur = c == 0 ? s0 : (c == 1 ? s1 : (c == 2 ? s2 : s3));
                 uint32_t pk[16];
 #pragma unroll
                 for (int i = 0; i < 16; ++i) {
