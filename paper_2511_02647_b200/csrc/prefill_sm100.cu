@@ -59,7 +59,7 @@ constexpr int kProducerWarp = 4 * kSplit, kMmaWarp = 4 * kSplit + 1;
 static_assert(kSplit == 2 || kSplit == 4, "column split");
 constexpr uint32_t kTileBytes = kTileM * kD * 2;      // 32 KB: one Q, K or V tile
 constexpr uint32_t kHalfBytes = kTileBytes / 2;       // one 64-column TMA box
-constexpr uint32_t kSmemBytes = 6 * kTileBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr uint32_t kSmemBytes = 6 * kTileBytes + 1024 /*alignment slack*/ + 256 /*barriers*/ + 256 /*published items*/;
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kColS = 0, kColO = 256;   // S (and P, aliased) of sub-tile t at kColS + 128 t; O at kColO + 128 t
 // P (bf16 pairs) of keys kCols q .. kCols q + kCols - 1 sits at S column kCols q: every 32-key chunk of P
@@ -159,6 +159,12 @@ __device__ __forceinline__ void tma_load_3d(void *dst, const CUtensorMap *map, u
                  " [%0], [%1, {%3, %4, %5}], [%2];"
                  ::"r"(smem_u32(dst)), "l"((uint64_t)map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2)
                  : "memory");
+}
+
+__device__ __forceinline__ void tma_prefetch_3d(const CUtensorMap *map, int c0, int c1, int c2)
+{
+    asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];"
+                 ::"l"((uint64_t)map), "r"(c0), "r"(c1), "r"(c2) : "memory");
 }
 
 // true in exactly one lane of a converged warp
@@ -479,6 +485,10 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     // what the producer tells the MMA issuer about an item, published before the item's Q load is issued
     // and read after q_full: {KV tiles, sub-tiles}; -1 tiles = no more items.  Two slots, like the phases.
     volatile int *item_info = reinterpret_cast<volatile int *>(bars + 26);
+    // The producer decodes every work item once and publishes it here for the softmax warps (two slots of
+    // 16 ints, filled an item ahead), so that decoding is not on their path between two items.
+    uint64_t *item_full = bars + 20, *item_empty = bars + 22;
+    volatile int *item_pub = reinterpret_cast<volatile int *>(bars + 32);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int n_items = kp.n_items;
@@ -496,6 +506,7 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             mbar_init(k_full + i, 1); mbar_init(k_empty + i, 1); mbar_init(v_full + i, 1); mbar_init(v_empty + i, 1);
             mbar_init(s_full + i, 1); mbar_init(o_done + i, 1); mbar_init(o_free + i, 4);
             for (int q = 0; q < kSplit; ++q) mbar_init(p_full + kSplit * i + q, 4);
+            mbar_init(item_full + i, 1); mbar_init(item_empty + i, 2 * kSplit * 2);
         }
         *abort_flag = (*reinterpret_cast<volatile int32_t *>(kp.status) == FEDATTN_ERR_TIMEOUT) ? 1 : 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -525,11 +536,29 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&map_k) : "memory");
             asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&map_v) : "memory");
         }
-        int git = 0, qn = 0;
+        int git = 0, qn = 0, pn = 0;
         for (int k = 0; k < n_rounds; ++k) {
             const int item = item_of(k);
             if (item >= n_items) continue;
             const Item it = decode_item<kSpecial>(kp, item, lane);
+            if (lane == 0) {
+                if (pn >= 2) mbar_wait(item_empty + (pn & 1), ((pn >> 1) - 1) & 1, abort_flag, kp.status);
+                volatile int *slot = item_pub + (pn & 1) * 16;
+                slot[0] = it.kvh; slot[1] = it.head0; slot[2] = it.q_row0; slot[3] = it.n_valid; slot[4] = it.seg;
+                slot[5] = it.kv_begin; slot[6] = it.n_tiles; slot[7] = it.n_a; slot[8] = it.t_b0; slot[9] = it.a;
+                slot[10] = it.b; slot[11] = it.valid1 ? 1 : 0;
+                mbar_arrive(item_full + (pn & 1));
+                if (it.n_tiles > 0) {
+                    // this item's Q on its way into L2: the load itself has to wait for the Q buffer
+                    tma_prefetch_3d(&map_q, 0, it.head0, it.q_row0);
+                    tma_prefetch_3d(&map_q, 64, it.head0, it.q_row0);
+                    if (it.valid1) {
+                        tma_prefetch_3d(&map_q, 0, it.head0 + 1, it.q_row0);
+                        tma_prefetch_3d(&map_q, 64, it.head0 + 1, it.q_row0);
+                    }
+                }
+            }
+            ++pn;
             if (it.n_tiles == 0) continue;
             if (lane == 0) {
                 if (qn > 0) mbar_wait(q_empty, (qn - 1) & 1, abort_flag, kp.status);   // previous item's S MMAs done
@@ -783,10 +812,22 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             if (tid == 0) TRACE(j, t ? 6 : 1);
         };
 
+        int pn = 0;                                             // items read from the producer's slots
         for (int k = 0; k < n_rounds; ++k) {
             const int item = item_of(k);
             if (item >= n_items) continue;
-            const Item it = decode_item<kSpecial>(kp, item, lane);
+            Item it;
+            {
+                mbar_wait(item_full + (pn & 1), (pn >> 1) & 1, abort_flag, kp.status);
+                const volatile int *slot = item_pub + (pn & 1) * 16;
+                it.kvh = slot[0]; it.head0 = slot[1]; it.q_row0 = slot[2]; it.n_valid = slot[3]; it.seg = slot[4];
+                it.kv_begin = slot[5]; it.n_tiles = slot[6]; it.n_a = slot[7]; it.t_b0 = slot[8]; it.a = slot[9];
+                it.b = slot[10]; it.valid1 = slot[11] != 0;
+                it.kvp = p.kv_pos ? p.kv_pos + (p.kv_head_major ? (int64_t)it.kvh * p.total_kv : 0) : nullptr;
+                __syncwarp();
+                if (lane == 0) mbar_arrive(item_empty + (pn & 1));
+                ++pn;
+            }
             if (t == 1 && !it.valid1) continue;                 // the pair's second head does not exist
             const int n_tiles = it.n_tiles;
             const bool valid = r < it.n_valid;
