@@ -59,7 +59,9 @@ constexpr int kProducerWarp = 4 * kSplit, kMmaWarp = 4 * kSplit + 1;
 static_assert(kSplit == 2 || kSplit == 4, "column split");
 constexpr uint32_t kTileBytes = kTileM * kD * 2;      // 32 KB: one Q, K or V tile
 constexpr uint32_t kHalfBytes = kTileBytes / 2;       // one 64-column TMA box
-constexpr uint32_t kSmemBytes = 6 * kTileBytes + 1024 /*alignment slack*/ + 256 /*barriers*/ + 256 /*published items*/;
+constexpr uint32_t kStageBytes = 32 * 128;            // output staging per softmax warp: 32 rows x 64 columns
+constexpr uint32_t kSmemBytes = 6 * kTileBytes + 1024 /*alignment slack*/ + 1024 /*barriers, published items*/ +
+                                2 * kSplit * 2 * kStageBytes;
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kColS = 0, kColO = 256;   // S (and P, aliased) of sub-tile t at kColS + 128 t; O at kColO + 128 t
 // P (bf16 pairs) of keys kCols q .. kCols q + kCols - 1 sits at S column kCols q: every 32-key chunk of P
@@ -78,6 +80,7 @@ struct KernelParams {
     int32_t n_items;                 // query tiles x KV heads x head pairs
     int32_t n_kt;                    // KV tiles: ceil(total_kv / kTileN)
     int32_t *status;
+    int32_t o_tma;                   // the output may leave through TMA stores (tensor map encoded)
 };
 
 // Position tables of a general-position call (ints, in this order): minimum and maximum position of
@@ -166,6 +169,16 @@ __device__ __forceinline__ void tma_prefetch_3d(const CUtensorMap *map, int c0, 
     asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];"
                  ::"l"((uint64_t)map), "r"(c0), "r"(c1), "r"(c2) : "memory");
 }
+
+// [32 rows x 64 columns] from shared memory (128-byte swizzle) to the output, one bulk group per call
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap *map, const void *src, int c0, int c1, int c2)
+{
+    asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4}], [%1];"
+                 ::"l"((uint64_t)map), "r"(smem_u32(src)), "r"(c0), "r"(c1), "r"(c2) : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+// the issuing thread's earlier bulk stores have read their shared memory
+__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 
 // true in exactly one lane of a converged warp
 __device__ __forceinline__ bool elect_one()
@@ -467,7 +480,8 @@ __device__ __forceinline__ Item decode_item(const KernelParams &kp, int item, in
 template <bool kSpecial>
 __global__ void __launch_bounds__(kThreads, 1)
 prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-                     const __grid_constant__ CUtensorMap map_v, const __grid_constant__ KernelParams kp)
+                     const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_o,
+                     const __grid_constant__ KernelParams kp)
 {
     extern __shared__ uint8_t smem_raw[];
     const PrefillParams &p = kp.p;
@@ -489,6 +503,7 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     // 16 ints, filled an item ahead), so that decoding is not on their path between two items.
     uint64_t *item_full = bars + 20, *item_empty = bars + 22;
     volatile int *item_pub = reinterpret_cast<volatile int *>(bars + 32);
+    uint8_t *stage = smem + 6 * kTileBytes + 1024;       // [softmax warp][32 rows][128 B], 128-byte swizzle
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int n_items = kp.n_items;
@@ -921,6 +936,14 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             mbar_wait(o_done + t, (gsub + n_tiles - 1) & 1, abort_flag, kp.status);
             tc_fence_after();
             const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
+            // Full warps of rows leave through shared memory and TMA stores (a warp's 32 rows x 64 columns at a
+            // time); a warp with rows beyond the segment writes its valid rows directly.
+            const bool by_tma = kp.o_tma && (r | 31) < it.n_valid;
+            uint8_t *my_stage = stage + (size_t)warp * kStageBytes;
+            if (by_tma) {
+                if (lane == 0) tma_store_wait_read();           // the previous item's last store has read the staging rows
+                __syncwarp();
+            }
             uint32_t oa[32], ob[32];
             FEDATTN_TMEM_LD32(tO, oa);
 #pragma unroll
@@ -934,7 +957,26 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                     __syncwarp();
                     if (lane == 0) mbar_arrive(o_free + t);     // one arrival per warp: O_t may be overwritten
                 }
-                if (valid) {
+                if (by_tma) {
+                    if (c == 2) {                               // the first half's store has read the staging rows
+                        if (lane == 0) tma_store_wait_read();
+                        __syncwarp();
+                    }
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {               // 16-byte unit 4 (c & 1) + u of the row's 128 staged bytes
+                        uint32_t w[4];
+#pragma unroll
+                        for (int i = 0; i < 4; ++i)
+                            w[i] = pack_bf16(__uint_as_float(cur[8 * u + 2 * i]) * inv, __uint_as_float(cur[8 * u + 2 * i + 1]) * inv);
+                        const int unit = 4 * (c & 1) + u;
+                        *reinterpret_cast<uint4 *>(my_stage + lane * 128 + ((unit ^ (lane & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+                    }
+                    if (c & 1) {
+                        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                        __syncwarp();
+                        if (lane == 0) tma_store_3d(&map_o, my_stage, 64 * (c >> 1), it.head0 + t, it.q_row0 + (r & ~31));
+                    }
+                } else if (valid) {
 #pragma unroll
                     for (int h2 = 0; h2 < 2; ++h2) {
                         uint32_t w[8];
@@ -955,6 +997,7 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             if (valid && lse_p) *lse_p = l_run > 0.f ? (m_run + log2f(l_run)) * 0.6931471805599453f : -INFINITY;
             gsub += n_tiles;
         }
+        if (lane == 0) tma_store_wait_read();                   // the staging rows stay alive until they are read
     }
 
     // ---- teardown -----------------------------------------------------------------------------------
@@ -1074,7 +1117,8 @@ extern "C" int fedattn_debug_read_trace(long long *host, int n)
 bool prefill_sm100_supported(const Context *ctx) { return ctx->encode_tiled != nullptr; }
 
 // [rows, heads, 128] bf16 (token-major) or [heads, rows, 128] (head-major); boxes of 64 columns x 128 rows.
-static bool encode_map(const Context *ctx, CUtensorMap *map, const void *base, int64_t rows, int heads, bool head_major)
+static bool encode_map(const Context *ctx, CUtensorMap *map, const void *base, int64_t rows, int heads, bool head_major,
+                       int box_rows = kTileN)
 {
     EncodeTiledFn fn = reinterpret_cast<EncodeTiledFn>(ctx->encode_tiled);
     cuuint64_t dims[3], strides[2];
@@ -1083,11 +1127,11 @@ static bool encode_map(const Context *ctx, CUtensorMap *map, const void *base, i
     if (head_major) {
         dims[1] = (cuuint64_t)rows; dims[2] = (cuuint64_t)heads;
         strides[0] = kD * 2; strides[1] = (cuuint64_t)rows * kD * 2;
-        box[0] = 64; box[1] = kTileN; box[2] = 1;
+        box[0] = 64; box[1] = (cuuint32_t)box_rows; box[2] = 1;
     } else {
         dims[1] = (cuuint64_t)heads; dims[2] = (cuuint64_t)rows;
         strides[0] = kD * 2; strides[1] = (cuuint64_t)heads * kD * 2;
-        box[0] = 64; box[1] = 1; box[2] = kTileN;
+        box[0] = 64; box[1] = 1; box[2] = (cuuint32_t)box_rows;
     }
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -1144,11 +1188,15 @@ cudaError_t launch_prefill_sm100(Context *ctx, const PrefillParams &p, cudaStrea
     kp.magic_ppg = magic((g + 1) / 2);
     for (int i = 0; i < kMaxP; ++i) kp.magic_small[i] = magic(i + 1);
     const int64_t blocks = items < ctx->sm_count ? items : ctx->sm_count;     // persistent: one CTA per SM
-    CUtensorMap mq, mk, mv;
+    CUtensorMap mq, mk, mv, mo;
     if (!encode_map(ctx, &mq, p.q, p.n_q_rows, p.hq, false) ||
         !encode_map(ctx, &mk, p.k, p.total_kv, p.hkv, p.kv_head_major != 0) ||
         !encode_map(ctx, &mv, p.v, p.total_kv, p.hkv, p.kv_head_major != 0))
         return cudaErrorInvalidValue;
+    // the output as [rows, heads, 128] in boxes of 32 rows x 64 columns; a base the encoder refuses (alignment)
+    // leaves the kernel on its direct stores
+    kp.o_tma = encode_map(ctx, &mo, p.o, p.n_q_rows, p.hq, false, 32) ? 1 : 0;
+    if (!kp.o_tma) mo = mq;
     static bool attr_set[64] = {};
     if (!attr_set[ctx->device & 63]) {
         cudaError_t e = cudaFuncSetAttribute(prefill_sm100_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
@@ -1171,8 +1219,8 @@ cudaError_t launch_prefill_sm100(Context *ctx, const PrefillParams &p, cudaStrea
     }
     // the plain instance serves local attention and sync attention under the prefix mask; explicit positions
     // and remote-only attention run the instance that carries their extra state
-    if (p.general || p.remote_only) prefill_sm100_kernel<true><<<(unsigned)blocks, kThreads, kSmemBytes, s>>>(mq, mk, mv, kp);
-    else prefill_sm100_kernel<false><<<(unsigned)blocks, kThreads, kSmemBytes, s>>>(mq, mk, mv, kp);
+    if (p.general || p.remote_only) prefill_sm100_kernel<true><<<(unsigned)blocks, kThreads, kSmemBytes, s>>>(mq, mk, mv, mo, kp);
+    else prefill_sm100_kernel<false><<<(unsigned)blocks, kThreads, kSmemBytes, s>>>(mq, mk, mv, mo, kp);
     ++ctx->launches;
     ++ctx->tc_launches;
     cudaError_t e = cudaGetLastError();

@@ -20,6 +20,40 @@ def gen(seed, lens, hq, hkv, d, dtype, gain=1.0):
     return w.qkv()
 
 
+def test_buffers_on_16_byte_boundaries_and_ragged_tiles(oracle):
+    """Q, K, V and O at addresses that are multiples of 16 but not of 32 bytes, with full and ragged
+    128-row tiles in one call: rows leave through both store paths (whole warps of rows in bulk, the
+    rows of a ragged warp one by one) and both must land where the layout says."""
+    lens = [256, 130, 300, 128, 17]
+    hq, hkv, d = 8, 2, 128
+    q, k, v = gen(91, lens, hq, hkv, d, "bf16")
+    L = sum(lens)
+    m = fa()
+    shape = m.Shape(len(lens), hq, hkv, d, m.BF16, 1, 0.0)
+    ctx = m.Context(shape, L, L)
+
+    def shifted(x):                       # the same values, 16 bytes further
+        flat = torch.empty(x.numel() + 8, dtype=torch.bfloat16, device="cuda")
+        view = flat[8:].view(x.shape)
+        view.copy_(x)
+        assert view.data_ptr() % 32 == 16
+        return view
+
+    qd, kd, vd = (shifted(dev(x, "bf16")) for x in (q, k, v))
+    o = shifted(torch.full_like(dev(q, "bf16"), float("nan")))
+    cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
+    m.fedattn_local(ctx, shape, qd, kd, vd, cu, o)
+    assert ctx.poll() == 0
+    oo, _ = oracle.local(q, k, v, lens)
+    check_close(host(o), oo, TOL["bf16"], "local, shifted buffers")
+    o2 = shifted(torch.full_like(dev(q, "bf16"), float("nan")))
+    m.fedattn_sync(ctx, shape, qd, None, kd, vd, None, L, False, o2)
+    assert ctx.poll() == 0
+    oo, _ = oracle.sync(q, k, v)
+    check_close(host(o2), oo, TOL["bf16"], "sync, shifted buffers")
+    assert ctx.tensor_core_launch_count() == 2
+
+
 # ---------------------------------------------------------------------------------------------
 # config 1: fp32, N=2 x 128, 4 heads, d=64 -- full comparison, local and sync
 # ---------------------------------------------------------------------------------------------
