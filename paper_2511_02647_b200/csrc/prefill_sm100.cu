@@ -156,6 +156,24 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volati
     return false;
 }
 
+// The same wait for the roles that hold few registers (producer, MMA issuer): the polling loop lives in
+// one place instead of at every call site, which keeps those roles' code short.
+__device__ __noinline__ bool mbar_wait_loop(uint64_t *bar, uint32_t parity, volatile int *abort_flag, int32_t *status)
+{
+    for (uint32_t it = 0; it < kWaitLimit; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+    }
+    *abort_flag = 1;
+    atomicMax(status, (int32_t)FEDATTN_ERR_TIMEOUT);
+    return false;
+}
+__device__ __forceinline__ bool mbar_wait_call(uint64_t *bar, uint32_t parity, volatile int *abort_flag, int32_t *status)
+{
+    if (mbar_test_wait(bar, parity)) return true;
+    return mbar_wait_loop(bar, parity, abort_flag, status);
+}
+
 __device__ __forceinline__ void tma_load_3d(void *dst, const CUtensorMap *map, uint64_t *bar, int c0, int c1, int c2)
 {
     asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
@@ -557,7 +575,7 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             if (item >= n_items) continue;
             const Item it = decode_item<kSpecial>(kp, item, lane);
             if (lane == 0) {
-                if (pn >= 2) mbar_wait(item_empty + (pn & 1), ((pn >> 1) - 1) & 1, abort_flag, kp.status);
+                if (pn >= 2) mbar_wait_call(item_empty + (pn & 1), ((pn >> 1) - 1) & 1, abort_flag, kp.status);
                 volatile int *slot = item_pub + (pn & 1) * 16;
                 slot[0] = it.kvh; slot[1] = it.head0; slot[2] = it.q_row0; slot[3] = it.n_valid; slot[4] = it.seg;
                 slot[5] = it.kv_begin; slot[6] = it.n_tiles; slot[7] = it.n_a; slot[8] = it.t_b0; slot[9] = it.a;
@@ -576,7 +594,7 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             ++pn;
             if (it.n_tiles == 0) continue;
             if (lane == 0) {
-                if (qn > 0) mbar_wait(q_empty, (qn - 1) & 1, abort_flag, kp.status);   // previous item's S MMAs done
+                if (qn > 0) mbar_wait_call(q_empty, (qn - 1) & 1, abort_flag, kp.status);   // previous item's S MMAs done
                 item_info[(qn & 1) * 2] = it.n_tiles;
                 item_info[(qn & 1) * 2 + 1] = it.valid1 ? 2 : 1;
                 mbar_expect_tx(q_full, it.valid1 ? 2 * kTileBytes : kTileBytes);
@@ -590,12 +608,12 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                     const int gt = git + j, st = gt & 1, use = gt >> 1;
                     const int row = it.kv_begin + (kSpecial ? tile_of(it, j) : j) * kTileN;
                     const int c1 = p.kv_head_major ? row : it.kvh, c2 = p.kv_head_major ? it.kvh : row;
-                    if (gt >= 2) mbar_wait(k_empty + st, (use - 1) & 1, abort_flag, kp.status);
+                    if (gt >= 2) mbar_wait_call(k_empty + st, (use - 1) & 1, abort_flag, kp.status);
                     TRACE(j, 7);
                     mbar_expect_tx(k_full + st, kTileBytes);
                     tma_load_3d(sK + st * kTileBytes, &map_k, k_full + st, 0, c1, c2);
                     tma_load_3d(sK + st * kTileBytes + kHalfBytes, &map_k, k_full + st, 64, c1, c2);
-                    if (gt >= 2) mbar_wait(v_empty + st, (use - 1) & 1, abort_flag, kp.status);
+                    if (gt >= 2) mbar_wait_call(v_empty + st, (use - 1) & 1, abort_flag, kp.status);
                     mbar_expect_tx(v_full + st, kTileBytes);
                     tma_load_3d(sV + st * kTileBytes, &map_v, v_full + st, 0, c1, c2);
                     tma_load_3d(sV + st * kTileBytes + kHalfBytes, &map_v, v_full + st, 64, c1, c2);
@@ -607,7 +625,7 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         }
         if (lane == 0) {
             // end marker for the MMA issuer, in the slot and phase the next item would have used
-            if (qn > 0) mbar_wait(q_empty, (qn - 1) & 1, abort_flag, kp.status);
+            if (qn > 0) mbar_wait_call(q_empty, (qn - 1) & 1, abort_flag, kp.status);
             item_info[(qn & 1) * 2] = -1;
             mbar_arrive(q_full);
             if (*abort_flag) {
@@ -648,11 +666,11 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         for (;;) {
             // the producer decodes the work items; this warp only learns their shape (decoding them here as
             // well does not fit into this role's 64 registers)
-            if (!mbar_wait(q_full, qn & 1, abort_flag, kp.status)) break;
+            if (!mbar_wait_call(q_full, qn & 1, abort_flag, kp.status)) break;
             const int n = item_info[(qn & 1) * 2];
             if (n < 0) break;
             const int n_sub = item_info[(qn & 1) * 2 + 1];
-            mbar_wait(k_full + (git & 1), (git >> 1) & 1, abort_flag, kp.status);
+            mbar_wait_call(k_full + (git & 1), (git >> 1) & 1, abort_flag, kp.status);
             tc_fence_after();
             for (int t = 0; t < n_sub; ++t) {
                 issue_s(t, git & 1);
@@ -665,11 +683,11 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                 const int st1 = (gt + 1) & 1, ph1 = ((gt + 1) >> 1) & 1;
                 for (int t = 0; t < n_sub; ++t) {
                     const int gsub = (t ? git1 : git) + j, qsub = t ? qn1 : qn;
-                    if (t == 0) mbar_wait(v_full + st, ph, abort_flag, kp.status);
-                    if (j == 0 && qsub > 0) mbar_wait(o_free + t, (qsub - 1) & 1, abort_flag, kp.status);
+                    if (t == 0) mbar_wait_call(v_full + st, ph, abort_flag, kp.status);
+                    if (j == 0 && qsub > 0) mbar_wait_call(o_free + t, (qsub - 1) & 1, abort_flag, kp.status);
 #pragma unroll
                     for (int q = 0; q < kSplit; ++q) {
-                        mbar_wait(p_full + kSplit * t + q, gsub & 1, abort_flag, kp.status);
+                        mbar_wait_call(p_full + kSplit * t + q, gsub & 1, abort_flag, kp.status);
                         if (lane == 0 && q == 0) TRACE(j, 2 + t);
                         tc_fence_after();
                         if (leader) {
@@ -685,7 +703,7 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                     commit(o_done + t);
                     if (t == n_sub - 1) commit(v_empty + st);
                     if (j + 1 < n) {
-                        if (t == 0) mbar_wait(k_full + st1, ph1, abort_flag, kp.status);
+                        if (t == 0) mbar_wait_call(k_full + st1, ph1, abort_flag, kp.status);
                         issue_s(t, st1);
                         commit(s_full + t);
                         if (t == n_sub - 1) {
@@ -729,7 +747,6 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         const float sl2 = p.scale * 1.4426950408889634f;
         const uint64_t sl2_2 = pack_f32x2(sl2, sl2);
         int gsub = 0;                                           // KV tiles this sub-tile has been through
-        const bool o_aligned32 = (reinterpret_cast<uintptr_t>(p.o) & 31) == 0;
         auto below32 = [](int n) -> uint32_t { return n <= 0 ? 0u : (n >= 32 ? 0xffffffffu : (1u << n) - 1u); };
 
         // One visit = the softmax of one S tile.  kPartial: some row of the tile has masked columns; bit i of
@@ -943,21 +960,19 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             if (by_tma) {
                 if (lane == 0) tma_store_wait_read();           // the previous item's last store has read the staging rows
                 __syncwarp();
-            }
-            uint32_t oa[32], ob[32];
-            FEDATTN_TMEM_LD32(tO, oa);
+                uint32_t oa[32], ob[32];
+                FEDATTN_TMEM_LD32(tO, oa);
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                uint32_t *cur = (c & 1) ? ob : oa, *nxt = (c & 1) ? oa : ob;
-                tmem_wait_ld();
-                if (c < 3) {
-                    FEDATTN_TMEM_LD32(tO + 32 * (c + 1), nxt);
-                } else {
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(o_free + t);     // one arrival per warp: O_t may be overwritten
-                }
-                if (by_tma) {
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t *cur = (c & 1) ? ob : oa, *nxt = (c & 1) ? oa : ob;
+                    tmem_wait_ld();
+                    if (c < 3) {
+                        FEDATTN_TMEM_LD32(tO + 32 * (c + 1), nxt);
+                    } else {
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(o_free + t); // one arrival per warp: O_t may be overwritten
+                    }
                     if (c == 2) {                               // the first half's store has read the staging rows
                         if (lane == 0) tma_store_wait_read();
                         __syncwarp();
@@ -976,20 +991,27 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                         __syncwarp();
                         if (lane == 0) tma_store_3d(&map_o, my_stage, 64 * (c >> 1), it.head0 + t, it.q_row0 + (r & ~31));
                     }
-                } else if (valid) {
+                }
+            } else {
+                // the rare path (a warp with rows beyond the segment) is kept short rather than fast
+#pragma unroll 1
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t o[32];
+                    FEDATTN_TMEM_LD32(tO + 32 * c, o);
+                    tmem_wait_ld();
+                    if (c == 3) {
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(o_free + t);
+                    }
+                    if (valid) {
 #pragma unroll
-                    for (int h2 = 0; h2 < 2; ++h2) {
-                        uint32_t w[8];
+                        for (int u = 0; u < 4; ++u) {
+                            uint32_t w[4];
 #pragma unroll
-                        for (int i = 0; i < 8; ++i)
-                            w[i] = pack_bf16(__uint_as_float(cur[16 * h2 + 2 * i]) * inv, __uint_as_float(cur[16 * h2 + 2 * i + 1]) * inv);
-                        __nv_bfloat16 *dst = orow + 32 * c + 16 * h2;
-                        if (o_aligned32) {
-                            asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(dst), "r"(w[0]), "r"(w[1]),
-                                         "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7]) : "memory");
-                        } else {
-                            *reinterpret_cast<uint4 *>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
-                            *reinterpret_cast<uint4 *>(dst + 8) = make_uint4(w[4], w[5], w[6], w[7]);
+                            for (int i = 0; i < 4; ++i)
+                                w[i] = pack_bf16(__uint_as_float(o[8 * u + 2 * i]) * inv, __uint_as_float(o[8 * u + 2 * i + 1]) * inv);
+                            *reinterpret_cast<uint4 *>(orow + 32 * c + 8 * u) = make_uint4(w[0], w[1], w[2], w[3]);
                         }
                     }
                 }
