@@ -5,6 +5,8 @@
 #include <cooperative_groups.h>
 #include <string.h>
 
+#include <limits.h>
+
 #include "common.cuh"
 
 namespace fedattn {
@@ -163,9 +165,16 @@ topk_fused_kernel(const PartsParams pp, int hkv, int vpr /* 16-byte vectors per 
             if (tid == 0 && my_seq > 0) atomicMax(reinterpret_cast<unsigned long long *>(done_seq), (unsigned long long)(my_seq - 1));
         }
     };
-    auto may_write = [&]() {                                  // CTA-uniform
-        if (need_seq > 0 && *reinterpret_cast<volatile long long *>(done_seq) < need_seq)
-            asm volatile("griddepcontrol.wait;" ::: "memory");
+    // The call it has to see complete is an EARLIER grid of the stream, all of whose CTAs have started (a grid
+    // starts only when every CTA of its predecessor has released it), so it ends without anything from this
+    // grid: the thread polls the context's word for a bounded time, which costs less than waiting for the
+    // whole preceding grid when several calls are in flight, and falls back to that wait.
+    auto may_write = [&]() {
+        if (need_seq <= 0) return;
+        const volatile long long *done = reinterpret_cast<volatile long long *>(done_seq);
+        if (need_seq != LLONG_MAX)
+            for (int i = 0; i < 64 && *done < need_seq; ++i) __nanosleep(256);
+        if (*done < need_seq) asm volatile("griddepcontrol.wait;" ::: "memory");
     };
     const int len = pp.off[n + 1] - pp.off[n];
     const int k = pp.cu_kv[n + 1] - pp.cu_kv[n];
@@ -505,10 +514,11 @@ cudaError_t launch_topk_fused(const PartsParams &pp, int hkv, int d, int dtype, 
         if (e != cudaSuccess) return e;
         attr_set[device & 63] = true;
     }
-    // slices per (head, participant): a power of two <= 8 (one cluster), about two CTAs per SM in total
+    // slices per (head, participant): a power of two <= 8 (one cluster), about two CTAs per SM in total, and
+    // every slice keeps at least one token per lane of the CTA (a lane walks one key row at a time)
     const int pairs = hkv * pp.n;
     int slices = 1;
-    while (slices * 2 <= kMaxSlices && pairs * slices * 2 <= sm_count) slices *= 2;
+    while (slices * 2 <= kMaxSlices && pairs * slices * 2 <= sm_count && max_len >= kSelThreads * slices * 2) slices *= 2;
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof(cfg));
     cfg.gridDim = dim3(hkv, pp.n, slices);
