@@ -172,7 +172,9 @@ topk_fused_kernel(const PartsParams pp, int hkv, int vpr /* 16-byte vectors per 
     auto may_write = [&]() {
         if (need_seq <= 0) return;
         const volatile long long *done = reinterpret_cast<volatile long long *>(done_seq);
-        if (need_seq != LLONG_MAX)
+        // (the word learns of call s from the closing CTA of a later call; when the call needed is the one
+        // directly before this one, that later call is this one, and only the wait below can tell)
+        if (need_seq != LLONG_MAX && need_seq < my_seq - 1)
             for (int i = 0; i < 64 && *done < need_seq; ++i) __nanosleep(256);
         if (*done < need_seq) asm volatile("griddepcontrol.wait;" ::: "memory");
     };
