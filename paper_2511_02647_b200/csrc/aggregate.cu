@@ -544,54 +544,115 @@ cudaError_t launch_topk_fused(const PartsParams &pp, int hkv, int d, int dtype, 
 }
 
 // ---- indexed gather ------------------------------------------------------------------------------
+// One 16-byte vector per thread and step, kGatherBatch steps in flight.  Launched with programmatic stream
+// serialization like the fused kernel above: indices and rows are read at once (unless they might be
+// outputs of a grid that is still running: early == 0), everything is written after griddepcontrol.wait.
+constexpr int kGatherBatch = 4;
+
 __global__ void __launch_bounds__(256)
 gather_kernel(const PartsParams pp, int hkv, int64_t vpr /* 16-byte vectors per (row, head) */,
               const int32_t *sel_idx, uint4 *k_agg, uint4 *v_agg, int32_t *kv_pos, int32_t *cu_kv,
-              int32_t *sel_idx_out, int32_t *status)
+              int32_t *sel_idx_out, int32_t *status, int early)
 {
+    if (!early) asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    bool waited = !early;
     const int64_t T = pp.cu_kv[pp.n];
     const int64_t total = (int64_t)hkv * T * vpr;
     const bool is_v = blockIdx.y != 0;
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
     const int64_t tid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    for (int64_t i = tid; i < total; i += stride) {
-        const int64_t rowid = i / vpr;               // h * T + t
-        const int vi = (int)(i - rowid * vpr);
-        const int h = (int)(rowid / T);
-        const int32_t t = (int32_t)(rowid - (int64_t)h * T);
-        const int n = find_segment(pp.cu_kv, pp.n, t);
-        const int32_t j = sel_idx[rowid];
-        const int32_t len = pp.off[n + 1] - pp.off[n];
-        // in range, and strictly above its predecessor inside the same (head, participant) block: the
-        // aggregate's positions must come out ascending, which the attention over it relies on
-        if (j < 0 || j >= len || (t > pp.cu_kv[n] && sel_idx[rowid - 1] >= j)) {
-            if (vi == 0) atomicMax(status, (int32_t)FEDATTN_ERR_INDEX);
-            if (j < 0 || j >= len) continue;
+    for (int64_t i0 = tid; i0 < total; i0 += stride * kGatherBatch) {
+        uint4 val[kGatherBatch];
+        int32_t idx[kGatherBatch], pos[kGatherBatch];
+        bool keep[kGatherBatch], first[kGatherBatch];
+        bool bad = false;
+#pragma unroll
+        for (int b = 0; b < kGatherBatch; ++b) {
+            const int64_t i = i0 + b * stride;
+            keep[b] = false; first[b] = false; idx[b] = 0; pos[b] = 0;
+            if (i >= total) continue;
+            const int64_t rowid = i / vpr;               // h * T + t
+            const int vi = (int)(i - rowid * vpr);
+            const int h = (int)(rowid / T);
+            const int32_t t = (int32_t)(rowid - (int64_t)h * T);
+            const int n = find_segment(pp.cu_kv, pp.n, t);
+            const int32_t j = __ldg(sel_idx + rowid);
+            const int32_t len = pp.off[n + 1] - pp.off[n];
+            // in range, and strictly above its predecessor inside the same (head, participant) block: the
+            // aggregate's positions must come out ascending, which the attention over it relies on
+            if (j < 0 || j >= len || (t > pp.cu_kv[n] && __ldg(sel_idx + rowid - 1) >= j)) {
+                bad |= vi == 0;
+                if (j < 0 || j >= len) continue;
+            }
+            const uint4 *src = reinterpret_cast<const uint4 *>(is_v ? pp.v[n] : pp.k[n]) +
+                               ((int64_t)j * hkv + h) * vpr + vi;
+            val[b] = ld_stream(src);
+            keep[b] = true; first[b] = vi == 0; idx[b] = j; pos[b] = pp.off[n] + j;
         }
-        const uint4 *src = reinterpret_cast<const uint4 *>(is_v ? pp.v[n] : pp.k[n]) +
-                           ((int64_t)j * hkv + h) * vpr + vi;
-        (is_v ? v_agg : k_agg)[i] = ld_stream(src);
-        if (vi == 0 && !is_v) {
-            if (kv_pos) kv_pos[rowid] = pp.off[n] + j;
-            if (sel_idx_out && sel_idx_out != sel_idx) sel_idx_out[rowid] = j;
+        if (!waited) {
+            asm volatile("griddepcontrol.wait;" ::: "memory");
+            waited = true;
+        }
+        if (bad) atomicMax(status, (int32_t)FEDATTN_ERR_INDEX);
+#pragma unroll
+        for (int b = 0; b < kGatherBatch; ++b) {
+            if (!keep[b]) continue;
+            const int64_t i = i0 + b * stride;
+            (is_v ? v_agg : k_agg)[i] = val[b];
+            if (first[b] && !is_v) {
+                const int64_t rowid = i / vpr;
+                if (kv_pos) kv_pos[rowid] = pos[b];
+                if (sel_idx_out && sel_idx_out != sel_idx) sel_idx_out[rowid] = idx[b];
+            }
         }
     }
-    if (!is_v && cu_kv && tid <= pp.n) cu_kv[tid] = pp.cu_kv[tid];
+    if (!is_v && cu_kv && tid <= pp.n) {
+        if (!waited) asm volatile("griddepcontrol.wait;" ::: "memory");
+        cu_kv[tid] = pp.cu_kv[tid];
+    }
 }
 
 cudaError_t launch_gather(const PartsParams &pp, int hkv, int d, int elt_bytes, const int32_t *sel_idx,
                           void *k_agg, void *v_agg, int32_t *kv_pos, int32_t *cu_kv, int32_t *sel_idx_out,
-                          int32_t *status, int sm_count, cudaStream_t s, int64_t *launches)
+                          int32_t *status, int device, int sm_count, cudaStream_t s, int64_t *launches)
 {
     const int64_t vpr = (int64_t)d * elt_bytes / 16;
-    const int64_t total = (int64_t)hkv * pp.cu_kv[pp.n] * vpr;
-    int64_t blocks = (total + 255) / 256;
-    if (blocks > (int64_t)sm_count * 16) blocks = (int64_t)sm_count * 16;
+    const int64_t T = pp.cu_kv[pp.n];
+    const int64_t total = (int64_t)hkv * T * vpr;
+    // the whole grid is resident at once (the next grid of the stream starts when every CTA of this one has)
+    int64_t blocks = (total + 256 * kGatherBatch - 1) / (256 * kGatherBatch);
+    if (blocks > (int64_t)sm_count * 3) blocks = (int64_t)sm_count * 3;
     if (blocks < 1) blocks = 1;
-    gather_kernel<<<dim3((unsigned)blocks, 2), 256, 0, s>>>(pp, hkv, vpr, sel_idx, (uint4 *)k_agg, (uint4 *)v_agg,
-                                                            kv_pos, cu_kv, sel_idx_out, status);
+    int early;
+    {
+        const size_t row_bytes = (size_t)hkv * d * elt_bytes;
+        MemRange in[2 * kMaxP + 1];
+        for (int i = 0; i < pp.n; ++i) {
+            const size_t bytes = (size_t)(pp.off[i + 1] - pp.off[i]) * row_bytes;
+            in[2 * i] = {pp.k[i], bytes};
+            in[2 * i + 1] = {pp.v[i], bytes};
+        }
+        in[2 * pp.n] = {sel_idx, (size_t)T * hkv * 4};
+        const MemRange out[5] = {{k_agg, (size_t)T * row_bytes}, {v_agg, (size_t)T * row_bytes}, {kv_pos, kv_pos ? (size_t)T * hkv * 4 : 0},
+                                 {cu_kv, cu_kv ? (size_t)(pp.n + 1) * 4 : 0},
+                                 {sel_idx_out, (sel_idx_out && sel_idx_out != sel_idx) ? (size_t)T * hkv * 4 : 0}};
+        early = early_start(device, s, in, 2 * pp.n + 1, out, 5).early ? 1 : 0;
+    }
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3((unsigned)blocks, 2, 1);
+    cfg.blockDim = dim3(256, 1, 1);
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, gather_kernel, pp, hkv, vpr, sel_idx, (uint4 *)k_agg, (uint4 *)v_agg, kv_pos, cu_kv,
+                                             sel_idx_out, status, early);
     ++*launches;
-    return cudaGetLastError();
+    return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 }  // namespace fedattn

@@ -251,7 +251,7 @@ fedattn_status fedattn_aggregate_kv(fedattn_ctx *ctx, const fedattn_shape *shape
         return err == cudaSuccess ? FEDATTN_OK : FEDATTN_ERR_CUDA;
     }
     const int32_t *sel = sel_idx_in;
-    err = launch_gather(pp, hkv, d, eb, sel, k_agg, v_agg, kv_pos, cu_kv, sel_idx_out, ctx->c.status, ctx->c.sm_count, s,
+    err = launch_gather(pp, hkv, d, eb, sel, k_agg, v_agg, kv_pos, cu_kv, sel_idx_out, ctx->c.status, ctx->c.device, ctx->c.sm_count, s,
                         &ctx->c.launches);
     return err == cudaSuccess ? FEDATTN_OK : FEDATTN_ERR_CUDA;
 }

@@ -99,7 +99,7 @@ cudaError_t launch_topk_fused(const PartsParams &pp, int hkv, int d, int dtype, 
                               int32_t *kv_pos, int32_t *cu_kv, int32_t *sel_idx_out, Context *ctx, cudaStream_t s);
 cudaError_t launch_gather(const PartsParams &pp, int hkv, int d, int elt_bytes, const int32_t *sel_idx,
                           void *k_agg, void *v_agg, int32_t *kv_pos, int32_t *cu_kv, int32_t *sel_idx_out,
-                          int32_t *status, int sm_count, cudaStream_t s, int64_t *launches);
+                          int32_t *status, int device, int sm_count, cudaStream_t s, int64_t *launches);
 
 // ---- bf16 prefill on tensor cores (tcgen05 + TMEM + TMA), head_dim 128 ------------------------
 struct PrefillParams {

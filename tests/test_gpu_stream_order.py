@@ -139,3 +139,41 @@ def test_chain_on_two_streams_with_events_and_in_a_replayed_graph(oracle):
     assert c.ctx.poll() == 0
     for i in (0, 1):
         c.check(i, og[i], lg[i], "graph replay set %d" % i)
+
+
+def test_indexed_gather_right_behind_the_selection_that_writes_its_indices(oracle):
+    """top-k per KV head (writes the kept indices) -> indexed gather with exactly those indices, back to
+    back and alternating between two input sets: the gather starts early but must not read indices the
+    selection has yet to write; its rows are the selection's own rows, bit for bit."""
+    m = fa()
+    shape = make_shape(N, HQ, HKV, D, "bf16")
+    ctx = m.Context(shape, N * L, N * L)
+    T = N * KSEL
+    bf = torch.bfloat16
+    k1 = torch.zeros((HKV, T, D), dtype=bf, device="cuda"); v1 = torch.zeros_like(k1)
+    k2 = torch.zeros_like(k1); v2 = torch.zeros_like(k1)
+    pos1 = torch.zeros((HKV, T), dtype=torch.int32, device="cuda"); pos2 = torch.zeros_like(pos1)
+    sel = torch.zeros_like(pos1); cu1 = torch.zeros((N + 1,), dtype=torch.int32, device="cuda"); cu2 = torch.zeros_like(cu1)
+    sets, want = [], []
+    for seed in (81, 82):
+        _, kp, vp = _case(seed)
+        ka, va, pa, _, _ = oracle.aggregate_topk(kp, vp, [KSEL] * N)
+        want.append((ka, va, pa))
+        sets.append(([dev(x, "bf16") for x in kp], [dev(x, "bf16") for x in vp]))
+    reps = 12
+    got_k = torch.zeros((reps, 2) + tuple(k2.shape), dtype=bf, device="cuda")
+    got_v = torch.zeros_like(got_k)
+    got_p = torch.zeros((reps, 2) + tuple(pos2.shape), dtype=torch.int32, device="cuda")
+    for r in range(reps):
+        for i in (0, 1):
+            kd, vd = sets[i]
+            m.fedattn_aggregate_kv(ctx, shape, m.AGG_TOPK_KNORM, kd, vd, [L] * N, [KSEL] * N, None, k1, v1, pos1, cu1, sel)
+            m.fedattn_aggregate_kv(ctx, shape, m.AGG_INDEXED, kd, vd, [L] * N, [KSEL] * N, sel, k2, v2, pos2, cu2, None)
+            got_k[r, i].copy_(k2); got_v[r, i].copy_(v2); got_p[r, i].copy_(pos2)
+    torch.cuda.synchronize()
+    assert ctx.poll() == 0
+    for r in range(reps):
+        for i in (0, 1):
+            assert np.array_equal(host(got_k[r, i]), want[i][0]), (r, i)
+            assert np.array_equal(host(got_v[r, i]), want[i][1]), (r, i)
+            assert np.array_equal(got_p[r, i].cpu().numpy(), want[i][2]), (r, i)
