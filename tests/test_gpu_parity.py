@@ -812,3 +812,77 @@ def test_wait_timeout_is_reported_and_the_poll_and_repeat_protocol(oracle):
     check_close(host(o), oracle.local(q, k, v, lens)[0], TOL["bf16"], "local after a polled timeout")
     with pytest.raises(m.FedAttnError):
         r.ctx.selftest_wait_timeout(0)                          # limit out of range: rejected on the host
+
+
+# ---------------------------------------------------------------------------------------------
+# seeded random shapes: every bf16 head_dim-128 path on segment lengths around the tile edges
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("seed", [1, 2, 3])
+def test_seeded_random_shapes_prefill_paths(oracle, seed):
+    """Participants, segment lengths (0, 1, around 32 / 128 / 256 / 512), group sizes (1..4, odd ones
+    included) and kept counts drawn from a seeded generator; local, dense sync, per-head and token-level
+    selection, sync over the sparse aggregate, the exchange block, the indexed gather with the selected
+    indices, and a shuffled row order through explicit positions, all against the oracle."""
+    rng = np.random.default_rng(seed)
+    for case in range(6):
+        n = int(rng.integers(1, 7))
+        lens = [int(x) for x in rng.choice([0, 1, 5, 31, 32, 33, 64, 100, 127, 128, 129, 200, 256, 257, 300, 384, 513], size=n)]
+        if sum(lens) == 0:
+            lens[0] = 7
+        hkv = int(rng.choice([1, 2, 4])); hq = hkv * int(rng.choice([1, 2, 3, 4]))
+        causal = bool(rng.integers(0, 4) != 0)
+        q, k, v = gen(int(rng.integers(1, 10**6)), lens, hq, hkv, 128, "bf16")
+        what = "seed %d case %d lens %s hq %d hkv %d causal %s: " % (seed, case, lens, hq, hkv, causal)
+        r = Runner(n, hq, hkv, 128, "bf16", sum(lens), causal=causal)
+        o, lse = r.local(q, k, v, lens)
+        oo, ol = oracle.local(q, k, v, lens, causal=causal)
+        check_close(o, oo, TOL["bf16"], what + "local"); check_close(lse, ol, LSE_TOL["bf16"], what + "local lse")
+        o, lse = r.sync(q, k, v)
+        oo, ol = oracle.sync(q, k, v, causal=causal)
+        check_close(o, oo, TOL["bf16"], what + "sync"); check_close(lse, ol, LSE_TOL["bf16"], what + "sync lse")
+        kp, vp = split(k, lens), split(v, lens)
+        ksel = [int(rng.integers(0, x + 1)) for x in lens]
+        agg = r.aggregate(fa().AGG_TOPK_KNORM, kp, vp, ksel)
+        ka, va, pos, cu, sel = oracle.aggregate_topk(kp, vp, ksel)
+        assert agg["status"] == 0 and np.array_equal(agg["sel_idx"].cpu().numpy(), sel), what + "selection"
+        assert np.array_equal(host(agg["k_agg"]), ka) and np.array_equal(host(agg["v_agg"]), va), what + "rows"
+        if sum(ksel) > 0:
+            o, lse = r.sync(q, agg["k_agg"], agg["v_agg"], agg["kv_pos"], head_major=True)
+            oo, ol = oracle.sync(q, ka, va, kv_pos=pos, kv_head_major=True, causal=causal)
+            check_close(o, oo, TOL["bf16"], what + "sparse sync"); check_close(lse, ol, LSE_TOL["bf16"], what + "sparse sync lse")
+            o, lse = r.sync_exchange(q, k, v, lens, agg)
+            oo, ol = oracle.sync_exchange(q, k, v, lens, ka, va, pos, cu, causal=causal)
+            check_close(o, oo, TOL["bf16"], what + "exchange"); check_close(lse, ol, LSE_TOL["bf16"], what + "exchange lse")
+            again = r.aggregate(fa().AGG_INDEXED, kp, vp, ksel, sel_idx_in=sel)
+            assert again["status"] == 0 and np.array_equal(host(again["k_agg"]), ka), what + "indexed"
+            assert np.array_equal(again["kv_pos"].cpu().numpy(), pos), what + "indexed positions"
+        agg = r.aggregate(fa().AGG_TOPK_TOKEN, kp, vp, ksel)
+        ka, va, pos, cu, sel = oracle.aggregate_topk_token(kp, vp, ksel)
+        assert np.array_equal(agg["sel_idx"].cpu().numpy(), sel) and np.array_equal(host(agg["k_agg"]), ka), what + "token"
+        if causal and sum(lens) > 1:
+            perm = rng.permutation(sum(lens))
+            o, lse = r.sync(q[perm], k[perm], v[perm], kv_pos=perm.astype(np.int32), q_pos=perm.astype(np.int32))
+            oo, ol = oracle.sync(q, k, v, causal=True)
+            check_close(o, oo[perm], TOL["bf16"], what + "shuffled rows"); check_close(lse, ol[perm], LSE_TOL["bf16"], what + "shuffled rows lse")
+
+
+@pytest.mark.parametrize("seed", [1, 2])
+def test_seeded_random_shapes_decode(oracle, seed):
+    rng = np.random.default_rng(100 + seed)
+    for case in range(8):
+        n = int(rng.integers(1, 9)); cap = int(rng.choice([1, 17, 64, 65, 200, 512, 1000, 3000]))
+        hkv = int(rng.choice([1, 2, 8])); hq = hkv * int(rng.choice([1, 2, 4]))
+        w = fi.Workload("d", int(rng.integers(1, 10**6)), (cap,) * n, hq, hkv, 128, "bf16")
+        _, k, v = w.qkv()
+        q = w.decode_q(0)
+        kc, vc = k.reshape(n, cap, hkv, 128), v.reshape(n, cap, hkv, 128)
+        lens = [int(rng.integers(0, cap + 1)) for _ in range(n)]
+        T = int(rng.integers(1, n * cap + 1))
+        what = "seed %d case %d n %d cap %d hq %d hkv %d: " % (seed, case, n, cap, hq, hkv)
+        r = Runner(n, hq, hkv, 128, "bf16", n * cap)
+        o, lse = r.decode(q, kc, vc, lens, False, max_kv_len=cap)
+        oo, ol = oracle.decode(q, kc, vc, lens, False)
+        check_close(o, oo, TOL["bf16"], what + "local"); check_close(lse, ol, LSE_TOL["bf16"], what + "local lse")
+        o, lse = r.decode(q, k, v, [T], True, max_kv_len=n * cap)
+        oo, ol = oracle.decode(q, k, v, [T], True)
+        check_close(o, oo, TOL["bf16"], what + "sync"); check_close(lse, ol, LSE_TOL["bf16"], what + "sync lse")
