@@ -177,3 +177,76 @@ def test_indexed_gather_right_behind_the_selection_that_writes_its_indices(oracl
             assert np.array_equal(host(got_k[r, i]), want[i][0]), (r, i)
             assert np.array_equal(host(got_v[r, i]), want[i][1]), (r, i)
             assert np.array_equal(got_p[r, i].cpu().numpy(), want[i][2]), (r, i)
+
+
+# ---------------------------------------------------------------------------------------------
+# An invariance, not a parity: a seeded random sequence of calls over shared buffers gives, bit for
+# bit, what the same sequence gives with a host synchronisation after every call.  (Each call's parity
+# with the oracle is tested elsewhere; this draws the orders in which buffers are written, read and
+# written again by calls that start early.)
+# ---------------------------------------------------------------------------------------------
+def _fa():
+    return fa()
+
+
+def _random_sequence(seed, sync_every, n_ops=60):
+    fa = _fa()
+    bf = torch.bfloat16
+    N, L, KS, HQ, HKV, D = 4, 512, 256, 8, 2, 128
+    T, KS2 = N * KS, KS // 2
+    T2 = N * KS2
+    shape = fa.Shape(N, HQ, HKV, D, fa.BF16)
+    torch.manual_seed(1234)
+    ctx = fa.Context(shape, N * L, N * L)
+    g = torch.Generator(device='cuda'); g.manual_seed(77)
+    parts = [[(torch.randn(L, HKV, D, device='cuda', generator=g).to(bf), torch.randn(L, HKV, D, device='cuda', generator=g).to(bf)) for _ in range(N)] for _ in range(2)]
+    q = torch.randn(N, HQ, D, device='cuda', generator=g).to(bf)
+    qp = torch.randn(T, HQ, D, device='cuda', generator=g).to(bf)
+    tok_k = torch.zeros(T, HKV, D, dtype=bf, device='cuda'); tok_v = torch.zeros_like(tok_k)
+    tok_pos = torch.zeros(T, dtype=torch.int32, device='cuda'); tok_cu = torch.zeros(N + 1, dtype=torch.int32, device='cuda'); tok_sel = torch.zeros(T, dtype=torch.int32, device='cuda')
+    t2_k = torch.zeros(T2, HKV, D, dtype=bf, device='cuda'); t2_v = torch.zeros_like(t2_k)
+    t2_pos = torch.zeros(T2, dtype=torch.int32, device='cuda'); t2_cu = torch.zeros(N + 1, dtype=torch.int32, device='cuda'); t2_sel = torch.zeros(T2, dtype=torch.int32, device='cuda')
+    sp_k = torch.zeros(HKV, T, D, dtype=bf, device='cuda'); sp_v = torch.zeros_like(sp_k)
+    sp_pos = torch.zeros(HKV, T, dtype=torch.int32, device='cuda'); sp_cu = torch.zeros(N + 1, dtype=torch.int32, device='cuda'); sp_sel = torch.zeros(HKV, T, dtype=torch.int32, device='cuda')
+    ix_k = torch.zeros_like(sp_k); ix_v = torch.zeros_like(sp_k); ix_pos = torch.zeros_like(sp_pos); ix_cu = torch.zeros_like(sp_cu)
+    o_dec = torch.zeros(N, HQ, D, dtype=bf, device='cuda'); lse_dec = torch.zeros(N, HQ, device='cuda')
+    o_pre = torch.zeros(T, HQ, D, dtype=bf, device='cuda')
+    lensT = torch.tensor([T], dtype=torch.int32, device='cuda'); lensT2 = torch.tensor([T2], dtype=torch.int32, device='cuda')
+    have_sel = False
+    rng = np.random.default_rng(seed)
+    log = []
+    def snap(*ts): log.append([t.clone() for t in ts])
+    for op in range(n_ops):
+        c = int(rng.integers(0, 8)); i = int(rng.integers(0, 2))
+        kd = [p[0] for p in parts[i]]; vd = [p[1] for p in parts[i]]
+        if c == 0:
+            fa.fedattn_aggregate_kv(ctx, shape, fa.AGG_TOPK_TOKEN, kd, vd, [L] * N, [KS] * N, None, tok_k, tok_v, tok_pos, tok_cu, tok_sel)
+        elif c == 1:
+            fa.fedattn_aggregate_kv(ctx, shape, fa.AGG_TOPK_KNORM, kd, vd, [L] * N, [KS] * N, None, sp_k, sp_v, sp_pos, sp_cu, sp_sel); have_sel = True
+        elif c == 2 and have_sel:
+            fa.fedattn_aggregate_kv(ctx, shape, fa.AGG_INDEXED, kd, vd, [L] * N, [KS] * N, sp_sel, ix_k, ix_v, ix_pos, ix_cu, None); snap(ix_k, ix_pos)
+        elif c == 3:
+            fa.fedattn_decode(ctx, shape, fa.DECODE_SYNC, q, tok_k, tok_v, 0, lensT, T, o_dec, lse_dec); snap(o_dec, lse_dec)
+        elif c == 4:   # second-level selection: the token-level aggregate, cut in N parts, is the input
+            k2 = [tok_k[n * KS:(n + 1) * KS] for n in range(N)]; v2 = [tok_v[n * KS:(n + 1) * KS] for n in range(N)]
+            fa.fedattn_aggregate_kv(ctx, shape, fa.AGG_TOPK_TOKEN, k2, v2, [KS] * N, [KS2] * N, None, t2_k, t2_v, t2_pos, t2_cu, t2_sel)
+        elif c == 5:
+            fa.fedattn_decode(ctx, shape, fa.DECODE_SYNC, q, t2_k, t2_v, 0, lensT2, T2, o_dec, lse_dec); snap(o_dec, lse_dec)
+        elif c == 6:   # prefill over the sparse aggregate (reads what 1 wrote), then its output feeds nothing
+            fa.fedattn_sync(ctx, shape, qp, None, sp_k, sp_v, sp_pos if have_sel else None, T, True, o_pre); snap(o_pre)
+        elif c == 7:   # local decode over the raw parts of set i laid out as caches: uses tok buffers as caches of N x KS rows
+            lens = torch.full((N,), KS, dtype=torch.int32, device='cuda')
+            fa.fedattn_decode(ctx, shape, fa.DECODE_LOCAL, q, tok_k, tok_v, KS * HKV * D, lens, KS, o_dec, lse_dec); snap(o_dec, lse_dec)
+        if sync_every: torch.cuda.synchronize()
+    torch.cuda.synchronize()
+    st = ctx.poll()
+    return log, st
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_seeded_random_call_sequences_match_their_synchronised_run(seed):
+    a, status_a = _random_sequence(seed, True)
+    b, status_b = _random_sequence(seed, False)
+    assert status_a == 0 and status_b == 0 and len(a) == len(b) and len(a) > 0
+    for n, (x, y) in enumerate(zip(a, b)):
+        assert all(torch.equal(p, r) for p, r in zip(x, y)), "snapshot %d of %d differs" % (n, len(a))
