@@ -24,8 +24,11 @@
 // issues); warp 10 checks the order of the key positions, warp 11 only fills that warpgroup, which
 // hands most of its registers to the softmax warpgroups (setmaxnreg works on whole warpgroups).
 // 2/8 of the exponentials of unmasked tiles are evaluated by a polynomial on the FMA pipe, because for
-// this tile shape the ex2 unit alone is as slow as the tensor pipe.  Every wait is bounded; on expiry
-// the CTA sets the status word, stops waiting and runs to its normal end (TMEM is always released).
+// this tile shape the ex2 unit alone is as slow as the tensor pipe.  The producer decodes every work
+// item once and publishes it through shared memory for the softmax warps; finished rows leave through
+// shared-memory staging and TMA stores (a warp with rows beyond its segment stores them directly).
+// Every wait is bounded; on expiry the CTA sets the status word, stops waiting and runs to its normal
+// end (TMEM is always released).
 #include <cuda.h>
 
 #include <stdio.h>
@@ -49,10 +52,10 @@ constexpr int kCols = kTileN / kSplit;
 constexpr int kSoftmaxThreads = 128 * kSplit;
 constexpr int kThreads = kSoftmaxThreads + 128;  // then a warpgroup holding the TMA producer warp and the MMA issuer warp
 // Registers move from that warpgroup to the softmax warpgroups once the roles split (setmaxnreg):
-// 384 threads start with 168 each.  setmaxnreg.inc waits, without limit, until the register file of
-// its scheduler (16 K registers; it hosts two softmax warps and one other warp) can give what it
-// asks for, so the split leaves room: 2 x kSoftmaxRegs + kOtherRegs <= 496 of the 512 per lane.
-// (A 200 / 112 split, which fills the file exactly, never came back from the increase.)
+// 384 threads start with 168 each, and that allocation (3 x 168 = 504 registers per lane slot of a
+// scheduler) is the pool the increases draw from.  setmaxnreg.inc waits, without limit, until the pool
+// can give what it asks for, so the split must fit into it: 2 x kSoftmaxRegs + kOtherRegs <= 504; it
+// keeps 8 spare.  (A 200 / 112 split asks for 512 per lane slot and never came back from the increase.)
 constexpr int kSoftmaxRegs = 216, kOtherRegs = 64;
 static_assert(2 * kSoftmaxRegs + kOtherRegs <= 496 && kSoftmaxRegs % 8 == 0 && kOtherRegs % 8 == 0, "register budget");
 constexpr int kProducerWarp = 4 * kSplit, kMmaWarp = 4 * kSplit + 1;
@@ -1224,6 +1227,13 @@ cudaError_t launch_prefill_sm100(Context *ctx, const PrefillParams &p, cudaStrea
         cudaError_t e = cudaFuncSetAttribute(prefill_sm100_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
         if (e == cudaSuccess)
             e = cudaFuncSetAttribute(prefill_sm100_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        // the register split inside the kernel has to fit into what the launch allocates: an increase that
+        // the CTA's pool cannot serve would wait for ever, so such a build is refused here
+        cudaFuncAttributes fa0, fa1;
+        if (e == cudaSuccess) e = cudaFuncGetAttributes(&fa0, prefill_sm100_kernel<false>);
+        if (e == cudaSuccess) e = cudaFuncGetAttributes(&fa1, prefill_sm100_kernel<true>);
+        if (e == cudaSuccess && (3 * fa0.numRegs < 2 * kSoftmaxRegs + kOtherRegs || 3 * fa1.numRegs < 2 * kSoftmaxRegs + kOtherRegs))
+            e = cudaErrorLaunchOutOfResources;
         if (e != cudaSuccess) {
             if (getenv("FEDATTN_DEBUG")) fprintf(stderr, "prefill_sm100_kernel attribute: %s\n", cudaGetErrorString(e));
             return e;
