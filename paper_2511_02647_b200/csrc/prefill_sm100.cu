@@ -424,7 +424,7 @@ __device__ __forceinline__ int prefix_len(const PrefillParams &p, const Item &it
         const int seg_len = p.cu[it.seg + 1] - p.cu[it.seg];
         return p.causal ? min(pos - p.cu[it.seg] + 1, seg_len) : seg_len;
     }
-    if (kSpecial && p.remote_only) {                   // what lies before the row's own segment
+    if (p.remote_only) {                               // what lies before the row's own segment
         const int before = p.cu[it.seg];
         return it.kvp ? count_le_warp(it.kvp, T, before - 1, lane) : min(before, T);
     }
@@ -434,7 +434,8 @@ __device__ __forceinline__ int prefix_len(const PrefillParams &p, const Item &it
 }
 
 // Called by a converged warp (all lanes get the same item).  kSpecial: the kernel instance that also
-// serves explicit positions and remote-only attention; the plain instance carries none of their state.
+// serves explicit positions and bidirectional remote-only attention (two key ranges); the plain instance
+// carries none of their state.  Causal remote-only attention is one more prefix mask: plain instance.
 template <bool kSpecial>
 __device__ __forceinline__ Item decode_item(const KernelParams &kp, int item, int lane)
 {
@@ -474,14 +475,15 @@ __device__ __forceinline__ Item decode_item(const KernelParams &kp, int item, in
         const int32_t *suf = pt.suf_min + (p.kv_head_major ? (size_t)it.kvh * kp.n_kt : 0);
         it.n_tiles = count_le_warp(suf, kp.n_kt, __ldg(pt.q_max + (it.q_row0 >> 7)), lane);
         it.n_a = it.n_tiles;
-    } else if (kSpecial && p.sync && p.remote_only) {
-        // keys [0, a) lie before the rows' segment; when bidirectional, keys [b, T) after it count too
+    } else if (p.sync && p.remote_only) {
+        // keys [0, a) lie before the rows' segment; when bidirectional (special instance only), keys [b, T)
+        // after it count too
         const int T = (int)p.total_kv, n_t = (T + kTileN - 1) / kTileN;
         it.a = prefix_len<kSpecial>(p, it, 0, lane);
         it.n_a = (it.a + kTileN - 1) / kTileN;
         it.n_tiles = it.n_a;
         it.b = T;
-        if (!p.causal) {
+        if (kSpecial && !p.causal) {
             const int after = p.cu[seg + 1];
             it.b = it.kvp ? count_le_warp(it.kvp, T, after - 1, lane) : min(after, T);
             it.t_b0 = it.b >= T ? n_t : max(it.b / kTileN, it.n_a);
@@ -888,7 +890,7 @@ prefill_sm100_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                 const int row = it.q_row0 + min(r, it.n_valid - 1);
                 p_row = p.q_pos ? __ldg(p.q_pos + row) : row;
             } else {
-                if (kSpecial && p.sync && p.remote_only) {
+                if (p.sync && p.remote_only) {
                     c_row = it.a;                               // the same for every row of the segment
                 } else if (p.sync && p.causal && it.kvp) {
                     // Sparse aggregate, row position = row index.  One cooperative search gives the keys
@@ -1251,7 +1253,7 @@ cudaError_t launch_prefill_sm100(Context *ctx, const PrefillParams &p, cudaStrea
     }
     // the plain instance serves local attention and sync attention under the prefix mask; explicit positions
     // and remote-only attention run the instance that carries their extra state
-    if (p.general || p.remote_only) prefill_sm100_kernel<true><<<(unsigned)blocks, kThreads, kSmemBytes, s>>>(mq, mk, mv, mo, kp);
+    if (p.general || (p.remote_only && !p.causal)) prefill_sm100_kernel<true><<<(unsigned)blocks, kThreads, kSmemBytes, s>>>(mq, mk, mv, mo, kp);
     else prefill_sm100_kernel<false><<<(unsigned)blocks, kThreads, kSmemBytes, s>>>(mq, mk, mv, mo, kp);
     ++ctx->launches;
     ++ctx->tc_launches;
