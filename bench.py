@@ -59,11 +59,11 @@ N_SETS = 3            # rotating input sets: ~600 MB touched per cycle, larger t
 SPARSE_RATIO_NUM, SPARSE_RATIO_DEN = 1, 4
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
 # profiles/ (None: the kernel has changed since its counters were taken)
-PREFILL_DRAM_BYTES = 366_131_000        # prefill_sm100_kernel, the three cfg2 launches the roofline covers: local 132.7 MB,
-                                        # sync 133.7 MB, sparse sync 99.7 MB (read + written)
+PREFILL_DRAM_BYTES = 365_672_000        # prefill_sm100_kernel, the three cfg2 launches the roofline covers: local 133.5 MB,
+                                        # sync 132.5 MB, sparse sync 99.7 MB (read + written)
 DECODE_DRAM_BYTES = 140_620_000         # one cfg5 call: decode_stream_kernel 138.45 MB + decode_merge_kernel 2.17 MB
                                         # (the merge reads its partials from DRAM only under the profiler's cache flush)
-TOPK_DRAM_BYTES = 42_206_000            # topk_fused_kernel, one cfg4 sparse aggregation (42.0 MB read + 0.2 MB written)
+TOPK_DRAM_BYTES = 42_223_000            # topk_fused_kernel, one cfg4 sparse aggregation (42.0 MB read + 0.2 MB written)
 NOMINAL_TENSOR, NOMINAL_HBM = 2250.0, 8000.0     # B200 spec: dense bf16 TFLOP/s, HBM3e GB/s
 MIN_REGION_S = 0.2                  # every microsecond-scale leg is timed over a region at least this long
 
