@@ -886,3 +886,40 @@ def test_seeded_random_shapes_decode(oracle, seed):
         o, lse = r.decode(q, k, v, [T], True, max_kv_len=n * cap)
         oo, ol = oracle.decode(q, k, v, [T], True)
         check_close(o, oo, TOL["bf16"], what + "sync"); check_close(lse, ol, LSE_TOL["bf16"], what + "sync lse")
+
+
+def test_indexed_gather_empty_in_place_and_sixty_four_participants(oracle):
+    """INDEXED aggregation at its edges: nothing kept at all; the kept indices given and returned in the
+    same buffer, three calls in a row; the largest participant count the interface takes."""
+    m = fa()
+    lens = [40, 7, 300]
+    _, k, v = gen(5, lens, 4, 2, 128, "bf16")
+    kp, vp = split(k, lens), split(v, lens)
+    r = Runner(3, 4, 2, 128, "bf16", sum(lens))
+    agg = r.aggregate(m.AGG_INDEXED, kp, vp, [0, 0, 0], sel_idx_in=np.zeros((2, 0), dtype=np.int32))
+    assert agg["status"] == 0 and list(agg["cu_kv"].cpu().numpy()) == [0, 0, 0, 0]
+    ksel = [10, 7, 100]
+    ka, va, pos, cu, sel = oracle.aggregate_topk(kp, vp, ksel)
+    T = sum(ksel)
+    kd, vd = [dev(x, "bf16") for x in kp], [dev(x, "bf16") for x in vp]
+    sel_d = torch.from_numpy(sel.astype(np.int32)).cuda()
+    for _ in range(3):
+        k2 = torch.zeros((2, T, 128), dtype=torch.bfloat16, device="cuda"); v2 = torch.zeros_like(k2)
+        p2 = torch.zeros((2, T), dtype=torch.int32, device="cuda"); c2 = torch.zeros(4, dtype=torch.int32, device="cuda")
+        m.fedattn_aggregate_kv(r.ctx, r.shape, m.AGG_INDEXED, kd, vd, lens, ksel, sel_d, k2, v2, p2, c2, sel_d)
+        assert r.poll() == 0
+        assert np.array_equal(host(k2), ka) and np.array_equal(host(v2), va)
+        assert np.array_equal(p2.cpu().numpy(), pos) and np.array_equal(c2.cpu().numpy(), cu)
+        assert np.array_equal(sel_d.cpu().numpy(), sel)
+    lens = [16] * 64
+    _, k, v = gen(6, lens, 2, 1, 128, "bf16")
+    kp, vp = split(k, lens), split(v, lens)
+    r = Runner(64, 2, 1, 128, "bf16", sum(lens))
+    ksel = [4] * 64
+    ka, va, pos, cu, sel = oracle.aggregate_topk(kp, vp, ksel)
+    a1 = r.aggregate(m.AGG_TOPK_KNORM, kp, vp, ksel)
+    a2 = r.aggregate(m.AGG_INDEXED, kp, vp, ksel, sel_idx_in=sel)
+    assert a1["status"] == 0 and a2["status"] == 0
+    assert np.array_equal(a1["sel_idx"].cpu().numpy(), sel) and np.array_equal(host(a1["k_agg"]), ka)
+    assert np.array_equal(host(a2["k_agg"]), ka) and np.array_equal(host(a2["v_agg"]), va)
+    assert np.array_equal(a2["kv_pos"].cpu().numpy(), pos)
